@@ -1,0 +1,165 @@
+/*
+ * dp_ghost.h -- C ABI of the DP-SGD ghost-clipping hot path for NVIDIA B200 (sm_100a).
+ *
+ * What the library computes (paper: "DP-SGD", Eq. 2 and Eq. 3; "Ghost Clipping
+ * Mechanism", Eq. 4 - Eq. 7; "Corrected Ghost Norm for Tied Embeddings", Eq. 11 - Eq. 13):
+ *
+ *   1. per-example squared gradient norms, without materialising per-example gradients,
+ *      summed over the parameter blocks handed in (Eq. 6):
+ *        linear layer      sq[i] += || G_i^T A_i ||_F^2 = sum_{t,s} (a_t.a_s)(g_t.g_s)
+ *        embedding table   sq[i] += sum_{t,s} [id_t == id_s] (g_t.g_s)
+ *        tied cross term   sq[i] += 2 <g_in_i, g_out_i>                     (Eq. 11)
+ *   2. clip coefficients  R_i = min(1, C / sqrt(sq[i]))                     (Eq. 2, Eq. 7)
+ *   3. the clipped sum    sum_i R_i g_i  per parameter tensor               (inner sum of Eq. 3)
+ *   4. Gaussian noise     out = scale * (out + sigma*C*z), z ~ N(0, I)      (Eq. 3)
+ *
+ * Conventions
+ *   - Every pointer marked [dev] is CUDA device memory of the current device, owned by the
+ *     caller; [host] is ordinary host memory.  The library never allocates, frees or
+ *     synchronises: work is enqueued on `stream` (a cudaStream_t passed as void*) and the
+ *     call returns.  Scratch comes from a caller-provided [dev] workspace whose minimum
+ *     size the matching *_ws_bytes function reports (0 means none is needed).
+ *   - Tensors are row-major with an explicit leading dimension (elements between rows).
+ *     Activations A are (B*T, d), output gradients G are (B*T, p); example i owns rows
+ *     i*T .. i*T+T-1.  dp_dtype names the storage type of A / G; accumulation is fp32.
+ *   - DP_BF16 tensors feed TMA: base pointers 16-byte aligned and leading dimensions a
+ *     multiple of 8 elements, else DP_ERR_ALIGNMENT (no slower substitute path is taken).
+ *     The logical width may be anything (V = 50257 with ld = 50264 is fine); columns past
+ *     the logical width are never read.
+ *   - Norm functions ADD into sq; the caller zeroes sq once per step.
+ *   - `dev_status` [dev, int32, may be NULL] collects device-side problems by bitwise OR:
+ *     DP_DEV_BAD_ID (a token id outside [0,V): that token is skipped) and DP_DEV_TIMEOUT
+ *     (a bounded barrier wait gave up: the launch's results are invalid).  The caller
+ *     zeroes it and reads it after its own synchronisation.
+ *   - Return value: DP_OK or an error found BEFORE anything was enqueued, except
+ *     DP_ERR_CUDA (a launch failed; see dp_last_cuda_error).  Nothing aborts or throws.
+ *   - Results are deterministic: the same inputs give bitwise-equal outputs.
+ */
+#ifndef DP_GHOST_H_
+#define DP_GHOST_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  DP_OK = 0,
+  DP_ERR_INVALID_ARG = 1,   /* null required pointer, non-positive size, bad enum, bad scalar */
+  DP_ERR_UNSUPPORTED = 2,   /* a size beyond what the kernels were built for */
+  DP_ERR_ALIGNMENT = 3,     /* pointer / leading dimension breaks the TMA rules above */
+  DP_ERR_WORKSPACE = 4,     /* ws is NULL or smaller than *_ws_bytes reports */
+  DP_ERR_CUDA = 5           /* CUDA runtime / driver error; dp_last_cuda_error() has the code */
+} dp_status;
+
+typedef enum { DP_F32 = 0, DP_BF16 = 1 } dp_dtype;
+
+/* How a linear layer's per-example norm is evaluated.  GHOST forms the two T x T Gram
+ * matrices A_i A_i^T and G_i G_i^T and their Frobenius inner product; DIRECT forms the
+ * p x d gradient tile by tile on chip (never in memory) and sums its squares.  AUTO picks
+ * DIRECT iff T*T > d*p, else GHOST. */
+typedef enum { DP_NORM_AUTO = 0, DP_NORM_GHOST = 1, DP_NORM_DIRECT = 2 } dp_norm_mode;
+
+enum { DP_DEV_BAD_ID = 1, DP_DEV_TIMEOUT = 2 };
+
+/* One linear layer d -> p as seen by the backward pass (Eq. 4: a_i and delta_i). */
+typedef struct {
+  const void* A;       /* [dev] (B*T, d) layer input */
+  int64_t lda;
+  int32_t d;
+  const void* G;       /* [dev] (B*T, p) gradient w.r.t. the layer output */
+  int64_t ldg;
+  int32_t p;
+  int32_t mode;        /* in : dp_norm_mode */
+  int32_t mode_used;   /* out: DP_NORM_GHOST or DP_NORM_DIRECT, what was enqueued */
+} dp_linear_desc;
+
+/* ---- per-example norms of linear layers (Eq. 4 - Eq. 6; LM head = a layer with p = V) ----
+ * layers [host, n_layers entries, mode_used written back]; sq [dev, B floats, +=].
+ * All layers share B, T and dt.  DP_BF16 runs on tcgen05 tensor cores, DP_F32 on fp32 FMA. */
+dp_status dp_ghost_norms(dp_linear_desc* layers, int32_t n_layers, dp_dtype dt,
+                         int32_t B, int32_t T, float* sq,
+                         void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+size_t dp_ghost_norms_ws_bytes(const dp_linear_desc* layers, int32_t n_layers, dp_dtype dt,
+                               int32_t B, int32_t T);
+
+/* ---- per-example norm of an embedding table's gradient (Eq. 4 with one-hot inputs) ----
+ * ids [dev, (B,T) int32 in [0,V)]; G [dev, (B*T, d)] gradient reaching the embedding output;
+ * first_occ [dev, (B,T) int32 or NULL]: smallest s with ids[i,s] == ids[i,t].
+ * A learned position table is the same call with ids[i,t] = t and V = T.  T <= 4096. */
+dp_status dp_embed_norms(const int32_t* ids, const void* G, int64_t ldg, dp_dtype dt,
+                         int32_t B, int32_t T, int32_t d, int32_t V, float* sq,
+                         int32_t* first_occ, void* ws, size_t ws_bytes,
+                         int32_t* dev_status, void* stream);
+size_t dp_embed_norms_ws_bytes(int32_t B, int32_t T, int32_t d);
+
+/* ---- cross term of a weight-tied embedding / LM head (Eq. 11, Eq. 13) ----
+ * Adds 2*<g_in_i, g_out_i> to sq[i], with g_in_i the (V,d) embedding gradient of example i
+ * and g_out_i = G_lm_i^T A_lm_i, through
+ *    <g_in_i, g_out_i> = sum_{t,s} G_lm[i,s,ids[i,t]] * (G_emb[i,t,:] . A_lm[i,s,:])
+ * so neither V x d matrix is formed.  cross [dev, B floats or NULL] receives the bare inner
+ * product (overwritten).  G_emb, A_lm: (B*T, d); G_lm: (B*T, V). */
+dp_status dp_tied_cross_term(const int32_t* ids, const void* G_emb, int64_t ldge,
+                             const void* A_lm, int64_t ldal, const void* G_lm, int64_t ldgl,
+                             dp_dtype dt, int32_t B, int32_t T, int32_t d, int32_t V,
+                             float* sq, float* cross, void* ws, size_t ws_bytes,
+                             int32_t* dev_status, void* stream);
+size_t dp_tied_cross_term_ws_bytes(int32_t B, int32_t T, int32_t d, int32_t V);
+
+/* ---- clip coefficients (Eq. 2, Eq. 7) ----
+ * clip[i] = min(1, C / sqrt(sq[i])), 1 when sq[i] == 0 (no stabiliser is added);
+ * norms [dev, B or NULL] receives sqrt(sq[i]).  C > 0 and finite. */
+dp_status dp_clip_factors(const float* sq, int32_t B, float C, float* clip, float* norms,
+                          void* stream);
+
+/* ---- clipped sum of a linear layer: out = beta*out + sum_i R_i G_i^T A_i  (Eq. 3) ----
+ * One GEMM with M = p, N = d, K = B*T whose K rows are scaled by R_i = min(1, C/sqrt(sq[i]))
+ * on chip.  out [dev, (p,d) fp32, leading dimension ldo] has the layout of a linear layer's
+ * weight gradient.  beta is 0 (overwrite) or 1 (accumulate).  clip [dev, B or NULL] receives
+ * R.  This replaces the re-weighted second backward pass of ghost clipping by its result. */
+dp_status dp_clip_accumulate(const void* A, int64_t lda, const void* G, int64_t ldg,
+                             dp_dtype dt, int32_t B, int32_t T, int32_t d, int32_t p,
+                             const float* sq, float C, float* clip,
+                             float* out, int64_t ldo, float beta,
+                             void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+size_t dp_clip_accumulate_ws_bytes(dp_dtype dt, int32_t B, int32_t T, int32_t d, int32_t p);
+
+/* ---- clipped sum of an embedding table: out[v,:] = beta*out[v,:] + sum_{i,t: id=v} R_i g_{i,t} ----
+ * The B*T token positions are ordered by a stable counting sort on the id, then every
+ * distinct id is reduced in that order.  perm [dev, B*T int32 or NULL] and seg [dev, V+1
+ * int32 or NULL] receive the sort: perm lists flat positions by (id, position) and
+ * seg[v] = number of positions with id < v.  With a tied head, call with beta = 1 on the
+ * matrix dp_clip_accumulate wrote for the head. */
+dp_status dp_clip_accumulate_embed(const int32_t* ids, const void* G, int64_t ldg, dp_dtype dt,
+                                   int32_t B, int32_t T, int32_t d, int32_t V,
+                                   const float* sq, float C, float* clip,
+                                   float* out, int64_t ldo, float beta,
+                                   int32_t* perm, int32_t* seg,
+                                   void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+size_t dp_clip_accumulate_embed_ws_bytes(int32_t B, int32_t T, int32_t d, int32_t V);
+
+/* ---- Gaussian mechanism: out[j] = scale * (out[j] + sigma*C*z_j)  (Eq. 3) ----
+ * z_j is a pure function of (seed, tensor_id, step, j): Philox4x32-10 with key
+ * (seed low word, seed high word) and counter (j/4 low, j/4 high, tensor_id, step); word
+ * pairs (x0,x1), (x2,x3) go through Box-Muller with u1 = ((xa>>8)+1)/2^24,
+ * u2 = (xb>>8)/2^24, giving r cos(2 pi u2) and r sin(2 pi u2) for elements 4q+{0,1} and
+ * 4q+{2,3}.  out [dev, n floats, 16-byte aligned]; scale = 1 gives the noised sum,
+ * scale = 1/|B| the full Eq. 3.  sigma >= 0, C > 0, all finite. */
+dp_status dp_add_noise(float* out, int64_t n, float sigma, float C, float scale,
+                       uint64_t seed, uint32_t tensor_id, uint32_t step, void* stream);
+
+/* ---- helpers ---- */
+const char* dp_status_string(dp_status s);
+int32_t dp_last_cuda_error(void);      /* cudaError_t / CUresult of the last DP_ERR_CUDA */
+const char* dp_version(void);
+/* Test hook: when non-zero, DP_BF16 linear-layer calls run the plain fp32-FMA kernels
+ * instead of the tensor-core ones (used to cross-check the two on the device).  Returns
+ * the previous value.  Off by default; not meant for production use. */
+int32_t dp_debug_force_fma(int32_t on);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DP_GHOST_H_ */

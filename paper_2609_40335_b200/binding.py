@@ -1,0 +1,267 @@
+"""ctypes binding of libdp_ghost.so: same names as the C ABI, argument marshalling only.
+
+Every step runs in the CUDA kernels of the shared library; PyTorch is used for device
+memory and streams.  If the library is missing or a call fails, an exception is raised --
+there is no fallback implementation.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import List, Optional, Sequence
+
+import torch
+
+DP_F32, DP_BF16 = 0, 1
+DP_NORM_AUTO, DP_NORM_GHOST, DP_NORM_DIRECT = 0, 1, 2
+DP_DEV_BAD_ID, DP_DEV_TIMEOUT = 1, 2
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libdp_ghost.so")
+_lib = None
+
+
+class DpGhostError(RuntimeError):
+    def __init__(self, status: int, where: str, detail: str = ""):
+        self.status = status
+        super().__init__(f"{where}: status {status} ({detail})")
+
+
+class _LinearDesc(C.Structure):
+    _fields_ = [("A", C.c_void_p), ("lda", C.c_int64), ("d", C.c_int32),
+                ("G", C.c_void_p), ("ldg", C.c_int64), ("p", C.c_int32),
+                ("mode", C.c_int32), ("mode_used", C.c_int32)]
+
+
+EXPORTS = ["dp_ghost_norms", "dp_ghost_norms_ws_bytes", "dp_embed_norms", "dp_embed_norms_ws_bytes",
+           "dp_tied_cross_term", "dp_tied_cross_term_ws_bytes", "dp_clip_factors",
+           "dp_clip_accumulate", "dp_clip_accumulate_ws_bytes", "dp_clip_accumulate_embed",
+           "dp_clip_accumulate_embed_ws_bytes", "dp_add_noise", "dp_status_string",
+           "dp_last_cuda_error", "dp_version", "dp_debug_force_fma"]
+
+
+def lib_path() -> str:
+    return _LIB_PATH
+
+
+def load():
+    """Load libdp_ghost.so (built by `python -m paper_2609_40335_b200.build`)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise DpGhostError(-1, "load", f"{_LIB_PATH} not found: build it first; there is no fallback")
+    L = C.CDLL(_LIB_PATH)
+    vp, i32, i64, f32, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_size_t
+    L.dp_ghost_norms.argtypes = [C.POINTER(_LinearDesc), i32, i32, i32, i32, vp, vp, sz, vp, vp]
+    L.dp_ghost_norms_ws_bytes.argtypes = [C.POINTER(_LinearDesc), i32, i32, i32, i32]
+    L.dp_ghost_norms_ws_bytes.restype = sz
+    L.dp_embed_norms.argtypes = [vp, vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, sz, vp, vp]
+    L.dp_embed_norms_ws_bytes.argtypes = [i32, i32, i32]
+    L.dp_embed_norms_ws_bytes.restype = sz
+    L.dp_tied_cross_term.argtypes = [vp, vp, i64, vp, i64, vp, i64, i32, i32, i32, i32, i32, vp, vp,
+                                     vp, sz, vp, vp]
+    L.dp_tied_cross_term_ws_bytes.argtypes = [i32, i32, i32, i32]
+    L.dp_tied_cross_term_ws_bytes.restype = sz
+    L.dp_clip_factors.argtypes = [vp, i32, f32, vp, vp, vp]
+    L.dp_clip_accumulate.argtypes = [vp, i64, vp, i64, i32, i32, i32, i32, i32, vp, f32, vp, vp, i64,
+                                     f32, vp, sz, vp, vp]
+    L.dp_clip_accumulate_ws_bytes.argtypes = [i32, i32, i32, i32, i32]
+    L.dp_clip_accumulate_ws_bytes.restype = sz
+    L.dp_clip_accumulate_embed.argtypes = [vp, vp, i64, i32, i32, i32, i32, i32, vp, f32, vp, vp, i64,
+                                           f32, vp, vp, vp, sz, vp, vp]
+    L.dp_clip_accumulate_embed_ws_bytes.argtypes = [i32, i32, i32, i32]
+    L.dp_clip_accumulate_embed_ws_bytes.restype = sz
+    L.dp_add_noise.argtypes = [vp, i64, f32, f32, f32, C.c_uint64, C.c_uint32, C.c_uint32, vp]
+    L.dp_status_string.argtypes = [i32]
+    L.dp_status_string.restype = C.c_char_p
+    L.dp_last_cuda_error.restype = i32
+    L.dp_version.restype = C.c_char_p
+    L.dp_debug_force_fma.argtypes = [i32]
+    L.dp_debug_force_fma.restype = i32
+    for name in EXPORTS:
+        fn = getattr(L, name)
+        if fn.restype is C.c_int:          # ctypes default: the dp_status functions
+            fn.restype = i32
+    _lib = L
+    return L
+
+
+def _check(st: int, where: str):
+    if st != 0:
+        L = load()
+        msg = L.dp_status_string(st).decode()
+        if st == 5:
+            msg += f", cuda error {L.dp_last_cuda_error()}"
+        raise DpGhostError(st, where, msg)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise DpGhostError(1, "marshal", "tensor is not on a CUDA device; there is no CPU path")
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return DP_F32
+    if t.dtype == torch.bfloat16:
+        return DP_BF16
+    raise DpGhostError(1, "marshal", f"unsupported dtype {t.dtype}")
+
+
+def _rows_ld(t: torch.Tensor) -> int:
+    """Leading dimension of a (..., ld) tensor whose leading axes are densely packed."""
+    if t.stride(-1) != 1:
+        raise DpGhostError(1, "marshal", "innermost stride must be 1")
+    ld = t.stride(-2)
+    if t.dim() == 3 and t.stride(0) != t.shape[1] * ld:
+        raise DpGhostError(1, "marshal", "examples must be contiguous blocks of T rows")
+    return ld
+
+
+def _ws(nbytes: int, ws: Optional[torch.Tensor], device) -> torch.Tensor:
+    if ws is not None:
+        return ws
+    return torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device)
+
+
+@dataclass
+class Linear:
+    """One linear layer d -> p: A (B,T,>=d) inputs, G (B,T,>=p) output gradients."""
+    A: torch.Tensor
+    G: torch.Tensor
+    d: Optional[int] = None
+    p: Optional[int] = None
+    mode: int = DP_NORM_AUTO
+    mode_used: int = -1
+
+
+def _descs(layers: Sequence[Linear]):
+    arr = (_LinearDesc * len(layers))()
+    for k, l in enumerate(layers):
+        arr[k].A = _ptr(l.A)
+        arr[k].lda = _rows_ld(l.A)
+        arr[k].d = l.d if l.d is not None else l.A.shape[-1]
+        arr[k].G = _ptr(l.G)
+        arr[k].ldg = _rows_ld(l.G)
+        arr[k].p = l.p if l.p is not None else l.G.shape[-1]
+        arr[k].mode = l.mode
+        arr[k].mode_used = -1
+    return arr
+
+
+def dp_ghost_norms_ws_bytes(layers: Sequence[Linear], B: int, T: int) -> int:
+    L = load()
+    return int(L.dp_ghost_norms_ws_bytes(_descs(layers), len(layers), _dt(layers[0].A), B, T))
+
+
+def dp_ghost_norms(layers: Sequence[Linear], B: int, T: int, sq: torch.Tensor, ws=None,
+                   dev_status=None, stream=None) -> List[int]:
+    """sq[i] += ||G_i^T A_i||_F^2 for every layer; returns the mode each layer ran in."""
+    L = load()
+    arr = _descs(layers)
+    dt = _dt(layers[0].A)
+    need = int(L.dp_ghost_norms_ws_bytes(arr, len(layers), dt, B, T))
+    ws = _ws(need, ws, sq.device)
+    st = L.dp_ghost_norms(arr, len(layers), dt, B, T, _ptr(sq), _ptr(ws), ws.numel() * ws.element_size(),
+                          _ptr(dev_status), _stream(stream))
+    _check(st, "dp_ghost_norms")
+    used = [int(arr[k].mode_used) for k in range(len(layers))]
+    for l, u in zip(layers, used):
+        l.mode_used = u
+    return used
+
+
+def dp_embed_norms(ids: torch.Tensor, G: torch.Tensor, V: int, sq: torch.Tensor, d=None,
+                   first_occ=None, ws=None, dev_status=None, stream=None):
+    L = load()
+    B, T = ids.shape
+    d = d if d is not None else G.shape[-1]
+    need = int(L.dp_embed_norms_ws_bytes(B, T, d))
+    ws = _ws(need, ws, sq.device)
+    st = L.dp_embed_norms(_ptr(ids), _ptr(G), _rows_ld(G), _dt(G), B, T, d, V, _ptr(sq),
+                          _ptr(first_occ), _ptr(ws), ws.numel() * ws.element_size(),
+                          _ptr(dev_status), _stream(stream))
+    _check(st, "dp_embed_norms")
+
+
+def dp_tied_cross_term(ids, G_emb, A_lm, G_lm, V: int, sq=None, cross=None, d=None, ws=None,
+                       dev_status=None, stream=None):
+    L = load()
+    B, T = ids.shape
+    d = d if d is not None else G_emb.shape[-1]
+    need = int(L.dp_tied_cross_term_ws_bytes(B, T, d, V))
+    dev = G_emb.device
+    ws = _ws(need, ws, dev)
+    st = L.dp_tied_cross_term(_ptr(ids), _ptr(G_emb), _rows_ld(G_emb), _ptr(A_lm), _rows_ld(A_lm),
+                              _ptr(G_lm), _rows_ld(G_lm), _dt(G_emb), B, T, d, V, _ptr(sq),
+                              _ptr(cross), _ptr(ws), ws.numel() * ws.element_size(),
+                              _ptr(dev_status), _stream(stream))
+    _check(st, "dp_tied_cross_term")
+
+
+def dp_clip_factors(sq: torch.Tensor, C_: float, clip=None, norms=None, stream=None):
+    L = load()
+    _check(L.dp_clip_factors(_ptr(sq), sq.numel(), float(C_), _ptr(clip), _ptr(norms), _stream(stream)),
+           "dp_clip_factors")
+
+
+def dp_clip_accumulate_ws_bytes(dt: int, B: int, T: int, d: int, p: int) -> int:
+    return int(load().dp_clip_accumulate_ws_bytes(dt, B, T, d, p))
+
+
+def dp_clip_accumulate(A, G, sq, C_: float, out, beta: float = 0.0, d=None, p=None, clip=None,
+                       ws=None, dev_status=None, stream=None):
+    """out (p,d) = beta*out + sum_i min(1, C/sqrt(sq[i])) * G_i^T A_i."""
+    L = load()
+    B, T = A.shape[0], A.shape[1]
+    d = d if d is not None else A.shape[-1]
+    p = p if p is not None else G.shape[-1]
+    dt = _dt(A)
+    need = int(L.dp_clip_accumulate_ws_bytes(dt, B, T, d, p))
+    ws = _ws(need, ws, out.device)
+    st = L.dp_clip_accumulate(_ptr(A), _rows_ld(A), _ptr(G), _rows_ld(G), dt, B, T, d, p, _ptr(sq),
+                              float(C_), _ptr(clip), _ptr(out), out.stride(0), float(beta), _ptr(ws),
+                              ws.numel() * ws.element_size(), _ptr(dev_status), _stream(stream))
+    _check(st, "dp_clip_accumulate")
+
+
+def dp_clip_accumulate_embed(ids, G, V: int, sq, C_: float, out, beta: float = 0.0, d=None,
+                             clip=None, perm=None, seg=None, ws=None, dev_status=None, stream=None):
+    L = load()
+    B, T = ids.shape
+    d = d if d is not None else G.shape[-1]
+    need = int(L.dp_clip_accumulate_embed_ws_bytes(B, T, d, V))
+    ws = _ws(need, ws, out.device)
+    st = L.dp_clip_accumulate_embed(_ptr(ids), _ptr(G), _rows_ld(G), _dt(G), B, T, d, V, _ptr(sq),
+                                    float(C_), _ptr(clip), _ptr(out), out.stride(0), float(beta),
+                                    _ptr(perm), _ptr(seg), _ptr(ws), ws.numel() * ws.element_size(),
+                                    _ptr(dev_status), _stream(stream))
+    _check(st, "dp_clip_accumulate_embed")
+
+
+def dp_add_noise(out: torch.Tensor, sigma: float, C_: float, scale: float, seed: int,
+                 tensor_id: int, step: int, n=None, stream=None):
+    """out = scale * (out + sigma*C*z) in place, z from the (seed, tensor_id, step) stream."""
+    L = load()
+    n = out.numel() if n is None else n
+    st = L.dp_add_noise(_ptr(out), n, float(sigma), float(C_), float(scale), int(seed) & (2 ** 64 - 1),
+                        int(tensor_id), int(step), _stream(stream))
+    _check(st, "dp_add_noise")
+
+
+def dp_debug_force_fma(on: bool) -> bool:
+    return bool(load().dp_debug_force_fma(1 if on else 0))
+
+
+def dp_version() -> str:
+    return load().dp_version().decode()

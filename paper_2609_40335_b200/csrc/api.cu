@@ -1,0 +1,319 @@
+// extern "C" entry points: argument checks, work planning, workspace carving, launches.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+
+#include "dp_common.cuh"
+#include "fma_kernels.cuh"
+#include "gemm_gta.cuh"
+#include "ghost_plan.cuh"
+
+namespace dpg {
+
+int g_last_cuda_error = 0;
+int g_force_fma = 0;
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+      n = v;
+    else
+      return 148;          // B200; not cached so a later call can still query the device
+  }
+  return n;
+}
+
+// ---- planning of dp_ghost_norms ------------------------------------------------------------
+GhostPlan plan_ghost_norms(const dp_linear_desc* layers, int n_layers, int B, int T, int sms) {
+  GhostPlan plan;
+  const int nt = ceil_div(T, 128);
+  plan.ntp = nt * (nt + 1) / 2;
+  plan.layer.resize(n_layers);
+  plan.direct.resize(n_layers);
+  plan.mode_used.resize(n_layers);
+  for (int l = 0; l < n_layers; ++l) {
+    int mode = layers[l].mode;
+    if (mode == DP_NORM_AUTO)
+      mode = ((long long)T * T > (long long)layers[l].d * layers[l].p) ? DP_NORM_DIRECT : DP_NORM_GHOST;
+    plan.mode_used[l] = mode;
+    (mode == DP_NORM_GHOST ? plan.ghost_layers : plan.direct_layers).push_back(l);
+  }
+  // Column chunking of wide operands.  The per-item step budget shrinks until there are at
+  // least two items per SM (or the budget bottoms out).
+  int budget = 64;
+  for (;;) {
+    long long items = 0;
+    for (int l : plan.ghost_layers) {
+      GhostLayerPlan& L = plan.layer[l];
+      L.a_steps = ceil_div(layers[l].d, 64);
+      L.g_steps = ceil_div(layers[l].p, 64);
+      const int small = std::min(L.a_steps, L.g_steps), large = std::max(L.a_steps, L.g_steps);
+      L.split_on_g = L.g_steps >= L.a_steps;
+      int chunk = std::max(std::max(budget - small, small), 8);
+      if (small + large <= budget + budget / 2) chunk = large;
+      L.nsplit = ceil_div(large, chunk);
+      L.chunk_steps = ceil_div(large, L.nsplit);
+      L.nsplit = ceil_div(large, L.chunk_steps);
+      items += (long long)B * plan.ntp * L.nsplit;
+    }
+    if (items >= 2LL * sms || budget <= 8 || plan.ghost_layers.empty()) break;
+    budget /= 2;
+  }
+  int col = 0;
+  for (int l = 0; l < n_layers; ++l) {
+    if (plan.mode_used[l] == DP_NORM_GHOST) {
+      plan.layer[l].col_begin = col;
+      plan.layer[l].item_begin = 0;
+      col += plan.ntp * plan.layer[l].nsplit;
+    } else {
+      plan.direct[l].tiles_m = ceil_div(layers[l].p, 128);
+      plan.direct[l].tiles_n = ceil_div(layers[l].d, 256);
+      plan.direct[l].col_begin = col;
+      col += plan.direct[l].tiles_m * plan.direct[l].tiles_n;
+    }
+  }
+  plan.n_per = col;
+  return plan;
+}
+
+static bool finite_pos(float x) { return std::isfinite(x) && x > 0.f; }
+
+static dp_status check_linear(const dp_linear_desc& L, dp_dtype dt, bool tc) {
+  if (!L.A || !L.G || L.d <= 0 || L.p <= 0 || L.lda < L.d || L.ldg < L.p) return DP_ERR_INVALID_ARG;
+  if (L.mode != DP_NORM_AUTO && L.mode != DP_NORM_GHOST && L.mode != DP_NORM_DIRECT)
+    return DP_ERR_INVALID_ARG;
+  if (tc && (!aligned16(L.A) || !aligned16(L.G) || (L.lda % 8) || (L.ldg % 8))) return DP_ERR_ALIGNMENT;
+  (void)dt;
+  return DP_OK;
+}
+
+}  // namespace dpg
+
+using namespace dpg;
+
+extern "C" {
+
+const char* dp_status_string(dp_status s) {
+  switch (s) {
+    case DP_OK: return "ok";
+    case DP_ERR_INVALID_ARG: return "invalid argument";
+    case DP_ERR_UNSUPPORTED: return "size not supported by the built kernels";
+    case DP_ERR_ALIGNMENT: return "pointer or leading dimension not aligned for TMA";
+    case DP_ERR_WORKSPACE: return "workspace missing or too small";
+    case DP_ERR_CUDA: return "CUDA error (see dp_last_cuda_error)";
+  }
+  return "unknown status";
+}
+
+int32_t dp_last_cuda_error(void) { return g_last_cuda_error; }
+const char* dp_version(void) { return "dp_ghost 0.1.0 (sm_100a)"; }
+int32_t dp_debug_force_fma(int32_t on) {
+  const int prev = g_force_fma;
+  g_force_fma = on ? 1 : 0;
+  return prev;
+}
+
+// ---------------------------------------------------------------------------- ghost norms
+size_t dp_ghost_norms_ws_bytes(const dp_linear_desc* layers, int32_t n_layers, dp_dtype dt,
+                               int32_t B, int32_t T) {
+  if (!layers || n_layers <= 0 || B <= 0 || T <= 0) return 0;
+  if (dt == DP_F32 || g_force_fma) return 0;
+  const GhostPlan plan = plan_ghost_norms(layers, n_layers, B, T, sm_count());
+  return align_up(size_t(B) * plan.n_per * sizeof(float), 256);
+}
+
+dp_status dp_ghost_norms(dp_linear_desc* layers, int32_t n_layers, dp_dtype dt, int32_t B,
+                         int32_t T, float* sq, void* ws, size_t ws_bytes, int32_t* dev_status,
+                         void* stream) {
+  if (!layers || n_layers <= 0 || B <= 0 || T <= 0 || !sq) return DP_ERR_INVALID_ARG;
+  if (dt != DP_F32 && dt != DP_BF16) return DP_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const bool tc = (dt == DP_BF16) && !g_force_fma;
+  for (int l = 0; l < n_layers; ++l) {
+    const dp_status s = check_linear(layers[l], dt, tc);
+    if (s != DP_OK) return s;
+  }
+  const GhostPlan plan = plan_ghost_norms(layers, n_layers, B, T, sm_count());
+  if (!tc) {
+    for (int l = 0; l < n_layers; ++l) {
+      const dp_status s = launch_norms_fma(layers[l], dt, plan.mode_used[l], B, T, sq, st);
+      if (s != DP_OK) return s;
+      layers[l].mode_used = plan.mode_used[l];
+    }
+    return DP_OK;
+  }
+  const size_t need = align_up(size_t(B) * plan.n_per * sizeof(float), 256);
+  if (!ws || ws_bytes < need) return DP_ERR_WORKSPACE;
+  float* partials = static_cast<float*>(ws);
+  dp_status s = DP_OK;
+  if (!plan.ghost_layers.empty()) {
+    s = launch_ghost_norm_tc(layers, plan, B, T, partials, dev_status, st);
+    if (s != DP_OK) return s;
+  }
+  if (!plan.direct_layers.empty()) {
+    s = launch_direct_norm_tc(layers, plan, B, T, partials, dev_status, st);
+    if (s != DP_OK) return s;
+  }
+  s = launch_reduce_partials(partials, plan.n_per, B, sq, 1.f, nullptr, st);
+  if (s != DP_OK) return s;
+  for (int l = 0; l < n_layers; ++l) layers[l].mode_used = plan.mode_used[l];
+  return DP_OK;
+}
+
+// ------------------------------------------------------------------------ embedding norms
+size_t dp_embed_norms_ws_bytes(int32_t B, int32_t T, int32_t d) {
+  if (B <= 0 || T <= 0 || d <= 0) return 0;
+  return align_up(size_t(B) * ceil_div(d, kEmbedColsPerBlock) * sizeof(float), 256);
+}
+
+dp_status dp_embed_norms(const int32_t* ids, const void* G, int64_t ldg, dp_dtype dt, int32_t B,
+                         int32_t T, int32_t d, int32_t V, float* sq, int32_t* first_occ, void* ws,
+                         size_t ws_bytes, int32_t* dev_status, void* stream) {
+  if (!ids || !G || !sq || B <= 0 || T <= 0 || d <= 0 || V <= 0 || ldg < d) return DP_ERR_INVALID_ARG;
+  if (dt != DP_F32 && dt != DP_BF16) return DP_ERR_INVALID_ARG;
+  if (T > kEmbedMaxT) return DP_ERR_UNSUPPORTED;
+  if (!ws || ws_bytes < dp_embed_norms_ws_bytes(B, T, d)) return DP_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  float* partials = static_cast<float*>(ws);
+  dp_status s = launch_embed_norms(ids, G, ldg, dt, B, T, d, V, partials, first_occ, dev_status, st);
+  if (s != DP_OK) return s;
+  return launch_reduce_partials(partials, ceil_div(d, kEmbedColsPerBlock), B, sq, 1.f, nullptr, st);
+}
+
+// ------------------------------------------------------------------------ tied cross term
+size_t dp_tied_cross_term_ws_bytes(int32_t B, int32_t T, int32_t d, int32_t V) {
+  (void)d; (void)V;
+  if (B <= 0 || T <= 0) return 0;
+  return align_up(size_t(B) * ceil_div(T, 16) * sizeof(float), 256);
+}
+
+dp_status dp_tied_cross_term(const int32_t* ids, const void* G_emb, int64_t ldge, const void* A_lm,
+                             int64_t ldal, const void* G_lm, int64_t ldgl, dp_dtype dt, int32_t B,
+                             int32_t T, int32_t d, int32_t V, float* sq, float* cross, void* ws,
+                             size_t ws_bytes, int32_t* dev_status, void* stream) {
+  if (!ids || !G_emb || !A_lm || !G_lm || B <= 0 || T <= 0 || d <= 0 || V <= 0)
+    return DP_ERR_INVALID_ARG;
+  if (!sq && !cross) return DP_ERR_INVALID_ARG;
+  if (ldge < d || ldal < d || ldgl < V) return DP_ERR_INVALID_ARG;
+  if (dt != DP_F32 && dt != DP_BF16) return DP_ERR_INVALID_ARG;
+  if (!ws || ws_bytes < dp_tied_cross_term_ws_bytes(B, T, d, V)) return DP_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  float* partials = static_cast<float*>(ws);
+  dp_status s = launch_cross_term_fma(ids, G_emb, ldge, A_lm, ldal, G_lm, ldgl, dt, B, T, d, V,
+                                      partials, dev_status, st);
+  if (s != DP_OK) return s;
+  return launch_reduce_partials(partials, ceil_div(T, 16), B, sq, 2.f, cross, st);
+}
+
+// --------------------------------------------------------------------------- clip factors
+dp_status dp_clip_factors(const float* sq, int32_t B, float C, float* clip, float* norms,
+                          void* stream) {
+  if (!sq || B <= 0 || (!clip && !norms) || !finite_pos(C)) return DP_ERR_INVALID_ARG;
+  return launch_clip_factors(sq, B, C, clip, norms, (cudaStream_t)stream);
+}
+
+// ------------------------------------------------------------------------ clip accumulate
+size_t dp_clip_accumulate_ws_bytes(dp_dtype dt, int32_t B, int32_t T, int32_t d, int32_t p) {
+  if (B <= 0 || T <= 0 || d <= 0 || p <= 0) return 0;
+  size_t n = align_up(size_t(B) * sizeof(float), 256);          // clip factors
+  if (dt == DP_BF16 && !g_force_fma) n += gta_partial_bytes(B, T, d, p, sm_count());
+  return n;
+}
+
+dp_status dp_clip_accumulate(const void* A, int64_t lda, const void* G, int64_t ldg, dp_dtype dt,
+                             int32_t B, int32_t T, int32_t d, int32_t p, const float* sq, float C,
+                             float* clip, float* out, int64_t ldo, float beta, void* ws,
+                             size_t ws_bytes, int32_t* dev_status, void* stream) {
+  if (!A || !G || !sq || !out || B <= 0 || T <= 0 || d <= 0 || p <= 0) return DP_ERR_INVALID_ARG;
+  if (lda < d || ldg < p || ldo < d) return DP_ERR_INVALID_ARG;
+  if (dt != DP_F32 && dt != DP_BF16) return DP_ERR_INVALID_ARG;
+  if (!(beta == 0.f || beta == 1.f) || !finite_pos(C)) return DP_ERR_INVALID_ARG;
+  const bool tc = (dt == DP_BF16) && !g_force_fma;
+  if (tc && (!aligned16(A) || !aligned16(G) || (lda % 8) || (ldg % 8))) return DP_ERR_ALIGNMENT;
+  if (!ws || ws_bytes < dp_clip_accumulate_ws_bytes(dt, B, T, d, p)) return DP_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  float* clip_ws = static_cast<float*>(ws);
+  dp_status s = launch_clip_factors(sq, B, C, clip_ws, nullptr, st);
+  if (s != DP_OK) return s;
+  if (clip) DP_CUDA_OK(cudaMemcpyAsync(clip, clip_ws, size_t(B) * sizeof(float),
+                                       cudaMemcpyDeviceToDevice, st));
+  if (!tc)
+    return launch_clip_accumulate_fma(A, lda, G, ldg, dt, B, T, d, p, clip_ws, out, ldo, beta, st);
+  float* partial = reinterpret_cast<float*>(static_cast<char*>(ws) +
+                                            align_up(size_t(B) * sizeof(float), 256));
+  return launch_clip_accumulate_tc(A, lda, G, ldg, B, T, d, p, clip_ws, out, ldo, beta, partial,
+                                   dev_status, st);
+}
+
+// ------------------------------------------------------------------ clip accumulate, embedding
+static void embed_ws_layout(int B, int T, int V, size_t* off_clip, size_t* off_counts,
+                            size_t* off_seg, size_t* off_perm, size_t* total, int* chunks) {
+  const size_t n = size_t(B) * T;
+  *chunks = int((n + kSortChunk - 1) / kSortChunk);
+  size_t o = 0;
+  *off_clip = o;   o += align_up(size_t(B) * sizeof(float), 256);
+  *off_counts = o; o += align_up(size_t(*chunks) * V * sizeof(int), 256);
+  *off_seg = o;    o += align_up(size_t(V + 1) * sizeof(int), 256);
+  *off_perm = o;   o += align_up(n * sizeof(int), 256);
+  *total = o;
+}
+
+size_t dp_clip_accumulate_embed_ws_bytes(int32_t B, int32_t T, int32_t d, int32_t V) {
+  (void)d;
+  if (B <= 0 || T <= 0 || V <= 0) return 0;
+  size_t a, b, c, e, total; int chunks;
+  embed_ws_layout(B, T, V, &a, &b, &c, &e, &total, &chunks);
+  return total;
+}
+
+dp_status dp_clip_accumulate_embed(const int32_t* ids, const void* G, int64_t ldg, dp_dtype dt,
+                                   int32_t B, int32_t T, int32_t d, int32_t V, const float* sq,
+                                   float C, float* clip, float* out, int64_t ldo, float beta,
+                                   int32_t* perm, int32_t* seg, void* ws, size_t ws_bytes,
+                                   int32_t* dev_status, void* stream) {
+  if (!ids || !G || !sq || !out || B <= 0 || T <= 0 || d <= 0 || V <= 0) return DP_ERR_INVALID_ARG;
+  if (ldg < d || ldo < d) return DP_ERR_INVALID_ARG;
+  if (dt != DP_F32 && dt != DP_BF16) return DP_ERR_INVALID_ARG;
+  if (!(beta == 0.f || beta == 1.f) || !finite_pos(C)) return DP_ERR_INVALID_ARG;
+  if ((long long)B * T > 0x7fffffffLL) return DP_ERR_UNSUPPORTED;
+  size_t o_clip, o_counts, o_seg, o_perm, total; int chunks;
+  embed_ws_layout(B, T, V, &o_clip, &o_counts, &o_seg, &o_perm, &total, &chunks);
+  if (!ws || ws_bytes < total) return DP_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  char* w = static_cast<char*>(ws);
+  float* clip_ws = reinterpret_cast<float*>(w + o_clip);
+  EmbedSortWs sw;
+  sw.counts = reinterpret_cast<int*>(w + o_counts);
+  sw.seg = reinterpret_cast<int*>(w + o_seg);
+  sw.perm = reinterpret_cast<int*>(w + o_perm);
+  sw.block_sums = nullptr;
+  sw.chunks = chunks;
+  const int n = B * T;
+  dp_status s = launch_clip_factors(sq, B, C, clip_ws, nullptr, st);
+  if (s != DP_OK) return s;
+  if (clip) DP_CUDA_OK(cudaMemcpyAsync(clip, clip_ws, size_t(B) * sizeof(float),
+                                       cudaMemcpyDeviceToDevice, st));
+  s = launch_embed_sort(ids, n, V, sw, dev_status, st);
+  if (s != DP_OK) return s;
+  if (perm) DP_CUDA_OK(cudaMemcpyAsync(perm, sw.perm, size_t(n) * sizeof(int),
+                                       cudaMemcpyDeviceToDevice, st));
+  if (seg) DP_CUDA_OK(cudaMemcpyAsync(seg, sw.seg, size_t(V + 1) * sizeof(int),
+                                      cudaMemcpyDeviceToDevice, st));
+  return launch_embed_scatter(ids, G, ldg, dt, n, T, d, V, clip_ws, sw.perm, sw.seg, out, ldo, beta,
+                              st);
+}
+
+// ----------------------------------------------------------------------------------- noise
+dp_status dp_add_noise(float* out, int64_t n, float sigma, float C, float scale, uint64_t seed,
+                       uint32_t tensor_id, uint32_t step, void* stream) {
+  if (!out || n < 0) return DP_ERR_INVALID_ARG;
+  if (!std::isfinite(sigma) || sigma < 0.f || !finite_pos(C) || !std::isfinite(scale))
+    return DP_ERR_INVALID_ARG;
+  if (!aligned16(out)) return DP_ERR_ALIGNMENT;
+  return launch_add_noise(out, n, sigma * C, scale, seed, tensor_id, step, (cudaStream_t)stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,36 @@
+// Declarations for the tensor-core G^T A kernels (clipped sum and DIRECT per-example norm).
+#pragma once
+
+#include "dp_common.cuh"
+#include "ghost_plan.cuh"
+
+namespace dpg {
+
+constexpr int kGtaMaxLayers = 80;       // layers per launch (parameter-block limit)
+
+// Plain data: copied into kernel parameters.
+struct GtaLayer {
+  float* out;             // (M, N) destination when the K range is not split
+  float* partial;         // [nsplit][M][N] planes when it is
+  long long ldo;
+  int M, N;               // p, d
+  int tiles_m, tiles_n;   // 128 x 256 output tiles
+  int nsplit;
+  int ksteps_per_split;
+  int item_begin;
+  int col_begin;          // square-sum mode: first partial-sum column of this layer
+  float beta;
+};
+
+int gta_choose_nsplit(int B, int T, int d, int p, int sms);
+size_t gta_partial_bytes(int B, int T, int d, int p, int sms);
+
+dp_status launch_clip_accumulate_tc(const void* A, int64_t lda, const void* G, int64_t ldg, int B,
+                                    int T, int d, int p, const float* clip, float* out,
+                                    int64_t ldo, float beta, float* partial_ws, int* dev_status,
+                                    cudaStream_t st);
+
+dp_status launch_direct_norm_tc(const dp_linear_desc* layers, const GhostPlan& plan, int B, int T,
+                                float* partials, int* dev_status, cudaStream_t st);
+
+}  // namespace dpg

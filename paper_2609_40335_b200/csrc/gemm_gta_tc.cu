@@ -1,0 +1,436 @@
+// G^T A on tcgen05 tensor cores: the contraction over tokens shared by
+//   (a) the clipped gradient sum  out = beta*out + sum_i R_i G_i^T A_i   (inner sum of Eq. 3,
+//       R_i of Eq. 7), one GEMM with M = p, N = d, K = B*T whose K rows carry R_i, and
+//   (b) the DIRECT per-example norm  || G_i^T A_i ||_F^2  (Eq. 4 summed over tokens), where
+//       each 128 x 256 tile of the p x d gradient lives only in tensor memory and the
+//       epilogue sums its squares.
+//
+// Both operands are contiguous along M / N (token rows are the K dimension), so shared
+// memory holds MN-major tiles: every TMA box is 64 token rows x 64 columns (128-byte rows,
+// 128-byte swizzle).  A K step never straddles two examples (the tensor map is 3-D:
+// column, token, example; the token tail of an example is zero-filled), so one clip factor
+// applies to a whole stage: four "scaler" warps multiply the G tile by R_i in shared memory
+// (fp32 multiply, bf16 round) between the TMA-full and MMA-ready barriers.
+//
+// Roles per CTA (320 threads): warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 scalers,
+// warps 6-9 epilogue; two TMEM accumulators overlap the epilogue with the next tile.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <algorithm>
+#include <cstring>
+
+#include "dp_common.cuh"
+#include "gemm_gta.cuh"
+#include "ptx_sm100.cuh"
+#include "tma_host.cuh"
+
+namespace dpg {
+
+namespace {
+
+constexpr int kBM = 128, kBN = 256, kBK = 64;
+constexpr int kBoxBytes = 64 * 128;                 // 64 token rows x 128 bytes
+constexpr int kGBytes = (kBM / 64) * kBoxBytes;     // 16 KiB
+constexpr int kABytes = (kBN / 64) * kBoxBytes;     // 32 KiB
+constexpr int kStageBytes = kGBytes + kABytes;      // 48 KiB
+constexpr int kStages = 4;
+constexpr int kThreads = 320;
+constexpr int kTmemCols = 512;                      // 2 accumulators x 256 columns
+constexpr size_t kSmemBytes = size_t(kStages) * kStageBytes + 1024 + 256;
+
+struct __align__(64) GtaParams {
+  CUtensorMap tmG[kGtaMaxLayers];
+  CUtensorMap tmA[kGtaMaxLayers];
+  GtaLayer layer[kGtaMaxLayers];
+  int n_layers;
+  int B, T, tsteps;          // tsteps = ceil(T / 64) K steps per example
+  int total_items;
+  const float* clip;         // [B] R_i (scale mode)
+  float* sq_partials;        // [B][n_per] (square-sum mode)
+  int n_per;
+  int* dev_status;
+};
+static_assert(sizeof(GtaParams) <= 32000, "kernel parameter block too large");
+
+struct Item {
+  int layer, tm, tn, k0, k1, split, example;
+};
+
+template <bool kSqsum>
+__device__ __forceinline__ Item decode_item(const GtaParams& P, int item) {
+  Item it;
+  int l = 0;
+  while (l + 1 < P.n_layers && item >= P.layer[l + 1].item_begin) ++l;
+  const GtaLayer& L = P.layer[l];
+  int local = item - L.item_begin;
+  it.layer = l;
+  it.tn = local % L.tiles_n; local /= L.tiles_n;
+  it.tm = local % L.tiles_m; local /= L.tiles_m;
+  if (kSqsum) {
+    it.example = local; it.split = 0;
+    it.k0 = local * P.tsteps; it.k1 = it.k0 + P.tsteps;
+  } else {
+    it.example = -1; it.split = local;
+    it.k0 = local * L.ksteps_per_split;
+    it.k1 = min(it.k0 + L.ksteps_per_split, P.B * P.tsteps);
+  }
+  return it;
+}
+
+template <bool kScale, bool kSqsum>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_gta_kernel(const __grid_constant__ GtaParams P) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                              ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + size_t(kStages) * kStageBytes);
+  uint64_t* full = bars;                      // TMA landed
+  uint64_t* ready = bars + kStages;           // G tile scaled (scale mode)
+  uint64_t* empty = bars + 2 * kStages;       // MMAs retired
+  uint64_t* acc_full = bars + 3 * kStages;    // [2]
+  uint64_t* acc_empty = acc_full + 2;         // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* epi_red = reinterpret_cast<float*>(tmem_slot + 2);   // [2][4]
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      ptx::mbar_init(&full[s], 1);
+      ptx::mbar_init(&ready[s], 4);
+      ptx::mbar_init(&empty[s], 1);
+    }
+    for (int b = 0; b < 2; ++b) { ptx::mbar_init(&acc_full[b], 1); ptx::mbar_init(&acc_empty[b], 4); }
+    *abort_flag = 0;
+    ptx::fence_mbar_init();
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(tmem_slot, kTmemCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x) {
+        const Item it = decode_item<kSqsum>(P, item);
+        const CUtensorMap* tg = &P.tmG[it.layer];
+        const CUtensorMap* ta = &P.tmA[it.layer];
+        for (int ks = it.k0; ks < it.k1; ++ks) {
+          if (!ptx::mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+          const int ex = ks / P.tsteps, t0 = (ks - ex * P.tsteps) * kBK;
+          uint8_t* dst = tiles + size_t(stage) * kStageBytes;
+          ptx::mbar_arrive_expect_tx(&full[stage], kStageBytes);
+#pragma unroll
+          for (int j = 0; j < kBM / 64; ++j)
+            ptx::tma_load_3d(dst + j * kBoxBytes, tg, &full[stage], it.tm * kBM + j * 64, t0, ex);
+#pragma unroll
+          for (int j = 0; j < kBN / 64; ++j)
+            ptx::tma_load_3d(dst + kGBytes + j * kBoxBytes, ta, &full[stage],
+                             it.tn * kBN + j * 64, t0, ex);
+          if (++stage == kStages) { stage = 0; phase ^= 1; }
+        }
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        if (P.dev_status) atomicOr(P.dev_status, DP_DEV_TIMEOUT);
+      }
+    }
+  } else if (warp == 1) {
+    // --------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = ptx::idesc_bf16_f32(kBM, kBN, 1, 1);
+      // MN-major, 128-byte swizzle: 64-column chunks are one box (8 KiB) apart, groups of
+      // 8 token rows are 1 KiB apart
+      constexpr uint64_t dbase = ptx::smem_desc_base(kBoxBytes, 1024, ptx::SWIZZLE_128B);
+      uint32_t stage = 0, phase = 0, n_item = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x, ++n_item) {
+        const Item it = decode_item<kSqsum>(P, item);
+        const uint32_t buf = n_item & 1, acc_phase = (n_item >> 1) & 1;
+        if (!ptx::mbar_wait(&acc_empty[buf], acc_phase ^ 1, abort_flag)) { ok = false; break; }
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * kBN;
+        for (int ks = it.k0; ks < it.k1; ++ks) {
+          uint64_t* go = kScale ? &ready[stage] : &full[stage];
+          if (!ptx::mbar_wait(go, phase, abort_flag)) { ok = false; break; }
+          ptx::tc_fence_after();
+          const uint32_t sg = ptx::smem_u32(tiles + size_t(stage) * kStageBytes);
+          const uint32_t sa = sg + kGBytes;
+#pragma unroll
+          for (int kk = 0; kk < kBK / 16; ++kk) {
+            // 16 token rows further = two 1 KiB row groups
+            ptx::mma_bf16_ss(d_tmem, ptx::smem_desc(dbase, sg + kk * 2048),
+                             ptx::smem_desc(dbase, sa + kk * 2048), idesc,
+                             (ks > it.k0 || kk > 0) ? 1u : 0u);
+          }
+          ptx::mma_commit(&empty[stage]);
+          if (++stage == kStages) { stage = 0; phase ^= 1; }
+        }
+        if (ok) ptx::mma_commit(&acc_full[buf]);
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        if (P.dev_status) atomicOr(P.dev_status, DP_DEV_TIMEOUT);
+      }
+    }
+  } else if (warp < 6) {
+    // ------------------------------------------------------------------ scalers
+    if (kScale) {
+      const int st = threadIdx.x - 64;                 // 0..127
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x) {
+        const Item it = decode_item<kSqsum>(P, item);
+        for (int ks = it.k0; ks < it.k1; ++ks) {
+          if (!ptx::mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
+          const int ex = ks / P.tsteps;
+          const float r = __ldg(P.clip + ex);
+          if (r != 1.0f) {
+            uint4* g = reinterpret_cast<uint4*>(tiles + size_t(stage) * kStageBytes);
+#pragma unroll
+            for (int c = 0; c < kGBytes / 16 / 128; ++c) {
+              uint4 v = g[c * 128 + st];
+              uint32_t* w = reinterpret_cast<uint32_t*>(&v);
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float lo = __uint_as_float(w[e] << 16) * r;
+                const float hi = __uint_as_float(w[e] & 0xffff0000u) * r;
+                const __nv_bfloat162 pk = __floats2bfloat162_rn(lo, hi);
+                w[e] = *reinterpret_cast<const uint32_t*>(&pk);
+              }
+              g[c * 128 + st] = v;
+            }
+            ptx::fence_proxy_async_smem();
+          }
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&ready[stage]);
+          if (++stage == kStages) { stage = 0; phase ^= 1; }
+        }
+      }
+      if (!ok && lane == 0) {
+        *abort_flag = 1;
+        if (P.dev_status) atomicOr(P.dev_status, DP_DEV_TIMEOUT);
+      }
+    }
+  } else {
+    // ----------------------------------------------------------------- epilogue
+    const int q = warp & 3;
+    const int ew = warp - 6;
+    uint32_t n_item = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x, ++n_item) {
+      const Item it = decode_item<kSqsum>(P, item);
+      const GtaLayer& L = P.layer[it.layer];
+      const uint32_t buf = n_item & 1, acc_phase = (n_item >> 1) & 1;
+      if (!ptx::mbar_wait(&acc_full[buf], acc_phase, abort_flag)) { ok = false; break; }
+      ptx::tc_fence_after();
+      const uint32_t t0 = tmem_base + (uint32_t(q * 32) << 16) + buf * kBN;
+      const int row = it.tm * kBM + q * 32 + lane;
+      if (kSqsum) {
+        float acc = 0.f;
+#pragma unroll 1
+        for (int c = 0; c < kBN / 32; ++c) {
+          uint32_t r[32];
+          ptx::tmem_ld_32x32b_x32(t0 + c * 32, r);
+          ptx::tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) { const float v = __uint_as_float(r[j]); acc = fmaf(v, v, acc); }
+        }
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&acc_empty[buf]);
+        acc = warp_sum(acc);
+        if (lane == 0) epi_red[buf * 4 + ew] = acc;
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (ew == 0 && lane == 0) {
+          const float s = (epi_red[buf * 4 + 0] + epi_red[buf * 4 + 1]) +
+                          (epi_red[buf * 4 + 2] + epi_red[buf * 4 + 3]);
+          P.sq_partials[size_t(it.example) * P.n_per + L.col_begin + it.tm * L.tiles_n + it.tn] = s;
+        }
+      } else {
+        // destination: the layer's output (no K split) or this split's partial plane
+        float* dst;
+        long long ld;
+        float beta;
+        if (L.nsplit == 1) { dst = L.out; ld = L.ldo; beta = L.beta; }
+        else { dst = L.partial + size_t(it.split) * size_t(L.M) * L.N; ld = L.N; beta = 0.f; }
+        const bool vec_ok = ((ld & 3) == 0) && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0);
+#pragma unroll 1
+        for (int c = 0; c < kBN / 32; ++c) {
+          uint32_t r[32];
+          ptx::tmem_ld_32x32b_x32(t0 + c * 32, r);
+          ptx::tmem_ld_wait();
+          const int col0 = it.tn * kBN + c * 32;
+          if (row < L.M && col0 < L.N) {
+            float* o = dst + size_t(row) * ld + col0;
+            if (vec_ok && col0 + 32 <= L.N) {
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                float4 v = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
+                                       __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
+                if (beta != 0.f) {
+                  const float4 old = *reinterpret_cast<const float4*>(o + 4 * j);
+                  v.x += old.x; v.y += old.y; v.z += old.z; v.w += old.w;
+                }
+                *reinterpret_cast<float4*>(o + 4 * j) = v;
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                if (col0 + j < L.N) {
+                  float v = __uint_as_float(r[j]);
+                  if (beta != 0.f) v += o[j];
+                  o[j] = v;
+                }
+              }
+            }
+          }
+        }
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&acc_empty[buf]);
+      }
+    }
+    if (!ok && lane == 0) {
+      *abort_flag = 1;
+      if (P.dev_status) atomicOr(P.dev_status, DP_DEV_TIMEOUT);
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// out = beta*out + sum over K splits of the partial planes, in split order
+__global__ void splitk_reduce_kernel(const float* __restrict__ partial, int nsplit, int M, int N,
+                                     float* __restrict__ out, long long ldo, float beta) {
+  const size_t total = size_t(M) * N;
+  for (size_t e = size_t(blockIdx.x) * blockDim.x + threadIdx.x; e < total;
+       e += size_t(gridDim.x) * blockDim.x) {
+    const int r = int(e / N), c = int(e - size_t(r) * N);
+    float s = 0.f;
+    for (int k = 0; k < nsplit; ++k) s += partial[size_t(k) * total + e];
+    float* o = out + size_t(r) * ldo + c;
+    *o = (beta != 0.f) ? (*o + s) : s;
+  }
+}
+
+template <bool kScale, bool kSqsum>
+dp_status set_attr_once() {
+  static bool done = false;
+  if (!done) {
+    DP_CUDA_OK(cudaFuncSetAttribute(gemm_gta_kernel<kScale, kSqsum>,
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
+    done = true;
+  }
+  return DP_OK;
+}
+
+}  // namespace
+
+int gta_choose_nsplit(int B, int T, int d, int p, int sms) {
+  const int tiles = ceil_div(p, kBM) * ceil_div(d, kBN);
+  const int ksteps = B * ceil_div(T, kBK);
+  if (tiles >= sms) return 1;
+  int ns = std::max(1, sms / tiles);
+  ns = std::min(ns, std::max(1, ksteps / 4));     // at least 4 K steps per split
+  return std::max(1, ns);
+}
+
+size_t gta_partial_bytes(int B, int T, int d, int p, int sms) {
+  const int ns = gta_choose_nsplit(B, T, d, p, sms);
+  return ns > 1 ? align_up(size_t(ns) * size_t(p) * size_t(d) * sizeof(float), 256) : 0;
+}
+
+dp_status launch_clip_accumulate_tc(const void* A, int64_t lda, const void* G, int64_t ldg, int B,
+                                    int T, int d, int p, const float* clip, float* out,
+                                    int64_t ldo, float beta, float* partial_ws, int* dev_status,
+                                    cudaStream_t st) {
+  dp_status s = set_attr_once<true, false>();
+  if (s != DP_OK) return s;
+  const int sms = sm_count();
+  GtaParams P;
+  memset(&P, 0, sizeof(P));
+  s = make_tmap_bf16_3d(&P.tmG[0], G, ldg, p, T, B, 64, 64);
+  if (s != DP_OK) return s;
+  s = make_tmap_bf16_3d(&P.tmA[0], A, lda, d, T, B, 64, 64);
+  if (s != DP_OK) return s;
+  GtaLayer& L = P.layer[0];
+  L.out = out; L.ldo = ldo; L.beta = beta;
+  L.M = p; L.N = d;
+  L.tiles_m = ceil_div(p, kBM); L.tiles_n = ceil_div(d, kBN);
+  P.tsteps = ceil_div(T, kBK);
+  const int ksteps = B * P.tsteps;
+  L.nsplit = gta_choose_nsplit(B, T, d, p, sms);
+  L.ksteps_per_split = ceil_div(ksteps, L.nsplit);
+  L.nsplit = ceil_div(ksteps, L.ksteps_per_split);      // drop empty trailing splits
+  L.partial = L.nsplit > 1 ? partial_ws : nullptr;
+  L.item_begin = 0; L.col_begin = 0;
+  P.n_layers = 1; P.B = B; P.T = T;
+  P.total_items = L.tiles_m * L.tiles_n * L.nsplit;
+  P.clip = clip;
+  P.dev_status = dev_status;
+  const int grid = std::min(P.total_items, sms);
+  gemm_gta_kernel<true, false><<<grid, kThreads, kSmemBytes, st>>>(P);
+  DP_LAUNCH_OK();
+  if (L.nsplit > 1) {
+    const size_t total = size_t(p) * d;
+    const int blocks = (int)std::min<size_t>((total + 255) / 256, size_t(sms) * 8);
+    splitk_reduce_kernel<<<blocks, 256, 0, st>>>(partial_ws, L.nsplit, p, d, out, ldo, beta);
+    DP_LAUNCH_OK();
+  }
+  return DP_OK;
+}
+
+dp_status launch_direct_norm_tc(const dp_linear_desc* layers, const GhostPlan& plan, int B, int T,
+                                float* partials, int* dev_status, cudaStream_t st) {
+  dp_status s = set_attr_once<false, true>();
+  if (s != DP_OK) return s;
+  const int sms = sm_count();
+  for (size_t g0 = 0; g0 < plan.direct_layers.size(); g0 += kGtaMaxLayers) {
+    const size_t g1 = std::min(plan.direct_layers.size(), g0 + kGtaMaxLayers);
+    GtaParams P;
+    memset(&P, 0, sizeof(P));
+    int items = 0;
+    for (size_t g = g0; g < g1; ++g) {
+      const int li = plan.direct_layers[g];
+      const dp_linear_desc& D = layers[li];
+      s = make_tmap_bf16_3d(&P.tmG[g - g0], D.G, D.ldg, D.p, T, B, 64, 64);
+      if (s != DP_OK) return s;
+      s = make_tmap_bf16_3d(&P.tmA[g - g0], D.A, D.lda, D.d, T, B, 64, 64);
+      if (s != DP_OK) return s;
+      GtaLayer& L = P.layer[g - g0];
+      L.M = D.p; L.N = D.d;
+      L.tiles_m = plan.direct[li].tiles_m; L.tiles_n = plan.direct[li].tiles_n;
+      L.nsplit = 1; L.ksteps_per_split = 0;
+      L.col_begin = plan.direct[li].col_begin;
+      L.item_begin = items;
+      items += B * L.tiles_m * L.tiles_n;
+    }
+    P.n_layers = int(g1 - g0);
+    P.B = B; P.T = T; P.tsteps = ceil_div(T, kBK);
+    P.total_items = items;
+    P.sq_partials = partials; P.n_per = plan.n_per;
+    P.dev_status = dev_status;
+    const int grid = std::min(items, sms);
+    gemm_gta_kernel<false, true><<<grid, kThreads, kSmemBytes, st>>>(P);
+    DP_LAUNCH_OK();
+  }
+  return DP_OK;
+}
+
+}  // namespace dpg

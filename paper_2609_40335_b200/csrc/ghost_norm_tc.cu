@@ -1,0 +1,303 @@
+// Ghost norm of linear layers on tcgen05 tensor cores (bf16 in, fp32 accumulate).
+//
+// For example i and a linear layer with input A_i (T x d) and output gradient G_i (T x p),
+// the squared Frobenius norm of the per-example weight gradient G_i^T A_i equals
+// <A_i A_i^T, G_i G_i^T>_F (Eq. 4 - Eq. 5 extended from one token to T tokens).  A work item
+// is one 128 x 128 tile pair (ti <= tj) of the two T x T Gram matrices of one (layer,
+// example): both tiles are accumulated in tensor memory, multiplied element by element and
+// summed by the epilogue warps; off-diagonal tile pairs count twice (symmetry).
+//
+// The Frobenius product is linear in each Gram matrix, so a very wide operand (the LM head's
+// V = 50257 columns) is split into column chunks handled by different CTAs; each chunk CTA
+// recomputes the full Gram tile of the narrow operand.
+//
+// Roles per CTA (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer (one thread),
+// warps 2..5 = epilogue.  Two TMEM accumulator sets let the epilogue of one item overlap the
+// MMAs of the next.  Partial sums go to a workspace and are added in a fixed order by a
+// second kernel, so results are deterministic.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "dp_common.cuh"
+#include "ghost_plan.cuh"
+#include "ptx_sm100.cuh"
+#include "tma_host.cuh"
+
+namespace dpg {
+
+namespace {
+
+constexpr int kTile = 128;                       // Gram tile edge (rows of A_i / G_i)
+constexpr int kKStep = 64;                       // bf16 columns per stage row (128 bytes)
+constexpr int kTileBytes = kTile * kKStep * 2;   // 16 KiB
+constexpr int kStageBytes = 2 * kTileBytes;      // row tile ti and row tile tj
+constexpr int kStages = 6;
+constexpr int kThreads = 192;
+constexpr int kTmemCols = 512;                   // 2 buffers x (S_A 128 + S_G 128) columns
+constexpr size_t kSmemBytes = size_t(kStages) * kStageBytes + 1024 /*alignment slack*/ + 256;
+
+struct __align__(64) GhostParams {
+  CUtensorMap tmA[kGhostMaxLayers];
+  CUtensorMap tmG[kGhostMaxLayers];
+  GhostLayerPlan layer[kGhostMaxLayers];
+  int n_layers;
+  int B, T, nt, ntp;
+  int total_items;
+  int n_per;                 // partial sums per example in the workspace
+  float* partials;           // [B][n_per]
+  int* dev_status;
+};
+
+struct Item {
+  int layer, example, ti, tj, a0, a1, g0, g1, pidx;
+};
+
+__device__ __forceinline__ Item decode_item(const GhostParams& P, int item) {
+  Item it;
+  int l = 0;
+  while (l + 1 < P.n_layers && item >= P.layer[l + 1].item_begin) ++l;
+  const GhostLayerPlan& L = P.layer[l];
+  const int local = item - L.item_begin;
+  const int s = local % L.nsplit;
+  const int tp = (local / L.nsplit) % P.ntp;
+  it.example = local / (L.nsplit * P.ntp);
+  it.layer = l;
+  int ti = 0, rem = tp;                   // tile pairs enumerated row by row, tj >= ti
+  while (rem >= P.nt - ti) { rem -= P.nt - ti; ++ti; }
+  it.ti = ti;
+  it.tj = ti + rem;
+  const int c0 = s * L.chunk_steps;
+  if (L.split_on_g) {
+    it.a0 = 0; it.a1 = L.a_steps;
+    it.g0 = c0; it.g1 = min(c0 + L.chunk_steps, L.g_steps);
+  } else {
+    it.g0 = 0; it.g1 = L.g_steps;
+    it.a0 = c0; it.a1 = min(c0 + L.chunk_steps, L.a_steps);
+  }
+  it.pidx = it.example * P.n_per + L.col_begin + tp * L.nsplit + s;
+  return it;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+ghost_norm_tc_kernel(const __grid_constant__ GhostParams P) {
+  extern __shared__ uint8_t smem_raw[];
+  // 128-byte swizzled tiles need 1024-byte alignment
+  uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                              ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + size_t(kStages) * kStageBytes);
+  uint64_t* full = bars;                   // [kStages]  TMA -> MMA
+  uint64_t* empty = bars + kStages;        // [kStages]  MMA -> TMA
+  uint64_t* acc_full = bars + 2 * kStages; // [2]        MMA -> epilogue
+  uint64_t* acc_empty = acc_full + 2;      // [2]        epilogue -> MMA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* epi_red = reinterpret_cast<float*>(tmem_slot + 2);   // [2][4]
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { ptx::mbar_init(&acc_full[b], 1); ptx::mbar_init(&acc_empty[b], 4); }
+    *abort_flag = 0;
+    ptx::fence_mbar_init();
+  }
+  if (warp == 1) {                    // one warp owns the TMEM allocation
+    ptx::tmem_alloc(tmem_slot, kTmemCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x) {
+        const Item it = decode_item(P, item);
+        const bool diag = (it.ti == it.tj);
+        const uint32_t bytes = diag ? kTileBytes : kStageBytes;
+        for (int pass = 0; pass < 2 && ok; ++pass) {
+          const CUtensorMap* tm = pass == 0 ? &P.tmA[it.layer] : &P.tmG[it.layer];
+          const int k0 = pass == 0 ? it.a0 : it.g0, k1 = pass == 0 ? it.a1 : it.g1;
+          for (int k = k0; k < k1; ++k) {
+            if (!ptx::mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+            uint8_t* dst = tiles + size_t(stage) * kStageBytes;
+            ptx::mbar_arrive_expect_tx(&full[stage], bytes);
+            ptx::tma_load_3d(dst, tm, &full[stage], k * kKStep, it.ti * kTile, it.example);
+            if (!diag)
+              ptx::tma_load_3d(dst + kTileBytes, tm, &full[stage], k * kKStep, it.tj * kTile,
+                               it.example);
+            if (++stage == kStages) { stage = 0; phase ^= 1; }
+          }
+        }
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        if (P.dev_status) atomicOr(P.dev_status, DP_DEV_TIMEOUT);
+        // let copies already in flight land before the CTA may exit
+        for (int s = 0; s < kStages; ++s) {
+          (void)ptx::mbar_wait(&full[s], 0, abort_flag + 0 * s);   // bounded
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // --------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = ptx::idesc_bf16_f32(kTile, kTile, 0, 0);
+      // K-major operand, 128-byte swizzle: 8-row groups are 1024 bytes apart
+      constexpr uint64_t dbase = ptx::smem_desc_base(16, 1024, ptx::SWIZZLE_128B);
+      uint32_t stage = 0, phase = 0, n_item = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x, ++n_item) {
+        const Item it = decode_item(P, item);
+        const bool diag = (it.ti == it.tj);
+        const uint32_t buf = n_item & 1, acc_phase = (n_item >> 1) & 1;
+        if (!ptx::mbar_wait(&acc_empty[buf], acc_phase ^ 1, abort_flag)) { ok = false; break; }
+        ptx::tc_fence_after();
+        for (int pass = 0; pass < 2 && ok; ++pass) {
+          const uint32_t d_tmem = tmem_base + buf * 256 + pass * 128;
+          const int nsteps = pass == 0 ? it.a1 - it.a0 : it.g1 - it.g0;
+          for (int k = 0; k < nsteps; ++k) {
+            if (!ptx::mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
+            ptx::tc_fence_after();
+            const uint32_t sa = ptx::smem_u32(tiles + size_t(stage) * kStageBytes);
+            const uint32_t sb = diag ? sa : sa + kTileBytes;
+#pragma unroll
+            for (int kk = 0; kk < kKStep / 16; ++kk) {
+              // 16 bf16 = 32 bytes further along K inside the swizzle atom
+              ptx::mma_bf16_ss(d_tmem, ptx::smem_desc(dbase, sa + kk * 32),
+                               ptx::smem_desc(dbase, sb + kk * 32), idesc,
+                               (k > 0 || kk > 0) ? 1u : 0u);
+            }
+            ptx::mma_commit(&empty[stage]);          // stage reusable once these MMAs retire
+            if (++stage == kStages) { stage = 0; phase ^= 1; }
+          }
+        }
+        if (ok) ptx::mma_commit(&acc_full[buf]);     // both Gram tiles complete
+      }
+      if (!ok) {
+        *abort_flag = 1;
+        if (P.dev_status) atomicOr(P.dev_status, DP_DEV_TIMEOUT);
+      }
+    }
+  } else {
+    // ----------------------------------------------------------------- epilogue
+    const int q = warp & 3;                          // TMEM lane quarter this warp may read
+    const int ew = warp - 2;
+    uint32_t n_item = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x, ++n_item) {
+      const Item it = decode_item(P, item);
+      const uint32_t buf = n_item & 1, acc_phase = (n_item >> 1) & 1;
+      if (!ptx::mbar_wait(&acc_full[buf], acc_phase, abort_flag)) { ok = false; break; }
+      ptx::tc_fence_after();
+      const uint32_t t0 = tmem_base + (uint32_t(q * 32) << 16) + buf * 256;
+      float acc = 0.f;
+#pragma unroll 1
+      for (int c = 0; c < kTile / 32; ++c) {
+        uint32_t ra[32], rg[32];
+        ptx::tmem_ld_32x32b_x32(t0 + c * 32, ra);
+        ptx::tmem_ld_32x32b_x32(t0 + 128 + c * 32, rg);
+        ptx::tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) acc = fmaf(__uint_as_float(ra[j]), __uint_as_float(rg[j]), acc);
+      }
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&acc_empty[buf]);   // accumulators may be overwritten
+      acc = warp_sum(acc);
+      if (lane == 0) epi_red[buf * 4 + ew] = acc;
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (ew == 0 && lane == 0) {
+        const float s = (epi_red[buf * 4 + 0] + epi_red[buf * 4 + 1]) +
+                        (epi_red[buf * 4 + 2] + epi_red[buf * 4 + 3]);
+        P.partials[it.pidx] = (it.ti == it.tj) ? s : 2.f * s;
+      }
+    }
+    if (!ok && lane == 0) {
+      *abort_flag = 1;
+      if (P.dev_status) atomicOr(P.dev_status, DP_DEV_TIMEOUT);
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+__global__ void reduce_partials_kernel(const float* __restrict__ partials, int n_per, int B,
+                                       float* __restrict__ sq, float factor,
+                                       float* __restrict__ plain_out) {
+  const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (i >= B) return;
+  float s = 0.f;
+  for (int j = lane; j < n_per; j += 32) s += partials[size_t(i) * n_per + j];
+  s = warp_sum(s);
+  if (lane == 0) {
+    if (plain_out) plain_out[i] = s;
+    if (sq) sq[i] += factor * s;
+  }
+}
+
+}  // namespace
+
+dp_status launch_reduce_partials(const float* partials, int n_per, int B, float* sq,
+                                 float factor, float* plain_out, cudaStream_t st) {
+  const int warps = 4;
+  reduce_partials_kernel<<<ceil_div(B, warps), warps * 32, 0, st>>>(partials, n_per, B, sq,
+                                                                  factor, plain_out);
+  DP_LAUNCH_OK();
+  return DP_OK;
+}
+
+// Enqueue the tensor-core ghost norm for the planned layers; partial sums land in
+// plan.partials layout inside `partials` (the caller reduces them afterwards).
+dp_status launch_ghost_norm_tc(const dp_linear_desc* layers, const GhostPlan& plan, int B, int T,
+                               float* partials, int* dev_status, cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    DP_CUDA_OK(cudaFuncSetAttribute(ghost_norm_tc_kernel,
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
+    attr_set = true;
+  }
+  const int nt = ceil_div(T, kTile);
+  // layers are processed in groups that fit one parameter block
+  for (size_t g0 = 0; g0 < plan.ghost_layers.size(); g0 += kGhostMaxLayers) {
+    const size_t g1 = std::min(plan.ghost_layers.size(), g0 + kGhostMaxLayers);
+    GhostParams P;
+    memset(&P, 0, sizeof(P));
+    int items = 0;
+    for (size_t g = g0; g < g1; ++g) {
+      const int li = plan.ghost_layers[g];
+      const dp_linear_desc& L = layers[li];
+      dp_status s = make_tmap_bf16_3d(&P.tmA[g - g0], L.A, L.lda, L.d, T, B, kKStep, kTile);
+      if (s != DP_OK) return s;
+      s = make_tmap_bf16_3d(&P.tmG[g - g0], L.G, L.ldg, L.p, T, B, kKStep, kTile);
+      if (s != DP_OK) return s;
+      GhostLayerPlan lp = plan.layer[li];
+      lp.item_begin = items;
+      items += B * plan.ntp * lp.nsplit;
+      P.layer[g - g0] = lp;
+    }
+    P.n_layers = int(g1 - g0);
+    P.B = B; P.T = T; P.nt = nt; P.ntp = plan.ntp;
+    P.total_items = items;
+    P.n_per = plan.n_per;
+    P.partials = partials;
+    P.dev_status = dev_status;
+    const int grid = std::min(items, sm_count());
+    ghost_norm_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(P);
+    DP_LAUNCH_OK();
+  }
+  return DP_OK;
+}
+
+}  // namespace dpg

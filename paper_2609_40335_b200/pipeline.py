@@ -1,0 +1,161 @@
+"""One DP-SGD clipping step as a sequence of library calls (no arithmetic of its own).
+
+Order (all enqueued on the current stream, no host synchronisation):
+  norms of the block linears and the LM head  -> dp_ghost_norms          (Eq. 4 - Eq. 6)
+  norm of the token (and position) embedding  -> dp_embed_norms
+  tied head: cross term                       -> dp_tied_cross_term      (Eq. 11, Eq. 13)
+  clipped sums per parameter tensor           -> dp_clip_accumulate[_embed]  (Eq. 2, Eq. 3, Eq. 7)
+  Gaussian noise per parameter tensor         -> dp_add_noise            (Eq. 3)
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Dict, List, Optional
+
+import numpy as np
+import torch
+
+from . import binding as dp
+from .workloads import HostTensor, Workload
+
+WPE_ROWS = 1024      # GPT-2's learned position table
+
+
+def to_device(ht: HostTensor, device="cuda") -> torch.Tensor:
+    """Upload a host tensor in its storage type (bf16 bit patterns are reinterpreted, not converted)."""
+    if ht.dtype == "f32":
+        return torch.from_numpy(np.ascontiguousarray(ht.data)).to(device)
+    return torch.from_numpy(np.ascontiguousarray(ht.data).view(np.int16)).to(device).view(torch.bfloat16)
+
+
+@dataclass
+class DeviceStep:
+    """Device-resident inputs, outputs and scratch of one step."""
+    B: int
+    T: int
+    V: int
+    C: float
+    sigma: float
+    tied: bool
+    positions: bool
+    linears: List[dp.Linear]
+    lm: Optional[dp.Linear]
+    ids: torch.Tensor
+    pos_ids: Optional[torch.Tensor]
+    G_emb: torch.Tensor
+    d_model: int
+    sq: torch.Tensor
+    clip: torch.Tensor
+    norms: torch.Tensor
+    cross: Optional[torch.Tensor]
+    dev_status: torch.Tensor
+    outs: Dict[str, torch.Tensor] = field(default_factory=dict)
+    ws: Optional[torch.Tensor] = None
+    launches_per_step: int = 0
+
+    def input_bytes(self) -> int:
+        n = self.ids.numel() * 4 + self.G_emb.numel() * self.G_emb.element_size()
+        for l in self.linears + ([self.lm] if self.lm else []):
+            n += l.A.numel() * l.A.element_size() + l.G.numel() * l.G.element_size()
+        return n
+
+
+def upload(w: Workload, device="cuda", share_by_identity: bool = True) -> DeviceStep:
+    cache = {}
+
+    def up(ht):
+        key = id(ht.data)
+        if share_by_identity and key in cache:
+            return cache[key]
+        t = to_device(ht, device)
+        cache[key] = t
+        return t
+
+    linears = [dp.Linear(up(l.A), up(l.G), d=l.d, p=l.p) for l in w.linears]
+    lm = dp.Linear(up(w.lm.A), up(w.lm.G), d=w.lm.d, p=w.lm.p) if w.lm is not None else None
+    ids = torch.from_numpy(w.ids).to(device)
+    pos = None
+    if w.positions:
+        pos = torch.arange(w.T, dtype=torch.int32, device=device).repeat(w.B, 1).contiguous()
+    ds = DeviceStep(
+        B=w.B, T=w.T, V=w.V, C=w.C, sigma=w.sigma, tied=w.tied, positions=w.positions,
+        linears=linears, lm=lm, ids=ids, pos_ids=pos, G_emb=up(w.G_emb), d_model=w.d_model,
+        sq=torch.zeros(w.B, dtype=torch.float32, device=device),
+        clip=torch.zeros(w.B, dtype=torch.float32, device=device),
+        norms=torch.zeros(w.B, dtype=torch.float32, device=device),
+        cross=torch.zeros(w.B, dtype=torch.float32, device=device) if w.tied else None,
+        dev_status=torch.zeros(1, dtype=torch.int32, device=device))
+    allocate(ds)
+    return ds
+
+
+def allocate(ds: DeviceStep) -> None:
+    """Output tensors (one per parameter tensor) and one workspace large enough for every call."""
+    dev = ds.sq.device
+    f32 = dict(dtype=torch.float32, device=dev)
+    for k, l in enumerate(ds.linears):
+        ds.outs[f"linear{k}"] = torch.empty(l.p, l.d, **f32)
+    ds.outs["wte"] = torch.empty(ds.V, ds.d_model, **f32)
+    if ds.lm is not None and not ds.tied:
+        ds.outs["lm_head"] = torch.empty(ds.lm.p, ds.lm.d, **f32)
+    if ds.positions:
+        ds.outs["wpe"] = torch.empty(WPE_ROWS, ds.d_model, **f32)
+    every = ds.linears + ([ds.lm] if ds.lm else [])
+    dt = dp._dt(every[0].A) if every else dp._dt(ds.G_emb)
+    need = 256
+    if every:
+        need = max(need, dp.dp_ghost_norms_ws_bytes(every, ds.B, ds.T))
+        for l in every:
+            need = max(need, dp.dp_clip_accumulate_ws_bytes(dt, ds.B, ds.T, l.d, l.p))
+    L = dp.load()
+    need = max(need, int(L.dp_embed_norms_ws_bytes(ds.B, ds.T, ds.d_model)))
+    need = max(need, int(L.dp_clip_accumulate_embed_ws_bytes(ds.B, ds.T, ds.d_model, ds.V)))
+    if ds.positions:
+        need = max(need, int(L.dp_clip_accumulate_embed_ws_bytes(ds.B, ds.T, ds.d_model, WPE_ROWS)))
+    if ds.tied:
+        need = max(need, int(L.dp_tied_cross_term_ws_bytes(ds.B, ds.T, ds.d_model, ds.V)))
+    ds.ws = torch.empty(need, dtype=torch.uint8, device=dev)
+
+
+def norms_phase(ds: DeviceStep, stream=None) -> None:
+    """Per-example squared norms into ds.sq (zeroed first), then norms and clip factors."""
+    ds.sq.zero_()
+    every = ds.linears + ([ds.lm] if ds.lm else [])
+    if every:
+        dp.dp_ghost_norms(every, ds.B, ds.T, ds.sq, ws=ds.ws, dev_status=ds.dev_status, stream=stream)
+    dp.dp_embed_norms(ds.ids, ds.G_emb, ds.V, ds.sq, ws=ds.ws, dev_status=ds.dev_status, stream=stream)
+    if ds.positions:
+        dp.dp_embed_norms(ds.pos_ids, ds.G_emb, ds.T, ds.sq, ws=ds.ws, dev_status=ds.dev_status,
+                          stream=stream)
+    if ds.tied:
+        dp.dp_tied_cross_term(ds.ids, ds.G_emb, ds.lm.A, ds.lm.G, ds.V, sq=ds.sq, cross=ds.cross,
+                              d=ds.d_model, ws=ds.ws, dev_status=ds.dev_status, stream=stream)
+    dp.dp_clip_factors(ds.sq, ds.C, clip=ds.clip, norms=ds.norms, stream=stream)
+
+
+def clip_phase(ds: DeviceStep, stream=None) -> None:
+    """Clipped sums of every parameter tensor from ds.sq."""
+    kw = dict(ws=ds.ws, dev_status=ds.dev_status, stream=stream)
+    for k, l in enumerate(ds.linears):
+        dp.dp_clip_accumulate(l.A, l.G, ds.sq, ds.C, ds.outs[f"linear{k}"], beta=0.0, d=l.d, p=l.p, **kw)
+    if ds.lm is not None:
+        head_out = ds.outs["wte"] if ds.tied else ds.outs["lm_head"]
+        dp.dp_clip_accumulate(ds.lm.A, ds.lm.G, ds.sq, ds.C, head_out, beta=0.0, d=ds.lm.d, p=ds.lm.p, **kw)
+    dp.dp_clip_accumulate_embed(ds.ids, ds.G_emb, ds.V, ds.sq, ds.C, ds.outs["wte"],
+                                beta=1.0 if (ds.tied and ds.lm is not None) else 0.0, d=ds.d_model, **kw)
+    if ds.positions:
+        dp.dp_clip_accumulate_embed(ds.pos_ids, ds.G_emb, WPE_ROWS, ds.sq, ds.C, ds.outs["wpe"],
+                                    beta=0.0, d=ds.d_model, **kw)
+
+
+def noise_phase(ds: DeviceStep, seed: int, step: int, scale: float = 1.0, stream=None) -> None:
+    """One Gaussian draw per parameter tensor; tensor_id = position in the sorted key order."""
+    for tid, name in enumerate(sorted(ds.outs)):
+        dp.dp_add_noise(ds.outs[name], ds.sigma, ds.C, scale, seed, tid, step, stream=stream)
+
+
+def dp_step(ds: DeviceStep, seed: int = 0, step: int = 0, noise: bool = True, stream=None) -> None:
+    norms_phase(ds, stream)
+    clip_phase(ds, stream)
+    if noise:
+        noise_phase(ds, seed, step, stream=stream)

@@ -1,0 +1,407 @@
+"""GPU parity: every C-ABI entry point against the float64 CPU oracle on the same seeded inputs.
+
+Tolerances (from the benchmark spec): per-example norms and clip factors 1e-4 relative for fp32
+inputs, 1e-2 relative for bf16 inputs with fp32 accumulation; clipped sums 1e-2 relative
+Frobenius error; integer outputs bit-exact; noise 1e-6 absolute per element.  Because both sides
+start from the same bf16 values, the kernels land far inside the bf16 bound; the tests assert a
+tighter 2e-3 there so that a wrong tile or a dropped K step cannot hide under the tolerance.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import dp_oracle as O
+from oracle import noise_oracle as NO
+from paper_2609_40335_b200 import binding as dp
+from paper_2609_40335_b200 import pipeline as P
+from paper_2609_40335_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+TOL_F32 = 1e-4
+TOL_BF16 = 1e-2
+TIGHT_BF16 = 2e-3
+TOL_SUM = 1e-2
+
+
+def dev():
+    return torch.device("cuda:0")
+
+
+def rel(a, b):
+    a, b = np.asarray(a, dtype=np.float64), np.asarray(b, dtype=np.float64)
+    return np.abs(a - b) / np.maximum(np.abs(b), 1e-300)
+
+
+def frob_rel(a, b):
+    a, b = np.asarray(a, dtype=np.float64), np.asarray(b, dtype=np.float64)
+    return np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300)
+
+
+def host_linear(B, T, d, p, dtype, seed, a_std=1.0, g_std=1e-2, ldg=None):
+    rng = np.random.default_rng(seed)
+    A = W._normal((B, T, d), a_std, dtype, int(rng.integers(1 << 60)))
+    G = W._normal((B, T, p), g_std, dtype, int(rng.integers(1 << 60)), ld=ldg)
+    return A, G
+
+
+def dev_linear(A, G, mode=dp.DP_NORM_AUTO):
+    return dp.Linear(P.to_device(A), P.to_device(G), d=A.cols, p=G.cols, mode=mode)
+
+
+def check_status(ds_status):
+    assert int(ds_status.item()) == 0
+
+
+# ------------------------------------------------------------------ config 1, end to end
+def test_cfg1_end_to_end_fp32():
+    w = W.named_workload("cfg1")
+    ds = P.upload(w)
+    P.dp_step(ds, seed=0, step=0, noise=False)
+    torch.cuda.synchronize()
+    check_status(ds.dev_status)
+    lin = [(l.A.widened(), l.G.widened()) for l in w.linears]
+    ref = O.dp_step(lin, w.ids, w.G_emb.widened(), w.V, w.C)
+    assert rel(ds.sq.cpu().numpy(), ref["sq"]).max() < TOL_F32
+    assert rel(ds.norms.cpu().numpy(), ref["norms"]).max() < TOL_F32
+    assert rel(ds.clip.cpu().numpy(), ref["clip"]).max() < TOL_F32
+    assert frob_rel(ds.outs["linear0"].cpu().numpy(), ref["sums"]["linear0"]) < 1e-5
+    assert frob_rel(ds.outs["wte"].cpu().numpy(), ref["sums"]["wte"]) < 1e-5
+    # noised clipped sum: same stream convention as the oracle
+    before = {k: v.clone() for k, v in ds.outs.items()}
+    P.noise_phase(ds, seed=0, step=0)
+    torch.cuda.synchronize()
+    for tid, name in enumerate(sorted(ds.outs)):
+        want = NO.add_noise(before[name].cpu().numpy().astype(np.float64), w.sigma, w.C, 1.0, 0, tid, 0)
+        got = ds.outs[name].cpu().numpy()
+        assert np.abs(got - want).max() < 2e-6 + 1e-6 * np.abs(want).max()
+
+
+# ------------------------------------------------------------------ linear-layer norms
+GHOST_CASES = [
+    # B, T, d, p, ld padding of G
+    (3, 128, 768, 256, None),       # one tile, the HBM-bound regime
+    (2, 100, 72, 136, None),        # ragged T, K tails not multiples of 64
+    (2, 200, 192, 320, None),       # two row tiles with a ragged second one (3 tile pairs)
+    (1, 384, 128, 64, None),        # three row tiles (6 tile pairs)
+    (2, 128, 256, 5003, 5008),      # wide operand split across CTAs, odd width, NaN padding
+    (5, 16, 64, 64, None),          # tiny T
+    (1, 1, 64, 128, None),          # single token: Eq. 5
+]
+
+
+@pytest.mark.parametrize("B,T,d,p,ldg", GHOST_CASES)
+@pytest.mark.parametrize("mode", [dp.DP_NORM_GHOST, dp.DP_NORM_DIRECT])
+def test_linear_norms_bf16_tensor_core(B, T, d, p, ldg, mode):
+    A, G = host_linear(B, T, d, p, "bf16", seed=B * 1000 + T + d + p, ldg=ldg)
+    lin = dev_linear(A, G, mode)
+    sq = torch.zeros(B, device=dev())
+    st = torch.zeros(1, dtype=torch.int32, device=dev())
+    used = dp.dp_ghost_norms([lin], B, T, sq, dev_status=st)
+    torch.cuda.synchronize()
+    check_status(st)
+    assert used == [mode]
+    want = O.linear_sq_norms(A.widened(), G.widened())
+    got = sq.cpu().numpy()
+    assert np.isfinite(got).all()
+    assert rel(got, want).max() < TIGHT_BF16, (got, want)
+    # accumulation semantics: a second call adds the same amount
+    dp.dp_ghost_norms([lin], B, T, sq, dev_status=st)
+    torch.cuda.synchronize()
+    assert rel(sq.cpu().numpy(), 2 * want).max() < TIGHT_BF16
+
+
+def test_linear_norms_grouped_layers_and_auto_rule():
+    B, T = 4, 128
+    shapes = [(768, 2304), (768, 768), (768, 3072), (3072, 768), (64, 64)]
+    host = [host_linear(B, T, d, p, "bf16", seed=77 + k) for k, (d, p) in enumerate(shapes)]
+    layers = [dev_linear(A, G) for A, G in host]
+    sq = torch.zeros(B, device=dev())
+    st = torch.zeros(1, dtype=torch.int32, device=dev())
+    used = dp.dp_ghost_norms(layers, B, T, sq, dev_status=st)
+    torch.cuda.synchronize()
+    check_status(st)
+    # AUTO: direct iff T*T > d*p (only the 64x64 layer: 16384 > 4096)
+    assert used == [dp.DP_NORM_GHOST] * 4 + [dp.DP_NORM_DIRECT]
+    want = sum(O.linear_sq_norms(A.widened(), G.widened()) for A, G in host)
+    assert rel(sq.cpu().numpy(), want).max() < TIGHT_BF16
+    # deterministic: same inputs, bitwise-equal result
+    sq2 = torch.zeros(B, device=dev())
+    dp.dp_ghost_norms(layers, B, T, sq2, dev_status=st)
+    torch.cuda.synchronize()
+    assert torch.equal(sq, sq2)
+
+
+def test_tensor_core_and_fma_paths_agree_on_device():
+    B, T, d, p = 8, 256, 768, 768
+    A, G = host_linear(B, T, d, p, "bf16", seed=5)
+    lin = dev_linear(A, G, dp.DP_NORM_GHOST)
+    sq_tc = torch.zeros(B, device=dev())
+    dp.dp_ghost_norms([lin], B, T, sq_tc)
+    prev = dp.dp_debug_force_fma(True)
+    try:
+        sq_fma = torch.zeros(B, device=dev())
+        dp.dp_ghost_norms([lin], B, T, sq_fma)
+    finally:
+        dp.dp_debug_force_fma(prev)
+    torch.cuda.synchronize()
+    assert rel(sq_tc.cpu().numpy(), sq_fma.cpu().numpy()).max() < 1e-4
+
+
+@pytest.mark.parametrize("mode", [dp.DP_NORM_GHOST, dp.DP_NORM_DIRECT])
+def test_linear_norms_fp32(mode):
+    B, T, d, p = 3, 21, 40, 33
+    A, G = host_linear(B, T, d, p, "f32", seed=9, g_std=1.0)
+    lin = dev_linear(A, G, mode)
+    sq = torch.zeros(B, device=dev())
+    dp.dp_ghost_norms([lin], B, T, sq)
+    torch.cuda.synchronize()
+    assert rel(sq.cpu().numpy(), O.linear_sq_norms(A.widened(), G.widened())).max() < TOL_F32
+
+
+# ------------------------------------------------------------------------ clipped sums
+ACC_CASES = [
+    # B, T, d, p
+    (4, 128, 768, 768),      # few tiles: K split across CTAs
+    (3, 100, 200, 300),      # ragged T, M and N tails inside a tile
+    (2, 64, 1024, 128),      # several N tiles
+    (6, 16, 64, 64),         # tiny T (a K step is mostly zero fill)
+    (2, 128, 256, 1003),     # odd M (LM-head like), padded ld
+]
+
+
+@pytest.mark.parametrize("B,T,d,p", ACC_CASES)
+@pytest.mark.parametrize("beta", [0.0, 1.0])
+def test_clip_accumulate_bf16_tensor_core(B, T, d, p, beta):
+    ldg = W.round_up(p, 8)
+    A, G = host_linear(B, T, d, p, "bf16", seed=B + T + d + p, ldg=ldg if ldg != p else None)
+    sq_true = O.linear_sq_norms(A.widened(), G.widened())
+    Cc = float(np.median(np.sqrt(sq_true)))              # some examples clipped, some not
+    sq = torch.from_numpy(sq_true.astype(np.float32)).to(dev())
+    out0 = torch.randn(p, d, device=dev())
+    out = out0.clone()
+    clip = torch.zeros(B, device=dev())
+    st = torch.zeros(1, dtype=torch.int32, device=dev())
+    dp.dp_clip_accumulate(P.to_device(A), P.to_device(G), sq, Cc, out, beta=beta, d=d, p=p, clip=clip,
+                          dev_status=st)
+    torch.cuda.synchronize()
+    check_status(st)
+    _, R = O.clip_factors(sq.cpu().numpy().astype(np.float64), Cc)
+    assert (R < 1).any() and (R == 1).any()
+    assert rel(clip.cpu().numpy(), R).max() < 1e-6
+    want = O.clipped_sum_linear(A.widened(), G.widened(), R) + beta * out0.cpu().numpy().astype(np.float64)
+    assert frob_rel(out.cpu().numpy(), want) < TOL_SUM
+    assert frob_rel(out.cpu().numpy(), want) < 5e-3      # bf16 rounding of R*g only
+
+
+def test_clip_accumulate_unclipped_is_plain_gemm_and_deterministic():
+    B, T, d, p = 4, 128, 256, 384
+    A, G = host_linear(B, T, d, p, "bf16", seed=3)
+    sq = torch.full((B,), 1e-12, device=dev())            # norms far below C: every R_i = 1
+    out = torch.empty(p, d, device=dev())
+    dp.dp_clip_accumulate(P.to_device(A), P.to_device(G), sq, 1.0, out)
+    out2 = torch.empty(p, d, device=dev())
+    dp.dp_clip_accumulate(P.to_device(A), P.to_device(G), sq, 1.0, out2)
+    torch.cuda.synchronize()
+    want = G.widened().reshape(B * T, p).T @ A.widened().reshape(B * T, d)
+    assert frob_rel(out.cpu().numpy(), want) < 1e-5       # no rescaling: fp32 accumulation only
+    assert torch.equal(out, out2)
+
+
+def test_clip_accumulate_fp32():
+    B, T, d, p = 3, 10, 70, 50
+    A, G = host_linear(B, T, d, p, "f32", seed=4, g_std=1.0)
+    sq_true = O.linear_sq_norms(A.widened(), G.widened())
+    Cc = float(np.median(np.sqrt(sq_true)))
+    sq = torch.from_numpy(sq_true.astype(np.float32)).to(dev())
+    out = torch.empty(p, d, device=dev())
+    dp.dp_clip_accumulate(P.to_device(A), P.to_device(G), sq, Cc, out)
+    torch.cuda.synchronize()
+    _, R = O.clip_factors(sq.cpu().numpy().astype(np.float64), Cc)
+    assert frob_rel(out.cpu().numpy(), O.clipped_sum_linear(A.widened(), G.widened(), R)) < 1e-5
+
+
+# --------------------------------------------------------------------------- embeddings
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("B,T,d,V,dist", [(4, 16, 64, 1000, "uniform"), (3, 128, 768, 50257, "zipf"),
+                                          (2, 300, 200, 50257, "zipf"), (2, 40, 768, 7, "uniform"),
+                                          (2, 33, 10, 5, "uniform")])
+def test_embed_norms_and_first_occurrence(dtype, B, T, d, V, dist):
+    ids = W.zipf_ids(B, T, V, 1.1, 11) if dist == "zipf" else W.uniform_ids(B, T, V, 11)
+    ids[0, :] = ids[0, 0]                                  # one example: a single repeated token
+    G = W._normal((B, T, d), 1.0 if dtype == "f32" else 1e-2, dtype, 12)
+    sq = torch.zeros(B, device=dev())
+    fo = torch.full((B, T), -1, dtype=torch.int32, device=dev())
+    st = torch.zeros(1, dtype=torch.int32, device=dev())
+    dp.dp_embed_norms(torch.from_numpy(ids).to(dev()), P.to_device(G), V, sq, first_occ=fo, dev_status=st)
+    torch.cuda.synchronize()
+    check_status(st)
+    np.testing.assert_array_equal(fo.cpu().numpy(), O.first_occurrence(ids))
+    tol = TOL_F32 if dtype == "f32" else TIGHT_BF16
+    assert rel(sq.cpu().numpy(), O.embed_sq_norms(ids, G.widened(), V)).max() < tol
+
+
+def test_embed_norms_position_table_and_bad_ids():
+    B, T, d = 2, 50, 96
+    G = W._normal((B, T, d), 1e-2, "bf16", 13)
+    pos = np.broadcast_to(np.arange(T, dtype=np.int32), (B, T)).copy()
+    sq = torch.zeros(B, device=dev())
+    dp.dp_embed_norms(torch.from_numpy(pos).to(dev()), P.to_device(G), T, sq)
+    torch.cuda.synchronize()
+    assert rel(sq.cpu().numpy(), (G.widened() ** 2).sum(axis=(1, 2))).max() < TIGHT_BF16
+    # out-of-range ids are flagged and skipped
+    bad = pos.copy()
+    bad[1, 7] = T + 3
+    bad[1, 9] = -1
+    sq.zero_()
+    st = torch.zeros(1, dtype=torch.int32, device=dev())
+    dp.dp_embed_norms(torch.from_numpy(bad).to(dev()), P.to_device(G), T, sq, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) & dp.DP_DEV_BAD_ID
+    g = G.widened()
+    want1 = (g[1] ** 2).sum() - (g[1, 7] ** 2).sum() - (g[1, 9] ** 2).sum()
+    assert rel(sq.cpu().numpy()[1], want1) < TIGHT_BF16
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("B,T,d,V,beta", [(4, 16, 64, 1000, 0.0), (3, 128, 768, 50257, 0.0),
+                                          (5, 700, 100, 300, 1.0), (2, 40, 132, 7, 1.0)])
+def test_clip_accumulate_embed(dtype, B, T, d, V, beta):
+    ids = W.zipf_ids(B, T, V, 1.1, 21)
+    G = W._normal((B, T, d), 1.0 if dtype == "f32" else 1e-2, dtype, 22)
+    sq_true = O.embed_sq_norms(ids, G.widened(), V)
+    Cc = float(np.median(np.sqrt(sq_true)))
+    sq = torch.from_numpy(sq_true.astype(np.float32)).to(dev())
+    out0 = torch.randn(V, d, device=dev())
+    out = out0.clone()
+    perm = torch.full((B * T,), -1, dtype=torch.int32, device=dev())
+    seg = torch.full((V + 1,), -1, dtype=torch.int32, device=dev())
+    st = torch.zeros(1, dtype=torch.int32, device=dev())
+    dp.dp_clip_accumulate_embed(torch.from_numpy(ids).to(dev()), P.to_device(G), V, sq, Cc, out, beta=beta,
+                                perm=perm, seg=seg, dev_status=st)
+    torch.cuda.synchronize()
+    check_status(st)
+    want_perm, want_seg = O.stable_token_sort(ids, V)
+    np.testing.assert_array_equal(perm.cpu().numpy(), want_perm)
+    np.testing.assert_array_equal(seg.cpu().numpy(), want_seg)
+    _, R = O.clip_factors(sq.cpu().numpy().astype(np.float64), Cc)
+    want = O.clipped_sum_embed(ids, G.widened(), R, V) + beta * out0.cpu().numpy().astype(np.float64)
+    assert frob_rel(out.cpu().numpy(), want) < 1e-5
+    if beta == 0.0:
+        untouched = np.setdiff1d(np.arange(V), ids.reshape(-1))
+        assert (out.cpu().numpy()[untouched] == 0).all()
+
+
+# --------------------------------------------------------------------------- tied cross term
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("B,T,d,V", [(3, 16, 64, 1000), (2, 128, 768, 50257), (2, 70, 100, 33)])
+def test_tied_cross_term(dtype, B, T, d, V):
+    g_std = 1.0 if dtype == "f32" else 1e-2
+    ids = W.zipf_ids(B, T, V, 1.1, 31)
+    G_emb = W._normal((B, T, d), g_std, dtype, 32)
+    A_lm = W._normal((B, T, d), 1.0, dtype, 33)
+    ld = W.round_up(V, 8) if dtype == "bf16" else V
+    G_lm = W._normal((B, T, V), g_std, dtype, 34, ld=ld if ld != V else None)
+    ref = O.tied_sq_norms(ids, G_emb.widened(), A_lm.widened(), G_lm.widened(), V)
+    sq = torch.zeros(B, device=dev())
+    cross = torch.zeros(B, device=dev())
+    st = torch.zeros(1, dtype=torch.int32, device=dev())
+    dp.dp_tied_cross_term(torch.from_numpy(ids).to(dev()), P.to_device(G_emb), P.to_device(A_lm),
+                          P.to_device(G_lm), V, sq=sq, cross=cross, d=d, dev_status=st)
+    torch.cuda.synchronize()
+    check_status(st)
+    scale = np.sqrt(ref["in"] * ref["out"])               # the term's natural scale (Cauchy-Schwarz)
+    tol = TOL_F32 if dtype == "f32" else TIGHT_BF16
+    assert (np.abs(cross.cpu().numpy() - ref["cross"]) / scale).max() < tol
+    assert (np.abs(sq.cpu().numpy() - 2 * ref["cross"]) / scale).max() < tol
+
+
+# ---------------------------------------------------------------------------------- noise
+@pytest.mark.parametrize("n", [1, 3, 4, 1023, 1 << 20])
+def test_noise_matches_oracle_stream(n):
+    seed, tid, step = (0xABCDEF12 << 32) | 0x3456789A, 5, 17
+    x = torch.zeros(n, device=dev())
+    dp.dp_add_noise(x, 1.0, 1.0, 1.0, seed, tid, step)
+    torch.cuda.synchronize()
+    want = NO.standard_normals(n, seed, tid, step)
+    assert np.abs(x.cpu().numpy() - want).max() < 1e-6
+
+
+def test_noise_tail_region_and_scaling():
+    n = 1 << 24                                            # ~60 thousand values beyond |z| = 3.3 pass through
+    x = torch.zeros(n, device=dev())
+    dp.dp_add_noise(x, 1.0, 1.0, 1.0, 7, 0, 0)
+    z = NO.standard_normals(n, 7, 0, 0)
+    got = x.cpu().numpy()
+    assert np.abs(got - z).max() < 1e-6
+    assert np.abs(z).max() > 4.5
+    base = torch.randn(4096, device=dev())
+    y = base.clone()
+    dp.dp_add_noise(y, 0.8, 0.5, 0.25, 7, 1, 2)
+    want = NO.add_noise(base.cpu().numpy(), 0.8, 0.5, 0.25, 7, 1, 2)
+    assert np.abs(y.cpu().numpy() - want).max() < 1e-6
+    y2 = base.clone()
+    dp.dp_add_noise(y2, 0.8, 0.5, 0.25, 7, 1, 2)
+    assert torch.equal(y, y2)
+    y3 = base.clone()
+    dp.dp_add_noise(y3, 0.0, 1.0, 1.0, 7, 1, 2)
+    assert torch.equal(y3, base)
+
+
+# ---------------------------------------------------------------------------- error paths
+def test_argument_errors_are_reported_before_any_launch():
+    B, T, d, p = 2, 16, 64, 64
+    A, G = host_linear(B, T, d, p, "bf16", seed=1)
+    a, g = P.to_device(A), P.to_device(G)
+    sq = torch.zeros(B, device=dev())
+    with pytest.raises(dp.DpGhostError) as e:
+        dp.dp_ghost_norms([dp.Linear(a[:, :, 1:], g, d=d - 1)], B, T, sq)    # misaligned base
+    assert e.value.status == 3
+    with pytest.raises(dp.DpGhostError) as e:
+        dp.dp_ghost_norms([dp.Linear(a, g, mode=7)], B, T, sq)
+    assert e.value.status == 1
+    with pytest.raises(dp.DpGhostError) as e:
+        dp.dp_ghost_norms([dp.Linear(a, g)], B, T, sq, ws=torch.empty(4, dtype=torch.uint8, device=dev()))
+    assert e.value.status == 4
+    out = torch.empty(p, d, device=dev())
+    with pytest.raises(dp.DpGhostError) as e:
+        dp.dp_clip_accumulate(a, g, sq, 1.0, out, beta=0.5)
+    assert e.value.status == 1
+    with pytest.raises(dp.DpGhostError) as e:
+        dp.dp_clip_accumulate(a, g, sq, -1.0, out)
+    assert e.value.status == 1
+    with pytest.raises(dp.DpGhostError) as e:
+        dp.dp_add_noise(out.view(-1)[1:], 1.0, 1.0, 1.0, 0, 0, 0)          # not 16-byte aligned
+    assert e.value.status == 3
+    with pytest.raises(dp.DpGhostError):
+        dp.dp_add_noise(torch.zeros(4), 1.0, 1.0, 1.0, 0, 0, 0)            # host tensor: no CPU path
+    torch.cuda.synchronize()
+    assert float(sq.abs().sum()) == 0.0
+
+
+# ------------------------------------------------------------- reduced model-shaped steps
+@pytest.mark.parametrize("name,over", [
+    ("cfg2", dict(B=4, n_blocks=1, V=5003)),
+    ("cfg3", dict(B=2, T=256, n_blocks=1, V=3001)),
+    ("cfg4", dict(B=3, n_blocks=1, V=4099)),
+])
+def test_reduced_model_step_matches_oracle(name, over):
+    w = W.named_workload(name, **over)
+    ds = P.upload(w)
+    P.dp_step(ds, noise=False)
+    torch.cuda.synchronize()
+    check_status(ds.dev_status)
+    lin = [(l.A.widened(), l.G.widened()) for l in w.linears]
+    ref = O.dp_step(lin, w.ids, w.G_emb.widened(), w.V, w.C, lm=(w.lm.A.widened(), w.lm.G.widened()),
+                    tied=w.tied, positions=w.positions)
+    assert rel(ds.sq.cpu().numpy(), ref["sq"]).max() < TIGHT_BF16
+    assert rel(ds.clip.cpu().numpy(), ref["clip"]).max() < TIGHT_BF16
+    if w.tied:
+        scale = np.sqrt(ref["sq_in"] * ref["sq_out"])
+        assert (np.abs(ds.cross.cpu().numpy() - ref["cross"]) / scale).max() < TIGHT_BF16
+    for k, want in ref["sums"].items():
+        got = ds.outs[k].cpu().numpy()
+        if k == "wpe":
+            assert (got[w.T:] == 0).all()
+            got = got[: w.T]
+        assert frob_rel(got, want) < TOL_SUM, k
