@@ -1,0 +1,400 @@
+#!/usr/bin/env python
+"""Benchmark of the DP-SGD ghost-clipping hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload cfg2]
+
+A step is one pass of the whole path over one synthetic batch: per-example norms of every
+block linear layer, the LM head and the embedding (plus the tied cross term / position table
+where the workload has them), clip factors, the clipped sum of every parameter tensor and its
+Gaussian noise.  Prints ONE JSON line (rank 0).  `--impl reference` times the float64 CPU
+oracle instead (a reported baseline, not a target).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "dp_sgd_examples_per_sec"
+UNIT = "examples/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
+            "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock, power and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ts, line in self.lines:
+            if ts < t0 - 0.05 or ts > t1 + 0.15:
+                continue
+            f = [x.strip() for x in line.split(",")]
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); power.append(float(f[2]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------- algorithmic work
+def work_counts(w):
+    """Algorithmic bytes / flops of one step (per-unit figures times the units of the batch)."""
+    B, T = w.B, w.T
+    es = 2 if w.dtype == "bf16" else 4
+    lin = [(l.d, l.p) for l in w.linears] + ([(w.lm.d, w.lm.p)] if w.lm else [])
+    norm_bytes = sum(es * B * T * (d + p) for d, p in lin)
+    gram_flops = sum(B * T * (T + 1) * (d + p) for d, p in lin)
+    acc_flops = sum(2 * B * T * d * p for d, p in lin)
+    acc_bytes = sum(es * B * T * (d + p) + 4 * d * p for d, p in lin)
+    n_params = sum(d * p for d, p in lin if True) + w.V * w.d_model * (0 if (w.tied and w.lm) else 1)
+    if w.positions:
+        n_params += 1024 * w.d_model
+    embed_bytes = es * B * T * w.d_model + 4 * B * T
+    return dict(norm_bytes=norm_bytes, gram_flops=gram_flops, acc_flops=acc_flops,
+                acc_bytes=acc_bytes, noise_bytes=8 * n_params, n_params=n_params,
+                embed_bytes=embed_bytes)
+
+
+def make_workload(name, seed=0):
+    from paper_2609_40335_b200 import workloads
+    return workloads.named_workload(name, seed=seed)
+
+
+# ------------------------------------------------------------------------ reference arm
+def oracle_sample_step(w, n_examples):
+    """The oracle, as it stands, on the first n examples of the workload (norms, clip factors,
+    clipped sums of every parameter tensor).  Returns seconds."""
+    from oracle import dp_oracle as O
+    sl = slice(0, n_examples)
+    t0 = time.perf_counter()
+    lin = [(l.A.widened_rows(sl), l.G.widened_rows(sl)) for l in w.linears]
+    lm = (w.lm.A.widened_rows(sl), w.lm.G.widened_rows(sl)) if w.lm else None
+    O.dp_step(lin, w.ids[sl], w.G_emb.widened_rows(sl), w.V, w.C, lm=lm, tied=w.tied,
+              positions=w.positions)
+    return time.perf_counter() - t0
+
+
+def oracle_noise_seconds(n):
+    from oracle import noise_oracle as NO
+    import numpy as np
+    t0 = time.perf_counter()
+    NO.add_noise(np.zeros(n), 1.0, 1.0, 1.0, 0, 0, 0)
+    return time.perf_counter() - t0
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cores = len(os.sched_getaffinity(0))
+    w = make_workload(args.workload)
+    for _ in range(args.warmup):
+        oracle_sample_step(w, 1)
+    ts = [oracle_sample_step(w, 1) for _ in range(args.steps)]
+    per = sum(ts) / len(ts)
+    val = 1.0 / per
+    sample = (f"each step = the float64 oracle on 1 of the {w.B} examples of {w.name} (all layers, "
+              "norms + clip factors + clipped sums; noise not included)")
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": per * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": w.name, "B": w.B, "T": w.T},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------ our arm
+def run_ours(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    from paper_2609_40335_b200 import binding as dp
+    from paper_2609_40335_b200 import pipeline as P
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+    dp.load()
+    peaks = measured_peaks()
+
+    # every rank holds its own batch of the same shape (weak scaling over examples)
+    w = make_workload(args.workload, seed=rank)
+    ds = P.upload(w, dev)
+    counts = work_counts(w)
+    stream = torch.cuda.current_stream()
+
+    def reduce_sums():
+        # data-parallel exchange: clipped sums are added over ranks before the single noise draw
+        if world > 1:
+            for name in sorted(ds.outs):
+                dist.all_reduce(ds.outs[name])
+
+    def step(k, ev=None):
+        if ev: ev[0].record(stream)
+        P.norms_phase(ds)
+        if ev: ev[1].record(stream)
+        P.clip_phase(ds)
+        if ev: ev[2].record(stream)
+        reduce_sums()
+        P.noise_phase(ds, seed=args.seed, step=k)
+        if ev: ev[3].record(stream)
+
+    for k in range(args.warmup):
+        step(k)
+    torch.cuda.synchronize()
+    assert int(ds.dev_status.item()) == 0, "device status flagged a problem during warm-up"
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    launches0 = dp.dp_kernel_launches()
+    t_wall0 = time.time()
+    e0.record(stream)
+    for k in range(args.steps):
+        step(args.warmup + k, evs[k])
+    e1.record(stream)
+    torch.cuda.synchronize()
+    t_wall1 = time.time()
+    if world > 1:
+        dist.barrier()
+    launches = dp.dp_kernel_launches() - launches0
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    ms_total = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    assert int(ds.dev_status.item()) == 0, "device status flagged a problem in the timed region"
+    ms_step = ms_total / args.steps
+    value = world * w.B / (ms_step * 1e-3)
+    ms_norm = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
+    ms_clip = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
+    ms_noise = statistics.mean(e[2].elapsed_time(e[3]) for e in evs)
+
+    # dominant kernel: the tensor-core G^T A GEMM of the clipped sums, timed live with events
+    # around its calls (one call per layer; the bracket also holds the tiny clip-factor and
+    # split-K reduce kernels of each call)
+    lin_layers = ds.linears + ([ds.lm] if ds.lm else [])
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    gemm_ms = []
+    for _ in range(max(3, min(args.steps, 10))):
+        g0.record(stream)
+        for k, l in enumerate(ds.linears):
+            dp.dp_clip_accumulate(l.A, l.G, ds.sq, ds.C, ds.outs[f"linear{k}"], d=l.d, p=l.p, ws=ds.ws,
+                                  dev_status=ds.dev_status)
+        if ds.lm is not None:
+            dp.dp_clip_accumulate(ds.lm.A, ds.lm.G, ds.sq, ds.C,
+                                  ds.outs["wte"] if ds.tied else ds.outs["lm_head"],
+                                  d=ds.lm.d, p=ds.lm.p, ws=ds.ws, dev_status=ds.dev_status)
+        g1.record(stream)
+        torch.cuda.synchronize()
+        gemm_ms.append(g0.elapsed_time(g1))
+    gemm_ms_avg = statistics.mean(gemm_ms)
+    n_gemm = len(lin_layers)
+    achieved_tf = counts["acc_flops"] / (gemm_ms_avg * 1e-3) / 1e12
+    peak_tf = peaks["bf16_tflops_sustained"]
+    roofline = {"kernel": "gemm_gta_kernel<scale> (dp_clip_accumulate)", "bound": "tensor",
+                "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
+                "frac": achieved_tf / peak_tf, "peak_source": peaks["source"] + " sustained bf16",
+                "launches_per_step": n_gemm, "ms_per_launch_avg": gemm_ms_avg / n_gemm,
+                "flops_per_step": counts["acc_flops"], "traffic": None}
+    # the norm phase is HBM-bound at T=128: algorithmic bytes = every A and G read once
+    g0.record(stream)
+    reps = 5
+    for _ in range(reps):
+        ds.sq.zero_()
+        dp.dp_ghost_norms(lin_layers, ds.B, ds.T, ds.sq, ws=ds.ws, dev_status=ds.dev_status)
+    g1.record(stream)
+    torch.cuda.synchronize()
+    ghost_ms = g0.elapsed_time(g1) / reps
+    ghost_gbs = counts["norm_bytes"] / (ghost_ms * 1e-3) / 1e9
+    ghost_tf = counts["gram_flops"] / (ghost_ms * 1e-3) / 1e12
+    floor_ms = max(counts["norm_bytes"] / (peaks["hbm_gbs"] * 1e9),
+                   counts["gram_flops"] / (peak_tf * 1e12)) * 1e3
+    others = {
+        "ghost_norm_tc_kernel (dp_ghost_norms)": {
+            "bound": "hbm" if counts["norm_bytes"] / (peaks["hbm_gbs"] * 1e9) >=
+            counts["gram_flops"] / (peak_tf * 1e12) else "tensor",
+            "ms": ghost_ms, "achieved_GBs": ghost_gbs, "achieved_TFLOPs": ghost_tf,
+            "peak_GBs": peaks["hbm_gbs"], "frac": floor_ms / ghost_ms},
+        "add_noise_kernel (dp_add_noise)": {
+            "bound": "hbm", "ms": ms_noise, "achieved_GBs": counts["noise_bytes"] / (ms_noise * 1e-3) / 1e9,
+            "peak_GBs": peaks["hbm_gbs"],
+            "frac": counts["noise_bytes"] / (ms_noise * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+    }
+
+    # end to end through the public API with HOST buffers: every step copies the step's inputs
+    # from pinned host memory and reads the per-example norms and clip factors back
+    host_in, dev_in = [], []
+    seen = set()
+    for t in [ds.ids, ds.G_emb] + [x for l in lin_layers for x in (l.A, l.G)]:
+        if t.data_ptr() in seen:
+            continue
+        seen.add(t.data_ptr())
+        h = torch.empty(t.shape, dtype=t.dtype, pin_memory=True)
+        h.copy_(t)
+        host_in.append(h); dev_in.append(t)
+    host_out = torch.empty(2, w.B, dtype=torch.float32, pin_memory=True)
+    h2d = sum(h.numel() * h.element_size() for h in host_in)
+    d2h = host_out.numel() * 4
+
+    def e2e_step(k):
+        for h, t in zip(host_in, dev_in):
+            t.copy_(h, non_blocking=True)
+        step(k)
+        host_out[0].copy_(ds.norms, non_blocking=True)
+        host_out[1].copy_(ds.clip, non_blocking=True)
+        torch.cuda.synchronize()
+
+    e2e_steps = max(3, min(args.steps, 10))
+    e2e_step(0)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for k in range(e2e_steps):
+        e2e_step(k)
+    t_e2e = time.perf_counter() - t0
+    if world > 1:
+        t = torch.tensor([t_e2e], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        t_e2e = float(t.item())
+    e2e_val = world * w.B * e2e_steps / t_e2e
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # CPU baseline: the oracle on a bounded sample, on this machine's host cores (rank 0, N=1 only)
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        n_ex = 4
+        t_ex = oracle_sample_step(w, n_ex)
+        n_noise = 4_000_000
+        t_noise = oracle_noise_seconds(n_noise)
+        est_step = t_ex * (w.B / n_ex) + t_noise * (counts["n_params"] / n_noise)
+        cpu = {"value": w.B / est_step, "unit": UNIT, "cores": len(os.sched_getaffinity(0)),
+               "kind": "oracle",
+               "sample": (f"{n_ex} of {w.B} examples through norms+clip+sums of all layers "
+                          f"({t_ex:.1f} s) and noise on {n_noise} of {counts['n_params']} parameters "
+                          f"({t_noise:.1f} s), scaled to one full step ({est_step:.1f} s)")}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": w.dtype if w.dtype != "f32" else "f32", "data": "synthetic",
+        "config": {"workload": w.name, "B_per_gpu": w.B, "T": w.T, "V": w.V, "layers": len(w.linears),
+                   "lm_head": bool(w.lm), "tied": w.tied, "positions": w.positions,
+                   "accumulate": "fp32", "input_bytes_per_step": ds.input_bytes(),
+                   "l2": "inputs (%.2f GB per step) are larger than the 126 MB L2" % (ds.input_bytes() / 1e9)},
+        "phases_ms": {"norms": ms_norm, "clip_accumulate": ms_clip, "noise": ms_noise,
+                      "norm_plus_clip": ms_norm + ms_clip},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": roofline,
+        "roofline_other": others,
+        "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+                "d2h_bytes_per_step": int(d2h), "steps": e2e_steps},
+        "cpu_baseline": cpu,
+        "peaks": peaks,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        if args.steps > 30:
+            args.steps = 30
+        run_reference(args)
+    else:
+        if args.warmup < 3:
+            args.warmup = 3
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -154,6 +154,9 @@ dp_status dp_add_noise(float* out, int64_t n, float sigma, float C, float scale,
 const char* dp_status_string(dp_status s);
 int32_t dp_last_cuda_error(void);      /* cudaError_t / CUresult of the last DP_ERR_CUDA */
 const char* dp_version(void);
+/* Number of CUDA kernels this library has enqueued since it was loaded (memsets and copies
+ * are not counted).  Lets a caller report how many of its launches a timed region held. */
+int64_t dp_kernel_launches(void);
 /* Test hook: when non-zero, DP_BF16 linear-layer calls run the plain fp32-FMA kernels
  * instead of the tensor-core ones (used to cross-check the two on the device).  Returns
  * the previous value.  Off by default; not meant for production use. */

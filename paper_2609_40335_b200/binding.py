@@ -37,7 +37,7 @@ EXPORTS = ["dp_ghost_norms", "dp_ghost_norms_ws_bytes", "dp_embed_norms", "dp_em
            "dp_tied_cross_term", "dp_tied_cross_term_ws_bytes", "dp_clip_factors",
            "dp_clip_accumulate", "dp_clip_accumulate_ws_bytes", "dp_clip_accumulate_embed",
            "dp_clip_accumulate_embed_ws_bytes", "dp_add_noise", "dp_status_string",
-           "dp_last_cuda_error", "dp_version", "dp_debug_force_fma"]
+           "dp_last_cuda_error", "dp_version", "dp_kernel_launches", "dp_debug_force_fma"]
 
 
 def lib_path() -> str:
@@ -77,6 +77,7 @@ def load():
     L.dp_status_string.restype = C.c_char_p
     L.dp_last_cuda_error.restype = i32
     L.dp_version.restype = C.c_char_p
+    L.dp_kernel_launches.restype = C.c_int64
     L.dp_debug_force_fma.argtypes = [i32]
     L.dp_debug_force_fma.restype = i32
     for name in EXPORTS:
@@ -261,6 +262,10 @@ def dp_add_noise(out: torch.Tensor, sigma: float, C_: float, scale: float, seed:
 
 def dp_debug_force_fma(on: bool) -> bool:
     return bool(load().dp_debug_force_fma(1 if on else 0))
+
+
+def dp_kernel_launches() -> int:
+    return int(load().dp_kernel_launches())
 
 
 def dp_version() -> str:

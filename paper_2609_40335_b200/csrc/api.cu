@@ -12,6 +12,7 @@ namespace dpg {
 
 int g_last_cuda_error = 0;
 int g_force_fma = 0;
+long long g_kernel_launches = 0;
 
 int sm_count() {
   static int n = 0;
@@ -110,6 +111,7 @@ const char* dp_status_string(dp_status s) {
 
 int32_t dp_last_cuda_error(void) { return g_last_cuda_error; }
 const char* dp_version(void) { return "dp_ghost 0.1.0 (sm_100a)"; }
+int64_t dp_kernel_launches(void) { return g_kernel_launches; }
 int32_t dp_debug_force_fma(int32_t on) {
   const int prev = g_force_fma;
   g_force_fma = on ? 1 : 0;

@@ -12,6 +12,7 @@ namespace dpg {
 // last CUDA error code seen by an entry point (returned by dp_last_cuda_error)
 extern int g_last_cuda_error;
 extern int g_force_fma;
+extern long long g_kernel_launches;   // kernels enqueued by this library since load
 
 inline dp_status cuda_fail(cudaError_t e) {
   g_last_cuda_error = (int)e;
@@ -28,6 +29,7 @@ inline dp_status cuda_fail(cudaError_t e) {
   do {                                                    \
     cudaError_t _e = cudaGetLastError();                  \
     if (_e != cudaSuccess) return ::dpg::cuda_fail(_e);   \
+    ++::dpg::g_kernel_launches;                           \
   } while (0)
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
