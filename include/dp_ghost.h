@@ -126,6 +126,18 @@ dp_status dp_clip_accumulate(const void* A, int64_t lda, const void* G, int64_t 
                              void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
 size_t dp_clip_accumulate_ws_bytes(dp_dtype dt, int32_t B, int32_t T, int32_t d, int32_t p);
 
+/* ---- the same clipped sums for many layers in ONE launch ----
+ * layers [host, n_layers entries; mode fields ignored]; outs [host array of n_layers [dev]
+ * pointers], ldos [host array].  The output tiles of all layers form one work list for a
+ * persistent kernel, which keeps every SM busy even when a single layer has few tiles.
+ * Same scalars, clip output and error rules as dp_clip_accumulate. */
+dp_status dp_clip_accumulate_grouped(const dp_linear_desc* layers, int32_t n_layers, dp_dtype dt,
+                                     int32_t B, int32_t T, const float* sq, float C, float* clip,
+                                     float* const* outs, const int64_t* ldos, float beta,
+                                     void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+size_t dp_clip_accumulate_grouped_ws_bytes(const dp_linear_desc* layers, int32_t n_layers,
+                                           dp_dtype dt, int32_t B, int32_t T);
+
 /* ---- clipped sum of an embedding table: out[v,:] = beta*out[v,:] + sum_{i,t: id=v} R_i g_{i,t} ----
  * The B*T token positions are ordered by a stable counting sort on the id, then every
  * distinct id is reduced in that order.  perm [dev, B*T int32 or NULL] and seg [dev, V+1

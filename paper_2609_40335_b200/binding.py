@@ -35,7 +35,8 @@ class _LinearDesc(C.Structure):
 
 EXPORTS = ["dp_ghost_norms", "dp_ghost_norms_ws_bytes", "dp_embed_norms", "dp_embed_norms_ws_bytes",
            "dp_tied_cross_term", "dp_tied_cross_term_ws_bytes", "dp_clip_factors",
-           "dp_clip_accumulate", "dp_clip_accumulate_ws_bytes", "dp_clip_accumulate_embed",
+           "dp_clip_accumulate", "dp_clip_accumulate_ws_bytes", "dp_clip_accumulate_grouped",
+           "dp_clip_accumulate_grouped_ws_bytes", "dp_clip_accumulate_embed",
            "dp_clip_accumulate_embed_ws_bytes", "dp_add_noise", "dp_status_string",
            "dp_last_cuda_error", "dp_version", "dp_kernel_launches", "dp_debug_force_fma"]
 
@@ -68,6 +69,10 @@ def load():
                                      f32, vp, sz, vp, vp]
     L.dp_clip_accumulate_ws_bytes.argtypes = [i32, i32, i32, i32, i32]
     L.dp_clip_accumulate_ws_bytes.restype = sz
+    L.dp_clip_accumulate_grouped.argtypes = [C.POINTER(_LinearDesc), i32, i32, i32, i32, vp, f32, vp,
+                                             C.POINTER(vp), C.POINTER(i64), f32, vp, sz, vp, vp]
+    L.dp_clip_accumulate_grouped_ws_bytes.argtypes = [C.POINTER(_LinearDesc), i32, i32, i32, i32]
+    L.dp_clip_accumulate_grouped_ws_bytes.restype = sz
     L.dp_clip_accumulate_embed.argtypes = [vp, vp, i64, i32, i32, i32, i32, i32, vp, f32, vp, vp, i64,
                                            f32, vp, vp, vp, sz, vp, vp]
     L.dp_clip_accumulate_embed_ws_bytes.argtypes = [i32, i32, i32, i32]
@@ -234,6 +239,29 @@ def dp_clip_accumulate(A, G, sq, C_: float, out, beta: float = 0.0, d=None, p=No
                               float(C_), _ptr(clip), _ptr(out), out.stride(0), float(beta), _ptr(ws),
                               ws.numel() * ws.element_size(), _ptr(dev_status), _stream(stream))
     _check(st, "dp_clip_accumulate")
+
+
+def dp_clip_accumulate_grouped_ws_bytes(layers: Sequence[Linear], B: int, T: int) -> int:
+    return int(load().dp_clip_accumulate_grouped_ws_bytes(_descs(layers), len(layers),
+                                                          _dt(layers[0].A), B, T))
+
+
+def dp_clip_accumulate_grouped(layers: Sequence[Linear], B: int, T: int, sq, C_: float,
+                               outs: Sequence[torch.Tensor], beta: float = 0.0, clip=None, ws=None,
+                               dev_status=None, stream=None):
+    """outs[k] (p_k, d_k) = beta*outs[k] + sum_i R_i G_i^T A_i for every layer, one launch."""
+    L = load()
+    arr = _descs(layers)
+    dt = _dt(layers[0].A)
+    n = len(layers)
+    optr = (C.c_void_p * n)(*[_ptr(o) for o in outs])
+    ldos = (C.c_int64 * n)(*[o.stride(0) for o in outs])
+    need = int(L.dp_clip_accumulate_grouped_ws_bytes(arr, n, dt, B, T))
+    ws = _ws(need, ws, outs[0].device)
+    st = L.dp_clip_accumulate_grouped(arr, n, dt, B, T, _ptr(sq), float(C_), _ptr(clip), optr, ldos,
+                                      float(beta), _ptr(ws), ws.numel() * ws.element_size(),
+                                      _ptr(dev_status), _stream(stream))
+    _check(st, "dp_clip_accumulate_grouped")
 
 
 def dp_clip_accumulate_embed(ids, G, V: int, sq, C_: float, out, beta: float = 0.0, d=None,

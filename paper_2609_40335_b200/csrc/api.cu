@@ -218,36 +218,75 @@ dp_status dp_clip_factors(const float* sq, int32_t B, float C, float* clip, floa
 }
 
 // ------------------------------------------------------------------------ clip accumulate
-size_t dp_clip_accumulate_ws_bytes(dp_dtype dt, int32_t B, int32_t T, int32_t d, int32_t p) {
-  if (B <= 0 || T <= 0 || d <= 0 || p <= 0) return 0;
+size_t dp_clip_accumulate_grouped_ws_bytes(const dp_linear_desc* layers, int32_t n_layers,
+                                           dp_dtype dt, int32_t B, int32_t T) {
+  if (!layers || n_layers <= 0 || B <= 0 || T <= 0) return 0;
   size_t n = align_up(size_t(B) * sizeof(float), 256);          // clip factors
-  if (dt == DP_BF16 && !g_force_fma) n += gta_partial_bytes(B, T, d, p, sm_count());
+  if (dt == DP_BF16 && !g_force_fma) n += gta_partial_bytes(layers, n_layers, B, T, sm_count());
   return n;
 }
 
-dp_status dp_clip_accumulate(const void* A, int64_t lda, const void* G, int64_t ldg, dp_dtype dt,
-                             int32_t B, int32_t T, int32_t d, int32_t p, const float* sq, float C,
-                             float* clip, float* out, int64_t ldo, float beta, void* ws,
-                             size_t ws_bytes, int32_t* dev_status, void* stream) {
-  if (!A || !G || !sq || !out || B <= 0 || T <= 0 || d <= 0 || p <= 0) return DP_ERR_INVALID_ARG;
-  if (lda < d || ldg < p || ldo < d) return DP_ERR_INVALID_ARG;
+dp_status dp_clip_accumulate_grouped(const dp_linear_desc* layers, int32_t n_layers, dp_dtype dt,
+                                     int32_t B, int32_t T, const float* sq, float C, float* clip,
+                                     float* const* outs, const int64_t* ldos, float beta, void* ws,
+                                     size_t ws_bytes, int32_t* dev_status, void* stream) {
+  if (!layers || n_layers <= 0 || !outs || !ldos || !sq || B <= 0 || T <= 0) return DP_ERR_INVALID_ARG;
   if (dt != DP_F32 && dt != DP_BF16) return DP_ERR_INVALID_ARG;
   if (!(beta == 0.f || beta == 1.f) || !finite_pos(C)) return DP_ERR_INVALID_ARG;
   const bool tc = (dt == DP_BF16) && !g_force_fma;
-  if (tc && (!aligned16(A) || !aligned16(G) || (lda % 8) || (ldg % 8))) return DP_ERR_ALIGNMENT;
-  if (!ws || ws_bytes < dp_clip_accumulate_ws_bytes(dt, B, T, d, p)) return DP_ERR_WORKSPACE;
+  for (int l = 0; l < n_layers; ++l) {
+    dp_linear_desc one = layers[l];
+    one.mode = DP_NORM_AUTO;
+    const dp_status s = check_linear(one, dt, tc);
+    if (s != DP_OK) return s;
+    if (!outs[l] || ldos[l] < layers[l].d) return DP_ERR_INVALID_ARG;
+  }
+  if (!ws || ws_bytes < dp_clip_accumulate_grouped_ws_bytes(layers, n_layers, dt, B, T))
+    return DP_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   float* clip_ws = static_cast<float*>(ws);
   dp_status s = launch_clip_factors(sq, B, C, clip_ws, nullptr, st);
   if (s != DP_OK) return s;
   if (clip) DP_CUDA_OK(cudaMemcpyAsync(clip, clip_ws, size_t(B) * sizeof(float),
                                        cudaMemcpyDeviceToDevice, st));
-  if (!tc)
-    return launch_clip_accumulate_fma(A, lda, G, ldg, dt, B, T, d, p, clip_ws, out, ldo, beta, st);
+  if (!tc) {
+    for (int l = 0; l < n_layers; ++l) {
+      s = launch_clip_accumulate_fma(layers[l].A, layers[l].lda, layers[l].G, layers[l].ldg, dt, B, T,
+                                     layers[l].d, layers[l].p, clip_ws, outs[l], ldos[l], beta, st);
+      if (s != DP_OK) return s;
+    }
+    return DP_OK;
+  }
   float* partial = reinterpret_cast<float*>(static_cast<char*>(ws) +
                                             align_up(size_t(B) * sizeof(float), 256));
-  return launch_clip_accumulate_tc(A, lda, G, ldg, B, T, d, p, clip_ws, out, ldo, beta, partial,
+  return launch_clip_accumulate_tc(layers, n_layers, B, T, clip_ws, outs, ldos, beta, partial,
                                    dev_status, st);
+}
+
+static dp_linear_desc one_layer(const void* A, int64_t lda, const void* G, int64_t ldg, int32_t d,
+                                int32_t p) {
+  dp_linear_desc L;
+  L.A = A; L.lda = lda; L.d = d; L.G = G; L.ldg = ldg; L.p = p;
+  L.mode = DP_NORM_AUTO; L.mode_used = 0;
+  return L;
+}
+
+size_t dp_clip_accumulate_ws_bytes(dp_dtype dt, int32_t B, int32_t T, int32_t d, int32_t p) {
+  if (B <= 0 || T <= 0 || d <= 0 || p <= 0) return 0;
+  const dp_linear_desc L = one_layer(nullptr, d, nullptr, p, d, p);
+  return dp_clip_accumulate_grouped_ws_bytes(&L, 1, dt, B, T);
+}
+
+dp_status dp_clip_accumulate(const void* A, int64_t lda, const void* G, int64_t ldg, dp_dtype dt,
+                             int32_t B, int32_t T, int32_t d, int32_t p, const float* sq, float C,
+                             float* clip, float* out, int64_t ldo, float beta, void* ws,
+                             size_t ws_bytes, int32_t* dev_status, void* stream) {
+  if (!A || !G || !out || d <= 0 || p <= 0) return DP_ERR_INVALID_ARG;
+  const dp_linear_desc L = one_layer(A, lda, G, ldg, d, p);
+  float* outs[1] = {out};
+  const int64_t ldos[1] = {ldo};
+  return dp_clip_accumulate_grouped(&L, 1, dt, B, T, sq, C, clip, outs, ldos, beta, ws, ws_bytes,
+                                    dev_status, stream);
 }
 
 // ------------------------------------------------------------------ clip accumulate, embedding

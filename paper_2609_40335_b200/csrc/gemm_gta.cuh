@@ -22,12 +22,13 @@ struct GtaLayer {
   float beta;
 };
 
-int gta_choose_nsplit(int B, int T, int d, int p, int sms);
-size_t gta_partial_bytes(int B, int T, int d, int p, int sms);
+int gta_choose_nsplit(const dp_linear_desc* layers, int n_layers, int B, int T, int sms);
+size_t gta_partial_bytes(const dp_linear_desc* layers, int n_layers, int B, int T, int sms);
 
-dp_status launch_clip_accumulate_tc(const void* A, int64_t lda, const void* G, int64_t ldg, int B,
-                                    int T, int d, int p, const float* clip, float* out,
-                                    int64_t ldo, float beta, float* partial_ws, int* dev_status,
+// One persistent launch over the output tiles of all layers (plus split-K reduces if needed).
+dp_status launch_clip_accumulate_tc(const dp_linear_desc* layers, int n_layers, int B, int T,
+                                    const float* clip, float* const* outs, const int64_t* ldos,
+                                    float beta, float* partial_ws, int* dev_status,
                                     cudaStream_t st);
 
 dp_status launch_direct_norm_tc(const dp_linear_desc* layers, const GhostPlan& plan, int B, int T,

@@ -342,56 +342,81 @@ dp_status set_attr_once() {
 
 }  // namespace
 
-int gta_choose_nsplit(int B, int T, int d, int p, int sms) {
-  const int tiles = ceil_div(p, kBM) * ceil_div(d, kBN);
+// K-split factor shared by all layers of one grouped call: 1 when the output tiles alone give
+// every SM at least two items, otherwise enough splits to get there (>= 4 K steps per split).
+int gta_choose_nsplit(const dp_linear_desc* layers, int n_layers, int B, int T, int sms) {
+  long long tiles = 0;
+  for (int l = 0; l < n_layers; ++l)
+    tiles += (long long)ceil_div(layers[l].p, kBM) * ceil_div(layers[l].d, kBN);
   const int ksteps = B * ceil_div(T, kBK);
-  if (tiles >= sms) return 1;
-  int ns = std::max(1, sms / tiles);
-  ns = std::min(ns, std::max(1, ksteps / 4));     // at least 4 K steps per split
-  return std::max(1, ns);
+  if (tiles >= 2LL * sms) return 1;
+  long long ns = std::max<long long>(1, (2LL * sms) / std::max<long long>(tiles, 1));
+  ns = std::min<long long>(ns, std::max(1, ksteps / 4));
+  return (int)std::max<long long>(1, ns);
 }
 
-size_t gta_partial_bytes(int B, int T, int d, int p, int sms) {
-  const int ns = gta_choose_nsplit(B, T, d, p, sms);
-  return ns > 1 ? align_up(size_t(ns) * size_t(p) * size_t(d) * sizeof(float), 256) : 0;
+size_t gta_partial_bytes(const dp_linear_desc* layers, int n_layers, int B, int T, int sms) {
+  const int ns = gta_choose_nsplit(layers, n_layers, B, T, sms);
+  if (ns <= 1) return 0;
+  size_t n = 0;
+  for (int l = 0; l < n_layers; ++l)
+    n += align_up(size_t(ns) * size_t(layers[l].p) * size_t(layers[l].d) * sizeof(float), 256);
+  return n;
 }
 
-dp_status launch_clip_accumulate_tc(const void* A, int64_t lda, const void* G, int64_t ldg, int B,
-                                    int T, int d, int p, const float* clip, float* out,
-                                    int64_t ldo, float beta, float* partial_ws, int* dev_status,
+dp_status launch_clip_accumulate_tc(const dp_linear_desc* layers, int n_layers, int B, int T,
+                                    const float* clip, float* const* outs, const int64_t* ldos,
+                                    float beta, float* partial_ws, int* dev_status,
                                     cudaStream_t st) {
   dp_status s = set_attr_once<true, false>();
   if (s != DP_OK) return s;
   const int sms = sm_count();
-  GtaParams P;
-  memset(&P, 0, sizeof(P));
-  s = make_tmap_bf16_3d(&P.tmG[0], G, ldg, p, T, B, 64, 64);
-  if (s != DP_OK) return s;
-  s = make_tmap_bf16_3d(&P.tmA[0], A, lda, d, T, B, 64, 64);
-  if (s != DP_OK) return s;
-  GtaLayer& L = P.layer[0];
-  L.out = out; L.ldo = ldo; L.beta = beta;
-  L.M = p; L.N = d;
-  L.tiles_m = ceil_div(p, kBM); L.tiles_n = ceil_div(d, kBN);
-  P.tsteps = ceil_div(T, kBK);
-  const int ksteps = B * P.tsteps;
-  L.nsplit = gta_choose_nsplit(B, T, d, p, sms);
-  L.ksteps_per_split = ceil_div(ksteps, L.nsplit);
-  L.nsplit = ceil_div(ksteps, L.ksteps_per_split);      // drop empty trailing splits
-  L.partial = L.nsplit > 1 ? partial_ws : nullptr;
-  L.item_begin = 0; L.col_begin = 0;
-  P.n_layers = 1; P.B = B; P.T = T;
-  P.total_items = L.tiles_m * L.tiles_n * L.nsplit;
-  P.clip = clip;
-  P.dev_status = dev_status;
-  const int grid = std::min(P.total_items, sms);
-  gemm_gta_kernel<true, false><<<grid, kThreads, kSmemBytes, st>>>(P);
-  DP_LAUNCH_OK();
-  if (L.nsplit > 1) {
-    const size_t total = size_t(p) * d;
-    const int blocks = (int)std::min<size_t>((total + 255) / 256, size_t(sms) * 8);
-    splitk_reduce_kernel<<<blocks, 256, 0, st>>>(partial_ws, L.nsplit, p, d, out, ldo, beta);
+  const int tsteps = ceil_div(T, kBK);
+  const int ksteps = B * tsteps;
+  int nsplit = gta_choose_nsplit(layers, n_layers, B, T, sms);
+  const int kps = ceil_div(ksteps, nsplit);
+  nsplit = ceil_div(ksteps, kps);                       // drop empty trailing splits
+  char* pw = reinterpret_cast<char*>(partial_ws);
+  for (int g0 = 0; g0 < n_layers; g0 += kGtaMaxLayers) {
+    const int g1 = std::min(n_layers, g0 + kGtaMaxLayers);
+    GtaParams P;
+    memset(&P, 0, sizeof(P));
+    int items = 0;
+    for (int g = g0; g < g1; ++g) {
+      const dp_linear_desc& D = layers[g];
+      s = make_tmap_bf16_3d(&P.tmG[g - g0], D.G, D.ldg, D.p, T, B, 64, 64);
+      if (s != DP_OK) return s;
+      s = make_tmap_bf16_3d(&P.tmA[g - g0], D.A, D.lda, D.d, T, B, 64, 64);
+      if (s != DP_OK) return s;
+      GtaLayer& L = P.layer[g - g0];
+      L.out = outs[g]; L.ldo = ldos[g]; L.beta = beta;
+      L.M = D.p; L.N = D.d;
+      L.tiles_m = ceil_div(D.p, kBM); L.tiles_n = ceil_div(D.d, kBN);
+      L.nsplit = nsplit; L.ksteps_per_split = kps;
+      L.partial = nullptr;
+      if (nsplit > 1) {
+        L.partial = reinterpret_cast<float*>(pw);
+        pw += align_up(size_t(nsplit) * size_t(D.p) * size_t(D.d) * sizeof(float), 256);
+      }
+      L.item_begin = items; L.col_begin = 0;
+      items += L.tiles_m * L.tiles_n * nsplit;
+    }
+    P.n_layers = g1 - g0; P.B = B; P.T = T; P.tsteps = tsteps;
+    P.total_items = items;
+    P.clip = clip;
+    P.dev_status = dev_status;
+    const int grid = std::min(items, sms);
+    gemm_gta_kernel<true, false><<<grid, kThreads, kSmemBytes, st>>>(P);
     DP_LAUNCH_OK();
+    if (nsplit > 1) {
+      for (int g = g0; g < g1; ++g) {
+        const GtaLayer& L = P.layer[g - g0];
+        const size_t total = size_t(L.M) * L.N;
+        const int blocks = (int)std::min<size_t>((total + 255) / 256, size_t(sms) * 8);
+        splitk_reduce_kernel<<<blocks, 256, 0, st>>>(L.partial, nsplit, L.M, L.N, L.out, L.ldo, beta);
+        DP_LAUNCH_OK();
+      }
+    }
   }
   return DP_OK;
 }

@@ -105,8 +105,7 @@ def allocate(ds: DeviceStep) -> None:
     need = 256
     if every:
         need = max(need, dp.dp_ghost_norms_ws_bytes(every, ds.B, ds.T))
-        for l in every:
-            need = max(need, dp.dp_clip_accumulate_ws_bytes(dt, ds.B, ds.T, l.d, l.p))
+        need = max(need, dp.dp_clip_accumulate_grouped_ws_bytes(every, ds.B, ds.T))
     L = dp.load()
     need = max(need, int(L.dp_embed_norms_ws_bytes(ds.B, ds.T, ds.d_model)))
     need = max(need, int(L.dp_clip_accumulate_embed_ws_bytes(ds.B, ds.T, ds.d_model, ds.V)))
@@ -136,11 +135,13 @@ def norms_phase(ds: DeviceStep, stream=None) -> None:
 def clip_phase(ds: DeviceStep, stream=None) -> None:
     """Clipped sums of every parameter tensor from ds.sq."""
     kw = dict(ws=ds.ws, dev_status=ds.dev_status, stream=stream)
-    for k, l in enumerate(ds.linears):
-        dp.dp_clip_accumulate(l.A, l.G, ds.sq, ds.C, ds.outs[f"linear{k}"], beta=0.0, d=l.d, p=l.p, **kw)
+    layers = list(ds.linears)
+    outs = [ds.outs[f"linear{k}"] for k in range(len(ds.linears))]
     if ds.lm is not None:
-        head_out = ds.outs["wte"] if ds.tied else ds.outs["lm_head"]
-        dp.dp_clip_accumulate(ds.lm.A, ds.lm.G, ds.sq, ds.C, head_out, beta=0.0, d=ds.lm.d, p=ds.lm.p, **kw)
+        layers.append(ds.lm)
+        outs.append(ds.outs["wte"] if ds.tied else ds.outs["lm_head"])
+    if layers:
+        dp.dp_clip_accumulate_grouped(layers, ds.B, ds.T, ds.sq, ds.C, outs, beta=0.0, **kw)
     dp.dp_clip_accumulate_embed(ds.ids, ds.G_emb, ds.V, ds.sq, ds.C, ds.outs["wte"],
                                 beta=1.0 if (ds.tied and ds.lm is not None) else 0.0, d=ds.d_model, **kw)
     if ds.positions:

@@ -194,6 +194,29 @@ def test_clip_accumulate_bf16_tensor_core(B, T, d, p, beta):
     assert frob_rel(out.cpu().numpy(), want) < 5e-3      # bf16 rounding of R*g only
 
 
+def test_clip_accumulate_grouped_matches_per_layer_calls_and_oracle():
+    B, T = 4, 128
+    shapes = [(768, 2304), (768, 768), (200, 136), (3072, 768)]
+    host = [host_linear(B, T, d, p, "bf16", seed=300 + k) for k, (d, p) in enumerate(shapes)]
+    layers = [dev_linear(A, G) for A, G in host]
+    sq_true = sum(O.linear_sq_norms(A.widened(), G.widened()) for A, G in host)
+    Cc = float(np.median(np.sqrt(sq_true)))
+    sq = torch.from_numpy(sq_true.astype(np.float32)).to(dev())
+    outs = [torch.empty(p, d, device=dev()) for d, p in shapes]
+    st = torch.zeros(1, dtype=torch.int32, device=dev())
+    dp.dp_clip_accumulate_grouped(layers, B, T, sq, Cc, outs, dev_status=st)
+    torch.cuda.synchronize()
+    check_status(st)
+    _, R = O.clip_factors(sq.cpu().numpy().astype(np.float64), Cc)
+    for (A, G), l, o in zip(host, layers, outs):
+        want = O.clipped_sum_linear(A.widened(), G.widened(), R)
+        assert frob_rel(o.cpu().numpy(), want) < 5e-3
+        single = torch.empty_like(o)
+        dp.dp_clip_accumulate(l.A, l.G, sq, Cc, single, d=l.d, p=l.p)
+        torch.cuda.synchronize()
+        assert frob_rel(single.cpu().numpy(), want) < 5e-3
+
+
 def test_clip_accumulate_unclipped_is_plain_gemm_and_deterministic():
     B, T, d, p = 4, 128, 256, 384
     A, G = host_linear(B, T, d, p, "bf16", seed=3)
