@@ -17,7 +17,8 @@ DP_F32, DP_BF16 = 0, 1
 DP_NORM_AUTO, DP_NORM_GHOST, DP_NORM_DIRECT = 0, 1, 2
 DP_DEV_BAD_ID, DP_DEV_TIMEOUT = 1, 2
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libdp_ghost.so")
+_LIB_PATH = os.environ.get("DP_GHOST_LIB") or os.path.join(os.path.dirname(os.path.abspath(__file__)),
+                                                       "libdp_ghost.so")
 _lib = None
 
 

@@ -9,11 +9,12 @@
 // memory holds MN-major tiles: every TMA box is 64 token rows x 64 columns (128-byte rows,
 // 128-byte swizzle).  A K step never straddles two examples (the tensor map is 3-D:
 // column, token, example; the token tail of an example is zero-filled), so one clip factor
-// applies to a whole stage: four "scaler" warps multiply the G tile by R_i in shared memory
-// (fp32 multiply, bf16 round) between the TMA-full and MMA-ready barriers.
+// applies to a whole stage: eight "scaler" warps multiply the G tile by R_i in shared memory
+// (packed bf16 FMAs with R_i split into two bf16 parts) between the TMA-full and MMA-ready
+// barriers.
 //
-// Roles per CTA (320 threads): warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 scalers,
-// warps 6-9 epilogue; two TMEM accumulators overlap the epilogue with the next tile.
+// Roles per CTA (448 threads): warp 0 TMA producer, warp 1 MMA issuer, warps 2-9 scalers,
+// warps 10-13 epilogue; two TMEM accumulators overlap the epilogue with the next tile.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -34,8 +35,13 @@ constexpr int kBoxBytes = 64 * 128;                 // 64 token rows x 128 bytes
 constexpr int kGBytes = (kBM / 64) * kBoxBytes;     // 16 KiB
 constexpr int kABytes = (kBN / 64) * kBoxBytes;     // 32 KiB
 constexpr int kStageBytes = kGBytes + kABytes;      // 48 KiB
-constexpr int kStages = 4;
-constexpr int kThreads = 320;
+#ifndef DPG_GTA_STAGES
+#define DPG_GTA_STAGES 4
+#endif
+constexpr int kStages = DPG_GTA_STAGES;
+constexpr int kScalerWarps = 8;
+constexpr int kEpiWarp0 = 2 + kScalerWarps;          // first epilogue warp
+constexpr int kThreads = (kEpiWarp0 + 4) * 32;
 constexpr int kTmemCols = 512;                      // 2 accumulators x 256 columns
 constexpr size_t kSmemBytes = size_t(kStages) * kStageBytes + 1024 + 256;
 
@@ -100,7 +106,7 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       ptx::mbar_init(&full[s], 1);
-      ptx::mbar_init(&ready[s], 4);
+      ptx::mbar_init(&ready[s], kScalerWarps);
       ptx::mbar_init(&empty[s], 1);
     }
     for (int b = 0; b < 2; ++b) { ptx::mbar_init(&acc_full[b], 1); ptx::mbar_init(&acc_empty[b], 4); }
@@ -183,10 +189,11 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
         if (P.dev_status) atomicOr(P.dev_status, DP_DEV_TIMEOUT);
       }
     }
-  } else if (warp < 6) {
+  } else if (warp < kEpiWarp0) {
     // ------------------------------------------------------------------ scalers
     if (kScale) {
-      const int st = threadIdx.x - 64;                 // 0..127
+      constexpr int kScalerThreads = kScalerWarps * 32;
+      const int st = threadIdx.x - 64;                 // 0 .. kScalerThreads-1
       uint32_t stage = 0, phase = 0;
       bool ok = true;
       for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x) {
@@ -196,19 +203,22 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
           const int ex = ks / P.tsteps;
           const float r = __ldg(P.clip + ex);
           if (r != 1.0f) {
+            // r = r_hi + r_lo with both parts in bf16 (16 mantissa bits in total); g*r is formed
+            // as fma(g, r_hi, g*r_lo) on packed bf16 pairs: one rounding of the exact g*r_hi plus
+            // a tiny correction, i.e. the correctly rounded bf16 product up to 2^-17 relative.
+            const __nv_bfloat16 rh = __float2bfloat16_rn(r);
+            const __nv_bfloat16 rl = __float2bfloat16_rn(r - __bfloat162float(rh));
+            const __nv_bfloat162 rh2 = __halves2bfloat162(rh, rh), rl2 = __halves2bfloat162(rl, rl);
             uint4* g = reinterpret_cast<uint4*>(tiles + size_t(stage) * kStageBytes);
+            uint4 v[kGBytes / 16 / kScalerThreads];
 #pragma unroll
-            for (int c = 0; c < kGBytes / 16 / 128; ++c) {
-              uint4 v = g[c * 128 + st];
-              uint32_t* w = reinterpret_cast<uint32_t*>(&v);
+            for (int c = 0; c < kGBytes / 16 / kScalerThreads; ++c) v[c] = g[c * kScalerThreads + st];
 #pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const float lo = __uint_as_float(w[e] << 16) * r;
-                const float hi = __uint_as_float(w[e] & 0xffff0000u) * r;
-                const __nv_bfloat162 pk = __floats2bfloat162_rn(lo, hi);
-                w[e] = *reinterpret_cast<const uint32_t*>(&pk);
-              }
-              g[c * 128 + st] = v;
+            for (int c = 0; c < kGBytes / 16 / kScalerThreads; ++c) {
+              __nv_bfloat162* w = reinterpret_cast<__nv_bfloat162*>(&v[c]);
+#pragma unroll
+              for (int e = 0; e < 4; ++e) w[e] = __hfma2(w[e], rh2, __hmul2(w[e], rl2));
+              g[c * kScalerThreads + st] = v[c];
             }
             ptx::fence_proxy_async_smem();
           }
@@ -225,7 +235,7 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
   } else {
     // ----------------------------------------------------------------- epilogue
     const int q = warp & 3;
-    const int ew = warp - 6;
+    const int ew = warp - kEpiWarp0;
     uint32_t n_item = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x, ++n_item) {
@@ -329,6 +339,12 @@ __global__ void splitk_reduce_kernel(const float* __restrict__ partial, int nspl
   }
 }
 
+#ifdef DPG_GTA_NOSCALE
+constexpr bool kClipScale = false;   // experiment only: clip factors are ignored
+#else
+constexpr bool kClipScale = true;
+#endif
+
 template <bool kScale, bool kSqsum>
 dp_status set_attr_once() {
   static bool done = false;
@@ -368,7 +384,7 @@ dp_status launch_clip_accumulate_tc(const dp_linear_desc* layers, int n_layers, 
                                     const float* clip, float* const* outs, const int64_t* ldos,
                                     float beta, float* partial_ws, int* dev_status,
                                     cudaStream_t st) {
-  dp_status s = set_attr_once<true, false>();
+  dp_status s = set_attr_once<kClipScale, false>();
   if (s != DP_OK) return s;
   const int sms = sm_count();
   const int tsteps = ceil_div(T, kBK);
@@ -406,7 +422,7 @@ dp_status launch_clip_accumulate_tc(const dp_linear_desc* layers, int n_layers, 
     P.clip = clip;
     P.dev_status = dev_status;
     const int grid = std::min(items, sms);
-    gemm_gta_kernel<true, false><<<grid, kThreads, kSmemBytes, st>>>(P);
+    gemm_gta_kernel<kClipScale, false><<<grid, kThreads, kSmemBytes, st>>>(P);
     DP_LAUNCH_OK();
     if (nsplit > 1) {
       for (int g = g0; g < g1; ++g) {

@@ -1,0 +1,91 @@
+"""Small single-kernel cases for profilers (each runs one entry point a few times on cuda:0).
+
+    python -m paper_2609_40335_b200.profile_case gemm|ghost|noise|embed|cross [reps]
+
+Sizes are chosen so that inputs exceed the 126 MB L2 but stay well under a few GB, which keeps
+a multi-pass `ncu` capture short.
+"""
+from __future__ import annotations
+
+import sys
+
+import torch
+
+from . import binding as dp
+
+
+def _randn_bf16(*shape, std=1.0):
+    return (torch.randn(*shape, device="cuda") * std).to(torch.bfloat16)
+
+
+def case_gemm(reps, sq_value=4.0):
+    B, T = 32, 128
+    # 148 x 3 output tiles of 128 x 256: exactly three full waves on 148 SMs
+    layers = [dp.Linear(_randn_bf16(B, T, 768), _randn_bf16(B, T, 148 * 128, std=1e-2))]
+    outs = [torch.empty(l.G.shape[-1], l.A.shape[-1], device="cuda") for l in layers]
+    sq = torch.full((B,), sq_value, device="cuda")
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    dp.dp_clip_accumulate_grouped(layers, B, T, sq, 1.0, outs)
+    e0.record()
+    for _ in range(reps):
+        dp.dp_clip_accumulate_grouped(layers, B, T, sq, 1.0, outs)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    flops = sum(2 * B * T * l.A.shape[-1] * l.G.shape[-1] for l in layers)
+    print(f"gemm: {ms:.4f} ms per call, {flops / ms / 1e9:.1f} TFLOP/s (clip {'on' if sq_value > 1 else 'off'})")
+
+
+def case_gemm_unclipped(reps):
+    case_gemm(reps, sq_value=1e-12)
+
+
+def case_ghost(reps):
+    B, T = 32, 128
+    layers = [dp.Linear(_randn_bf16(B, T, 768), _randn_bf16(B, T, 3072, std=1e-2)) for _ in range(6)]
+    layers.append(dp.Linear(_randn_bf16(B, T, 768), _randn_bf16(B, T, 16384, std=1e-2)))
+    sq = torch.zeros(B, device="cuda")
+    for _ in range(reps):
+        dp.dp_ghost_norms(layers, B, T, sq)
+
+
+def case_noise(reps):
+    x = torch.zeros(50257 * 768, device="cuda")
+    for k in range(reps):
+        dp.dp_add_noise(x, 0.8, 1.0, 1.0, 1234, 0, k)
+
+
+def case_embed(reps):
+    B, T, d, V = 256, 512, 1024, 50257
+    w = torch.arange(1, V + 1, device="cuda", dtype=torch.float64) ** -1.1
+    ids = torch.multinomial(w / w.sum(), B * T, replacement=True).to(torch.int32).view(B, T)
+    G = _randn_bf16(B, T, d, std=1e-2)
+    sq = torch.zeros(B, device="cuda")
+    out = torch.empty(V, d, device="cuda")
+    for _ in range(reps):
+        dp.dp_embed_norms(ids, G, V, sq)
+        dp.dp_clip_accumulate_embed(ids, G, V, sq, 1.0, out)
+
+
+def case_cross(reps):
+    B, T, d, V = 32, 128, 768, 50257
+    ids = torch.randint(0, V, (B, T), device="cuda", dtype=torch.int32)
+    G_emb, A_lm = _randn_bf16(B, T, d, std=1e-2), _randn_bf16(B, T, d)
+    G_lm = _randn_bf16(B, T, 50264, std=1e-2)
+    sq = torch.zeros(B, device="cuda")
+    for _ in range(reps):
+        dp.dp_tied_cross_term(ids, G_emb, A_lm, G_lm, V, sq=sq, d=d)
+
+
+def main():
+    which = sys.argv[1] if len(sys.argv) > 1 else "gemm"
+    reps = int(sys.argv[2]) if len(sys.argv) > 2 else 3
+    torch.manual_seed(0)
+    {"gemm": case_gemm, "gemm1": case_gemm_unclipped, "ghost": case_ghost, "noise": case_noise, "embed": case_embed,
+     "cross": case_cross}[which](reps)
+    torch.cuda.synchronize()
+    print("done", which, reps)
+
+
+if __name__ == "__main__":
+    main()
