@@ -189,11 +189,11 @@ def run_ours(args):
     counts = work_counts(w)
     stream = torch.cuda.current_stream()
 
+    from paper_2609_40335_b200 import parallel
+
     def reduce_sums():
         # data-parallel exchange: clipped sums are added over ranks before the single noise draw
-        if world > 1:
-            for name in sorted(ds.outs):
-                dist.all_reduce(ds.outs[name])
+        parallel.reduce_clipped_sums(ds.outs)
 
     def step(k, ev=None):
         if ev: ev[0].record(stream)

@@ -1,0 +1,68 @@
+"""World-size-2 gloo test of the data-parallel host logic: batch sharding, the all-reduce of the
+clipped sums and the single shared noise draw.  The per-rank arithmetic is played by the oracle
+(no GPU here); what is checked is that two ranks reproduce the single-process result."""
+import os
+import sys
+
+import numpy as np
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, ret):
+    sys.path.insert(0, ROOT)
+    from oracle import dp_oracle as O
+    from oracle import noise_oracle as NO
+    from paper_2609_40335_b200 import parallel
+
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    rng = np.random.default_rng(0)                     # same global batch on every rank
+    B, T, d, p, V, C = 5, 6, 4, 3, 9, 0.7
+    A, G = rng.standard_normal((B, T, d)), rng.standard_normal((B, T, p))
+    ids, Ge = rng.integers(0, V, (B, T)), rng.standard_normal((B, T, d))
+    lo, hi = parallel.shard_range(B, rank, world)
+    res = O.dp_step([(A[lo:hi], G[lo:hi])], ids[lo:hi], Ge[lo:hi], V, C)
+    outs = {k: torch.from_numpy(v.copy()) for k, v in res["sums"].items()}
+
+    def add_noise(t, tid):
+        t.copy_(torch.from_numpy(NO.add_noise(t.numpy(), 0.5, C, 1.0, 3, tid, 11)))
+
+    parallel.reduce_then_noise(outs, add_noise)
+    ret[rank] = {k: v.numpy().copy() for k, v in outs.items()}
+    ret[f"clip{rank}"] = (lo, hi, res["clip"])
+    dist.destroy_process_group()
+
+
+def test_two_ranks_reproduce_the_single_process_step():
+    from oracle import dp_oracle as O
+    from oracle import noise_oracle as NO
+    from paper_2609_40335_b200 import parallel
+
+    assert [parallel.shard_range(5, r, 2) for r in range(2)] == [(0, 3), (3, 5)]
+    assert [parallel.shard_range(7, r, 3) for r in range(3)] == [(0, 3), (3, 5), (5, 7)]
+    ctx = mp.get_context("spawn")
+    ret = ctx.Manager().dict()
+    port = 29500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, ret)) for r in range(2)]
+    for p_ in procs:
+        p_.start()
+    for p_ in procs:
+        p_.join(120)
+        assert p_.exitcode == 0
+    rng = np.random.default_rng(0)
+    B, T, d, p, V, C = 5, 6, 4, 3, 9, 0.7
+    A, G = rng.standard_normal((B, T, d)), rng.standard_normal((B, T, p))
+    ids, Ge = rng.integers(0, V, (B, T)), rng.standard_normal((B, T, d))
+    full = O.dp_step([(A, G)], ids, Ge, V, C)
+    for tid, k in enumerate(sorted(full["sums"])):
+        want = NO.add_noise(full["sums"][k], 0.5, C, 1.0, 3, tid, 11)
+        np.testing.assert_allclose(ret[0][k], want, rtol=1e-12, atol=1e-12)
+        np.testing.assert_array_equal(ret[0][k], ret[1][k])       # replicas stay identical
+    for r in range(2):
+        lo, hi, clip = ret[f"clip{r}"]
+        np.testing.assert_allclose(clip, full["clip"][lo:hi], rtol=1e-12)
