@@ -291,7 +291,8 @@ dp_status dp_clip_accumulate(const void* A, int64_t lda, const void* G, int64_t 
 
 // ------------------------------------------------------------------ clip accumulate, embedding
 static void embed_ws_layout(int B, int T, int V, size_t* off_clip, size_t* off_counts,
-                            size_t* off_seg, size_t* off_perm, size_t* total, int* chunks) {
+                            size_t* off_seg, size_t* off_perm, size_t* off_blk, size_t* total,
+                            int* chunks) {
   const size_t n = size_t(B) * T;
   *chunks = int((n + kSortChunk - 1) / kSortChunk);
   size_t o = 0;
@@ -299,14 +300,15 @@ static void embed_ws_layout(int B, int T, int V, size_t* off_clip, size_t* off_c
   *off_counts = o; o += align_up(size_t(*chunks) * V * sizeof(int), 256);
   *off_seg = o;    o += align_up(size_t(V + 1) * sizeof(int), 256);
   *off_perm = o;   o += align_up(n * sizeof(int), 256);
+  *off_blk = o;    o += align_up(size_t(ceil_div(V, 1024)) * sizeof(int), 256);
   *total = o;
 }
 
 size_t dp_clip_accumulate_embed_ws_bytes(int32_t B, int32_t T, int32_t d, int32_t V) {
   (void)d;
   if (B <= 0 || T <= 0 || V <= 0) return 0;
-  size_t a, b, c, e, total; int chunks;
-  embed_ws_layout(B, T, V, &a, &b, &c, &e, &total, &chunks);
+  size_t a, b, c, e, f, total; int chunks;
+  embed_ws_layout(B, T, V, &a, &b, &c, &e, &f, &total, &chunks);
   return total;
 }
 
@@ -320,8 +322,8 @@ dp_status dp_clip_accumulate_embed(const int32_t* ids, const void* G, int64_t ld
   if (dt != DP_F32 && dt != DP_BF16) return DP_ERR_INVALID_ARG;
   if (!(beta == 0.f || beta == 1.f) || !finite_pos(C)) return DP_ERR_INVALID_ARG;
   if ((long long)B * T > 0x7fffffffLL) return DP_ERR_UNSUPPORTED;
-  size_t o_clip, o_counts, o_seg, o_perm, total; int chunks;
-  embed_ws_layout(B, T, V, &o_clip, &o_counts, &o_seg, &o_perm, &total, &chunks);
+  size_t o_clip, o_counts, o_seg, o_perm, o_blk, total; int chunks;
+  embed_ws_layout(B, T, V, &o_clip, &o_counts, &o_seg, &o_perm, &o_blk, &total, &chunks);
   if (!ws || ws_bytes < total) return DP_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   char* w = static_cast<char*>(ws);
@@ -330,7 +332,7 @@ dp_status dp_clip_accumulate_embed(const int32_t* ids, const void* G, int64_t ld
   sw.counts = reinterpret_cast<int*>(w + o_counts);
   sw.seg = reinterpret_cast<int*>(w + o_seg);
   sw.perm = reinterpret_cast<int*>(w + o_perm);
-  sw.block_sums = nullptr;
+  sw.block_sums = reinterpret_cast<int*>(w + o_blk);
   sw.chunks = chunks;
   const int n = B * T;
   dp_status s = launch_clip_factors(sq, B, C, clip_ws, nullptr, st);

@@ -12,13 +12,53 @@ namespace dpg {
 
 namespace {
 
-// ------------------------------------------------------------------ norm kernel
-// One block per (example, 256-column slab).  Tokens are grouped by their first occurrence
-// (warp-level id matching, then a scan over earlier tokens for group leaders), ordered by
-// (first occurrence, position), and every thread walks the ordered rows for its two columns:
-// each row of G is read exactly once.
+// 8 consecutive columns of one row as floats; `nvalid` columns exist, `vec` says the 16-byte
+// (bf16) / 2 x 16-byte (fp32) vector path is aligned.
 template <typename T>
-__global__ void __launch_bounds__(128)
+__device__ __forceinline__ void load8(const T* p, int nvalid, bool vec, float (&v)[8]);
+
+template <>
+__device__ __forceinline__ void load8<__nv_bfloat16>(const __nv_bfloat16* p, int nvalid, bool vec,
+                                                     float (&v)[8]) {
+  if (vec && nvalid >= 8) {
+    const uint4 q = *reinterpret_cast<const uint4*>(p);
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      v[2 * e] = __uint_as_float(w[e] << 16);
+      v[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+    }
+  } else {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[e] = e < nvalid ? __bfloat162float(p[e]) : 0.f;
+  }
+}
+
+template <>
+__device__ __forceinline__ void load8<float>(const float* p, int nvalid, bool vec, float (&v)[8]) {
+  if (vec && nvalid >= 8) {
+    const float4 a = *reinterpret_cast<const float4*>(p);
+    const float4 b = *reinterpret_cast<const float4*>(p + 4);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+    v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+  } else {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[e] = e < nvalid ? p[e] : 0.f;
+  }
+}
+
+// ------------------------------------------------------------------ norm kernel
+// One block (8 warps) per (example, 256-column slab).  Tokens are grouped by their first
+// occurrence (warp-level id matching, then a scan over earlier tokens for group leaders) and
+// ordered by (first occurrence, position).  The ordered rows are cut into 8 contiguous ranges
+// at group boundaries, one per warp; a lane owns 8 columns, loads 8 rows at a time (16-byte
+// loads, all in flight together) and folds them into running group sums.  Each row of G is
+// read exactly once.
+constexpr int kEmbedNormThreads = 256;
+constexpr int kEmbedBatch = 8;
+
+template <typename T>
+__global__ void __launch_bounds__(kEmbedNormThreads)
 embed_norm_kernel(const int* __restrict__ ids, const T* __restrict__ G, long long ldg, int Tn, int d,
                   int V, int slabs, float* __restrict__ partials, int* __restrict__ first_occ,
                   int* __restrict__ dev_status) {
@@ -28,7 +68,8 @@ embed_norm_kernel(const int* __restrict__ ids, const T* __restrict__ G, long lon
   int* s_ord = sm_i + 2 * Tn;    // rows ordered by (first occurrence, position); sign bit = group end
   __shared__ float red[32];
   const int i = blockIdx.x / slabs, slab = blockIdx.x % slabs;
-  const int lane = threadIdx.x & 31;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  constexpr int kWarps = kEmbedNormThreads / 32;
 
   for (int t = threadIdx.x; t < Tn; t += blockDim.x) {
     int id = ids[size_t(i) * Tn + t];
@@ -82,25 +123,48 @@ embed_norm_kernel(const int* __restrict__ ids, const T* __restrict__ G, long lon
     if ((end_mask >> k) & 1u) s_ord[r] |= int(0x80000000u);
   __syncthreads();
 
-  // grouped row sums for this thread's two columns
-  const int c = slab * kEmbedColsPerBlock + 2 * threadIdx.x;
+  // this warp's range of ordered rows, snapped forward to group starts
+  auto snap = [&](int r) {
+    while (r > 0 && r < Tn && s_ord[r - 1] >= 0) ++r;      // previous row does not end a group
+    return min(r, Tn);
+  };
+  const int per = (Tn + kWarps - 1) / kWarps;
+  const int lo = snap(min(warp * per, Tn)), hi = snap(min((warp + 1) * per, Tn));
+
+  const int c = slab * kEmbedColsPerBlock + 8 * lane;
+  const int nvalid = min(8, d - c);
   float tot = 0.f;
-  if (c < d) {
-    const bool two = (c + 1 < d);
+  if (nvalid > 0) {
+    const bool vec = ((reinterpret_cast<uintptr_t>(G) & 15) == 0) && ((ldg * sizeof(T)) % 16 == 0);
     const T* Gi = G + size_t(i) * Tn * ldg + c;
-    float r0 = 0.f, r1 = 0.f;
-#pragma unroll 4
-    for (int r = 0; r < Tn; ++r) {
-      const int o = s_ord[r];
-      const int t = o & 0x7fffffff;
-      if (s_id[t] >= 0) {
-        r0 += to_f32(Gi[size_t(t) * ldg]);
-        if (two) r1 += to_f32(Gi[size_t(t) * ldg + 1]);
+    float run[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) run[e] = 0.f;
+    for (int r0 = lo; r0 < hi; r0 += kEmbedBatch) {
+      float v[kEmbedBatch][8];
+      int o[kEmbedBatch];
+#pragma unroll
+      for (int b = 0; b < kEmbedBatch; ++b) {
+        const int r = r0 + b;
+        o[b] = r < hi ? s_ord[r] : 0;
+        const int t = o[b] & 0x7fffffff;
+        if (r < hi && s_id[t] >= 0) {
+          load8<T>(Gi + size_t(t) * ldg, nvalid, vec, v[b]);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 8; ++e) v[b][e] = 0.f;
+        }
       }
-      if (o < 0) {
-        tot = fmaf(r0, r0, tot);
-        tot = fmaf(r1, r1, tot);
-        r0 = 0.f; r1 = 0.f;
+#pragma unroll
+      for (int b = 0; b < kEmbedBatch; ++b) {
+        if (r0 + b < hi) {
+#pragma unroll
+          for (int e = 0; e < 8; ++e) run[e] += v[b][e];
+          if (o[b] < 0) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) { tot = fmaf(run[e], run[e], tot); run[e] = 0.f; }
+          }
+        }
       }
     }
   }
@@ -122,41 +186,72 @@ __global__ void sort_hist_kernel(const int* __restrict__ ids, int n, int V, int*
   atomicAdd(&counts[size_t(chunk) * V + id], 1);
 }
 
-// counts[c][v] -> number of id v in chunks before c; seg[v] = total count of v
-__global__ void sort_chunk_prefix_kernel(int* __restrict__ counts, int chunks, int V,
-                                         int* __restrict__ seg) {
-  const int v = blockIdx.x * blockDim.x + threadIdx.x;
-  if (v >= V) return;
+// counts[c][v] -> number of id v in chunks before c; seg[v] = total count of v; block totals of
+// seg (1024 ids per block) go to blk[] for the scan that follows
+__global__ void __launch_bounds__(1024)
+sort_chunk_prefix_kernel(int* __restrict__ counts, int chunks, int V, int* __restrict__ seg,
+                         int* __restrict__ blk) {
+  __shared__ int wsum[32];
+  const int v = blockIdx.x * 1024 + threadIdx.x;
   int run = 0;
-  for (int c = 0; c < chunks; ++c) {
-    const int x = counts[size_t(c) * V + v];
-    counts[size_t(c) * V + v] = run;
-    run += x;
+  if (v < V) {
+    for (int c = 0; c < chunks; ++c) {
+      const int x = counts[size_t(c) * V + v];
+      counts[size_t(c) * V + v] = run;
+      run += x;
+    }
+    seg[v] = run;
   }
-  seg[v] = run;
+  int s = run;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  if ((threadIdx.x & 31) == 0) wsum[threadIdx.x >> 5] = s;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    int t = wsum[threadIdx.x];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+    if (threadIdx.x == 0) blk[blockIdx.x] = t;
+  }
 }
 
-// in-place exclusive scan of seg[0..V] (seg[V] receives the total); single block
-__global__ void __launch_bounds__(1024) sort_scan_kernel(int* __restrict__ seg, int V) {
-  __shared__ int part[1024];
-  const int per = (V + 1 + 1023) / 1024;
-  const int lo = threadIdx.x * per, hi = min(V + 1, lo + per);
-  int s = 0;
-  for (int v = lo; v < hi; ++v) s += (v < V) ? seg[v] : 0;
-  part[threadIdx.x] = s;
+// in-place exclusive scan of seg[0..V) (seg[V] receives the total): block b adds the totals of
+// the blocks before it to a block-local scan of its 1024 entries
+__global__ void __launch_bounds__(1024)
+sort_scan_kernel(int* __restrict__ seg, int V, const int* __restrict__ blk) {
+  __shared__ int wsum[32];
+  __shared__ int base_s;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  if (w == 0) {
+    int b = 0;
+    for (int k = lane; k < (int)blockIdx.x; k += 32) b += blk[k];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) b += __shfl_xor_sync(0xffffffffu, b, o);
+    if (lane == 0) base_s = b;
+  }
+  const int v = blockIdx.x * 1024 + threadIdx.x;
+  const int x = v < V ? seg[v] : 0;
+  int inc = x;                                         // inclusive scan inside the warp
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += y;
+  }
+  if (lane == 31) wsum[w] = inc;
   __syncthreads();
-  for (int off = 1; off < 1024; off <<= 1) {       // Hillis-Steele inclusive scan
-    const int x = (threadIdx.x >= off) ? part[threadIdx.x - off] : 0;
-    __syncthreads();
-    part[threadIdx.x] += x;
-    __syncthreads();
+  if (w == 0) {
+    int t = wsum[lane];
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, t, o);
+      if (lane >= o) t += y;
+    }
+    wsum[lane] = t;                                    // inclusive scan of warp totals
   }
-  int run = part[threadIdx.x] - s;
-  for (int v = lo; v < hi; ++v) {
-    const int x = (v < V) ? seg[v] : 0;
-    seg[v] = run;
-    run += x;
-  }
+  __syncthreads();
+  const int excl = base_s + (w > 0 ? wsum[w - 1] : 0) + inc - x;
+  if (v < V) seg[v] = excl;
+  if (v == V - 1) seg[V] = excl + x;
 }
 
 __global__ void __launch_bounds__(kSortChunk)
@@ -176,16 +271,22 @@ sort_place_kernel(const int* __restrict__ ids, int n, int V, const int* __restri
 }
 
 // ------------------------------------------------------------------ segmented row sum
-// grid = (sorted positions, 128-column slices); only the block sitting on the first sorted
-// position of a token id works.  8 warps take rows k = w, w+8, ... of the segment in order and
-// their partial sums are combined in warp order, so the result does not depend on timing.
+// grid = (sorted positions, 256-column slabs); only the block sitting on the first sorted
+// position of a token id works.  Rows of the segment are staged 64 at a time (position and clip
+// factor into shared memory), warp w takes rows w, w+8, ... of each stage with all its 16-byte
+// loads in flight together; the 8 per-warp sums are combined in warp order, so the result does
+// not depend on timing.
+constexpr int kScatStage = 64;
+
 template <typename T>
 __global__ void __launch_bounds__(256)
 embed_scatter_kernel(const int* __restrict__ ids, const T* __restrict__ G, long long ldg, int Tn,
                      int d, const float* __restrict__ clip, const int* __restrict__ perm,
                      const int* __restrict__ seg, int V, float* __restrict__ out, long long ldo,
                      float beta) {
-  __shared__ float part[8][128];
+  __shared__ float part[8][kEmbedColsPerBlock];
+  __shared__ int s_pos[kScatStage];
+  __shared__ float s_r[kScatStage];
   const int k0 = blockIdx.x;
   if (k0 >= seg[V]) return;
   const int pos0 = perm[k0];
@@ -193,25 +294,49 @@ embed_scatter_kernel(const int* __restrict__ ids, const T* __restrict__ G, long 
   if (seg[v] != k0) return;                    // not the head of its segment
   const int n = seg[v + 1] - k0;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  const int c = blockIdx.y * 128 + lane * 4;
-  float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-  if (c < d) {
-#pragma unroll 4
-    for (int k = w; k < n; k += 8) {
-      const int pos = perm[k0 + k];
-      const float r = clip[pos / Tn];
-      const T* g = G + size_t(pos) * ldg + c;
-      a0 = fmaf(r, to_f32(g[0]), a0);
-      if (c + 1 < d) a1 = fmaf(r, to_f32(g[1]), a1);
-      if (c + 2 < d) a2 = fmaf(r, to_f32(g[2]), a2);
-      if (c + 3 < d) a3 = fmaf(r, to_f32(g[3]), a3);
+  const int c = blockIdx.y * kEmbedColsPerBlock + lane * 8;
+  const int nvalid = min(8, d - c);
+  const bool vec = ((reinterpret_cast<uintptr_t>(G) & 15) == 0) && ((ldg * sizeof(T)) % 16 == 0);
+  float acc[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+  for (int base = 0; base < n; base += kScatStage) {
+    const int m = min(kScatStage, n - base);
+    __syncthreads();
+    if (threadIdx.x < m) {
+      const int pos = perm[k0 + base + threadIdx.x];
+      s_pos[threadIdx.x] = pos;
+      s_r[threadIdx.x] = clip[pos / Tn];
+    }
+    __syncthreads();
+    if (nvalid > 0) {
+      float vals[kScatStage / 8][8];
+#pragma unroll
+      for (int b = 0; b < kScatStage / 8; ++b) {
+        const int k = w + 8 * b;
+        if (k < m) {
+          load8<T>(G + size_t(s_pos[k]) * ldg + c, nvalid, vec, vals[b]);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 8; ++e) vals[b][e] = 0.f;
+        }
+      }
+#pragma unroll
+      for (int b = 0; b < kScatStage / 8; ++b) {
+        const int k = w + 8 * b;
+        if (k < m) {
+          const float r = s_r[k];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) acc[e] = fmaf(r, vals[b][e], acc[e]);
+        }
+      }
     }
   }
-  part[w][lane * 4 + 0] = a0; part[w][lane * 4 + 1] = a1;
-  part[w][lane * 4 + 2] = a2; part[w][lane * 4 + 3] = a3;
+#pragma unroll
+  for (int e = 0; e < 8; ++e) part[w][lane * 8 + e] = acc[e];
   __syncthreads();
-  if (threadIdx.x < 128) {
-    const int cc = blockIdx.y * 128 + threadIdx.x;
+  {
+    const int cc = blockIdx.y * kEmbedColsPerBlock + threadIdx.x;
     if (cc < d) {
       float s = 0.f;
 #pragma unroll
@@ -240,10 +365,10 @@ dp_status launch_embed_norms(const int* ids, const void* G, int64_t ldg, dp_dtyp
     attr = true;
   }
   if (dt == DP_F32)
-    embed_norm_kernel<float><<<B * slabs, 128, smem, st>>>(ids, (const float*)G, ldg, T, d, V, slabs,
+    embed_norm_kernel<float><<<B * slabs, kEmbedNormThreads, smem, st>>>(ids, (const float*)G, ldg, T, d, V, slabs,
                                                           partials, first_occ, dev_status);
   else
-    embed_norm_kernel<__nv_bfloat16><<<B * slabs, 128, smem, st>>>(
+    embed_norm_kernel<__nv_bfloat16><<<B * slabs, kEmbedNormThreads, smem, st>>>(
         ids, (const __nv_bfloat16*)G, ldg, T, d, V, slabs, partials, first_occ, dev_status);
   DP_LAUNCH_OK();
   return DP_OK;
@@ -254,9 +379,10 @@ dp_status launch_embed_sort(const int* ids, int n, int V, const EmbedSortWs& ws,
   DP_CUDA_OK(cudaMemsetAsync(ws.counts, 0, size_t(ws.chunks) * V * sizeof(int), st));
   sort_hist_kernel<<<ws.chunks, kSortChunk, 0, st>>>(ids, n, V, ws.counts, dev_status);
   DP_LAUNCH_OK();
-  sort_chunk_prefix_kernel<<<ceil_div(V, 256), 256, 0, st>>>(ws.counts, ws.chunks, V, ws.seg);
+  sort_chunk_prefix_kernel<<<ceil_div(V, 1024), 1024, 0, st>>>(ws.counts, ws.chunks, V, ws.seg,
+                                                             ws.block_sums);
   DP_LAUNCH_OK();
-  sort_scan_kernel<<<1, 1024, 0, st>>>(ws.seg, V);
+  sort_scan_kernel<<<ceil_div(V, 1024), 1024, 0, st>>>(ws.seg, V, ws.block_sums);
   DP_LAUNCH_OK();
   sort_place_kernel<<<ws.chunks, kSortChunk, 0, st>>>(ids, n, V, ws.counts, ws.seg, ws.perm);
   DP_LAUNCH_OK();
@@ -272,7 +398,7 @@ dp_status launch_embed_scatter(const int* ids, const void* G, int64_t ldg, dp_dt
     DP_CUDA_OK(cudaMemset2DAsync(out, size_t(ldo) * sizeof(float), 0, size_t(d) * sizeof(float),
                                  size_t(V), st));
   }
-  dim3 grid(n, ceil_div(d, 128));
+  dim3 grid(n, ceil_div(d, kEmbedColsPerBlock));
   if (dt == DP_F32)
     embed_scatter_kernel<float><<<grid, 256, 0, st>>>(ids, (const float*)G, ldg, T, d, clip, perm,
                                                      seg, V, out, ldo, 1.f);
