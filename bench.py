@@ -195,14 +195,22 @@ def run_ours(args):
         # data-parallel exchange: clipped sums are added over ranks before the single noise draw
         parallel.reduce_clipped_sums(ds.outs)
 
+    fused = (world == 1) and not args.unfused     # noise inside the clipped-sum kernels
+
     def step(k, ev=None):
         if ev: ev[0].record(stream)
+        if fused:
+            filled = P.prefill_embedding_noise(ds, args.seed, k)     # side stream, overlaps the norms
         P.norms_phase(ds)
         if ev: ev[1].record(stream)
-        P.clip_phase(ds)
-        if ev: ev[2].record(stream)
-        reduce_sums()
-        P.noise_phase(ds, seed=args.seed, step=k)
+        if fused:
+            P.clip_after_prefill(ds, args.seed, k, filled)
+            if ev: ev[2].record(stream)
+        else:
+            P.clip_phase(ds)
+            if ev: ev[2].record(stream)
+            reduce_sums()
+            P.noise_phase(ds, seed=args.seed, step=k)
         if ev: ev[3].record(stream)
 
     for k in range(args.warmup):
@@ -253,8 +261,13 @@ def run_ours(args):
         gemm_outs.append(ds.outs["wte"] if ds.tied else ds.outs["lm_head"])
     for _ in range(max(3, min(args.steps, 10))):
         g0.record(stream)
-        dp.dp_clip_accumulate_grouped(lin_layers, ds.B, ds.T, ds.sq, ds.C, gemm_outs, ws=ds.ws,
-                                      dev_status=ds.dev_status)
+        if fused:
+            dp.dp_clip_accumulate_noise_grouped(lin_layers, ds.B, ds.T, ds.sq, ds.C, gemm_outs, ds.sigma,
+                                                1.0, args.seed, list(range(len(gemm_outs))), 0,
+                                                ws=ds.ws, dev_status=ds.dev_status)
+        else:
+            dp.dp_clip_accumulate_grouped(lin_layers, ds.B, ds.T, ds.sq, ds.C, gemm_outs, ws=ds.ws,
+                                          dev_status=ds.dev_status)
         g1.record(stream)
         torch.cuda.synchronize()
         gemm_ms.append(g0.elapsed_time(g1))
@@ -262,7 +275,10 @@ def run_ours(args):
     n_gemm = 1          # one persistent launch over the output tiles of all layers
     achieved_tf = counts["acc_flops"] / (gemm_ms_avg * 1e-3) / 1e12
     peak_tf = peaks["bf16_tflops_sustained"]
-    roofline = {"kernel": "gemm_gta_kernel<scale> (dp_clip_accumulate)", "bound": "tensor",
+    roofline = {"kernel": "gemm_gta_kernel<scale> (%s)" % ("dp_clip_accumulate_noise_grouped, noise "
+                                                          "drawn in the epilogue" if fused else
+                                                          "dp_clip_accumulate_grouped"),
+                "bound": "tensor",
                 "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
                 "frac": achieved_tf / peak_tf, "peak_source": peaks["source"] + " sustained bf16",
                 "launches_per_step": n_gemm, "ms_per_launch_avg": gemm_ms_avg / n_gemm,
@@ -280,16 +296,23 @@ def run_ours(args):
     ghost_tf = counts["gram_flops"] / (ghost_ms * 1e-3) / 1e12
     floor_ms = max(counts["norm_bytes"] / (peaks["hbm_gbs"] * 1e9),
                    counts["gram_flops"] / (peak_tf * 1e12)) * 1e3
+    big = ds.outs["wte"]
+    noise_n = big.numel()
+    g0.record(stream)
+    for k in range(reps):
+        dp.dp_add_noise(big, ds.sigma, ds.C, 1.0, args.seed, 0, k)
+    g1.record(stream)
+    torch.cuda.synchronize()
+    noise_ms = g0.elapsed_time(g1) / reps
     others = {
         "ghost_norm_tc_kernel (dp_ghost_norms)": {
             "bound": "hbm" if counts["norm_bytes"] / (peaks["hbm_gbs"] * 1e9) >=
             counts["gram_flops"] / (peak_tf * 1e12) else "tensor",
             "ms": ghost_ms, "achieved_GBs": ghost_gbs, "achieved_TFLOPs": ghost_tf,
             "peak_GBs": peaks["hbm_gbs"], "frac": floor_ms / ghost_ms},
-        "add_noise_kernel (dp_add_noise)": {
-            "bound": "hbm", "ms": ms_noise, "achieved_GBs": counts["noise_bytes"] / (ms_noise * 1e-3) / 1e9,
-            "peak_GBs": peaks["hbm_gbs"],
-            "frac": counts["noise_bytes"] / (ms_noise * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+        "add_noise_kernel (dp_add_noise, %d elements)" % noise_n: {
+            "bound": "hbm", "ms": noise_ms, "achieved_GBs": 8 * noise_n / (noise_ms * 1e-3) / 1e9,
+            "peak_GBs": peaks["hbm_gbs"], "frac": 8 * noise_n / (noise_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
     }
 
     # end to end through the public API with HOST buffers: every step copies the step's inputs
@@ -358,7 +381,8 @@ def run_ours(args):
                    "accumulate": "fp32", "input_bytes_per_step": ds.input_bytes(),
                    "l2": "inputs (%.2f GB per step) are larger than the 126 MB L2" % (ds.input_bytes() / 1e9)},
         "phases_ms": {"norms": ms_norm, "clip_accumulate": ms_clip, "noise": ms_noise,
-                      "norm_plus_clip": ms_norm + ms_clip},
+                      "norm_plus_clip": ms_norm + ms_clip,
+                      "noise_fused_into_clip_accumulate": fused},
         "gpu_launches": int(launches),
         "clocks": clocks,
         "roofline": roofline,
@@ -382,6 +406,8 @@ def main():
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--unfused", action="store_true",
+                    help="separate noise pass (what the multi-GPU path uses) instead of fused noise")
     args = ap.parse_args()
     if args.impl == "reference":
         if args.steps > 30:

@@ -152,6 +152,31 @@ dp_status dp_clip_accumulate_embed(const int32_t* ids, const void* G, int64_t ld
                                    void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
 size_t dp_clip_accumulate_embed_ws_bytes(int32_t B, int32_t T, int32_t d, int32_t V);
 
+/* ---- clipped sums with the Gaussian mechanism fused in (Eq. 2, Eq. 3, Eq. 7 in one pass) ----
+ * Same as dp_clip_accumulate_grouped, then outs[k] = scale * (outs[k] + sigma*C*z) with the
+ * stream (seed, tensor_ids[k], step) of dp_add_noise, element j = row*d + col.  The noise is
+ * generated in the GEMM epilogue, so the clipped sum is never re-read from memory.  Values are
+ * identical to calling dp_clip_accumulate_grouped and then dp_add_noise on each tensor.
+ * tensor_ids [host, n_layers].  Use the unfused calls when several devices must add their sums
+ * before the single noise draw. */
+dp_status dp_clip_accumulate_noise_grouped(const dp_linear_desc* layers, int32_t n_layers,
+                                           dp_dtype dt, int32_t B, int32_t T, const float* sq,
+                                           float C, float* clip, float* const* outs,
+                                           const int64_t* ldos, float beta, float sigma, float scale,
+                                           uint64_t seed, const uint32_t* tensor_ids, uint32_t step,
+                                           void* ws, size_t ws_bytes, int32_t* dev_status,
+                                           void* stream);
+/* Embedding table with the Gaussian mechanism: beta == 0 fills the table with scale*sigma*C*z
+ * (write only, in place of the zero fill) and adds scale * the clipped row sums; beta == 1 adds
+ * scale * the clipped row sums to a table that already holds its noise (tied head).  Equal to the
+ * unfused calls up to fp32 rounding order. */
+dp_status dp_clip_accumulate_embed_noise(const int32_t* ids, const void* G, int64_t ldg, dp_dtype dt,
+                                         int32_t B, int32_t T, int32_t d, int32_t V, const float* sq,
+                                         float C, float* clip, float* out, int64_t ldo, float beta,
+                                         float sigma, float scale, uint64_t seed, uint32_t tensor_id,
+                                         uint32_t step, int32_t* perm, int32_t* seg, void* ws,
+                                         size_t ws_bytes, int32_t* dev_status, void* stream);
+
 /* ---- Gaussian mechanism: out[j] = scale * (out[j] + sigma*C*z_j)  (Eq. 3) ----
  * z_j is a pure function of (seed, tensor_id, step, j): Philox4x32-10 with key
  * (seed low word, seed high word) and counter (j/4 low, j/4 high, tensor_id, step); word
@@ -161,6 +186,12 @@ size_t dp_clip_accumulate_embed_ws_bytes(int32_t B, int32_t T, int32_t d, int32_
  * scale = 1/|B| the full Eq. 3.  sigma >= 0, C > 0, all finite. */
 dp_status dp_add_noise(float* out, int64_t n, float sigma, float C, float scale,
                        uint64_t seed, uint32_t tensor_id, uint32_t step, void* stream);
+
+/* Write-only form: out[j] = scale * sigma*C*z_j, the same stream as dp_add_noise on a zero
+ * buffer.  It depends on no gradient, so it can run on a second stream while the norms are
+ * computed; the clipped sums are then accumulated on top with beta = 1. */
+dp_status dp_fill_noise(float* out, int64_t n, float sigma, float C, float scale,
+                        uint64_t seed, uint32_t tensor_id, uint32_t step, void* stream);
 
 /* ---- helpers ---- */
 const char* dp_status_string(dp_status s);

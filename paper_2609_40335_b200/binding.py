@@ -37,8 +37,9 @@ class _LinearDesc(C.Structure):
 EXPORTS = ["dp_ghost_norms", "dp_ghost_norms_ws_bytes", "dp_embed_norms", "dp_embed_norms_ws_bytes",
            "dp_tied_cross_term", "dp_tied_cross_term_ws_bytes", "dp_clip_factors",
            "dp_clip_accumulate", "dp_clip_accumulate_ws_bytes", "dp_clip_accumulate_grouped",
-           "dp_clip_accumulate_grouped_ws_bytes", "dp_clip_accumulate_embed",
-           "dp_clip_accumulate_embed_ws_bytes", "dp_add_noise", "dp_status_string",
+           "dp_clip_accumulate_grouped_ws_bytes", "dp_clip_accumulate_noise_grouped",
+           "dp_clip_accumulate_embed_noise", "dp_clip_accumulate_embed",
+           "dp_clip_accumulate_embed_ws_bytes", "dp_add_noise", "dp_fill_noise", "dp_status_string",
            "dp_last_cuda_error", "dp_version", "dp_kernel_launches", "dp_debug_force_fma"]
 
 
@@ -74,11 +75,19 @@ def load():
                                              C.POINTER(vp), C.POINTER(i64), f32, vp, sz, vp, vp]
     L.dp_clip_accumulate_grouped_ws_bytes.argtypes = [C.POINTER(_LinearDesc), i32, i32, i32, i32]
     L.dp_clip_accumulate_grouped_ws_bytes.restype = sz
+    L.dp_clip_accumulate_noise_grouped.argtypes = [C.POINTER(_LinearDesc), i32, i32, i32, i32, vp, f32,
+                                                   vp, C.POINTER(vp), C.POINTER(i64), f32, f32, f32,
+                                                   C.c_uint64, C.POINTER(C.c_uint32), C.c_uint32,
+                                                   vp, sz, vp, vp]
+    L.dp_clip_accumulate_embed_noise.argtypes = [vp, vp, i64, i32, i32, i32, i32, i32, vp, f32, vp, vp,
+                                                 i64, f32, f32, f32, C.c_uint64, C.c_uint32,
+                                                 C.c_uint32, vp, vp, vp, sz, vp, vp]
     L.dp_clip_accumulate_embed.argtypes = [vp, vp, i64, i32, i32, i32, i32, i32, vp, f32, vp, vp, i64,
                                            f32, vp, vp, vp, sz, vp, vp]
     L.dp_clip_accumulate_embed_ws_bytes.argtypes = [i32, i32, i32, i32]
     L.dp_clip_accumulate_embed_ws_bytes.restype = sz
     L.dp_add_noise.argtypes = [vp, i64, f32, f32, f32, C.c_uint64, C.c_uint32, C.c_uint32, vp]
+    L.dp_fill_noise.argtypes = [vp, i64, f32, f32, f32, C.c_uint64, C.c_uint32, C.c_uint32, vp]
     L.dp_status_string.argtypes = [i32]
     L.dp_status_string.restype = C.c_char_p
     L.dp_last_cuda_error.restype = i32
@@ -265,6 +274,47 @@ def dp_clip_accumulate_grouped(layers: Sequence[Linear], B: int, T: int, sq, C_:
     _check(st, "dp_clip_accumulate_grouped")
 
 
+def dp_clip_accumulate_noise_grouped(layers: Sequence[Linear], B: int, T: int, sq, C_: float,
+                                     outs: Sequence[torch.Tensor], sigma: float, scale: float,
+                                     seed: int, tensor_ids: Sequence[int], step: int,
+                                     beta: float = 0.0, clip=None, ws=None, dev_status=None,
+                                     stream=None):
+    """Clipped sums of every layer with the Gaussian noise added in the GEMM epilogue."""
+    L = load()
+    arr = _descs(layers)
+    dt = _dt(layers[0].A)
+    n = len(layers)
+    optr = (C.c_void_p * n)(*[_ptr(o) for o in outs])
+    ldos = (C.c_int64 * n)(*[o.stride(0) for o in outs])
+    tids = (C.c_uint32 * n)(*[int(t) for t in tensor_ids])
+    need = int(L.dp_clip_accumulate_grouped_ws_bytes(arr, n, dt, B, T))
+    ws = _ws(need, ws, outs[0].device)
+    st = L.dp_clip_accumulate_noise_grouped(arr, n, dt, B, T, _ptr(sq), float(C_), _ptr(clip), optr,
+                                            ldos, float(beta), float(sigma), float(scale),
+                                            int(seed) & (2 ** 64 - 1), tids, int(step), _ptr(ws),
+                                            ws.numel() * ws.element_size(), _ptr(dev_status),
+                                            _stream(stream))
+    _check(st, "dp_clip_accumulate_noise_grouped")
+
+
+def dp_clip_accumulate_embed_noise(ids, G, V: int, sq, C_: float, out, sigma: float, scale: float,
+                                   seed: int, tensor_id: int, step: int, beta: float = 0.0, d=None,
+                                   clip=None, perm=None, seg=None, ws=None, dev_status=None,
+                                   stream=None):
+    L = load()
+    B, T = ids.shape
+    d = d if d is not None else G.shape[-1]
+    need = int(L.dp_clip_accumulate_embed_ws_bytes(B, T, d, V))
+    ws = _ws(need, ws, out.device)
+    st = L.dp_clip_accumulate_embed_noise(_ptr(ids), _ptr(G), _rows_ld(G), _dt(G), B, T, d, V, _ptr(sq),
+                                          float(C_), _ptr(clip), _ptr(out), out.stride(0), float(beta),
+                                          float(sigma), float(scale), int(seed) & (2 ** 64 - 1),
+                                          int(tensor_id), int(step), _ptr(perm), _ptr(seg), _ptr(ws),
+                                          ws.numel() * ws.element_size(), _ptr(dev_status),
+                                          _stream(stream))
+    _check(st, "dp_clip_accumulate_embed_noise")
+
+
 def dp_clip_accumulate_embed(ids, G, V: int, sq, C_: float, out, beta: float = 0.0, d=None,
                              clip=None, perm=None, seg=None, ws=None, dev_status=None, stream=None):
     L = load()
@@ -287,6 +337,16 @@ def dp_add_noise(out: torch.Tensor, sigma: float, C_: float, scale: float, seed:
     st = L.dp_add_noise(_ptr(out), n, float(sigma), float(C_), float(scale), int(seed) & (2 ** 64 - 1),
                         int(tensor_id), int(step), _stream(stream))
     _check(st, "dp_add_noise")
+
+
+def dp_fill_noise(out: torch.Tensor, sigma: float, C_: float, scale: float, seed: int,
+                  tensor_id: int, step: int, n=None, stream=None):
+    """out = scale * sigma*C*z (write only), z from the (seed, tensor_id, step) stream."""
+    L = load()
+    n = out.numel() if n is None else n
+    st = L.dp_fill_noise(_ptr(out), n, float(sigma), float(C_), float(scale), int(seed) & (2 ** 64 - 1),
+                         int(tensor_id), int(step), _stream(stream))
+    _check(st, "dp_fill_noise")
 
 
 def dp_debug_force_fma(on: bool) -> bool:

@@ -226,10 +226,11 @@ size_t dp_clip_accumulate_grouped_ws_bytes(const dp_linear_desc* layers, int32_t
   return n;
 }
 
-dp_status dp_clip_accumulate_grouped(const dp_linear_desc* layers, int32_t n_layers, dp_dtype dt,
-                                     int32_t B, int32_t T, const float* sq, float C, float* clip,
-                                     float* const* outs, const int64_t* ldos, float beta, void* ws,
-                                     size_t ws_bytes, int32_t* dev_status, void* stream) {
+static dp_status clip_accumulate_impl(const dp_linear_desc* layers, int32_t n_layers, dp_dtype dt,
+                                      int32_t B, int32_t T, const float* sq, float C, float* clip,
+                                      float* const* outs, const int64_t* ldos, float beta,
+                                      const GtaNoise* noise, void* ws, size_t ws_bytes,
+                                      int32_t* dev_status, void* stream) {
   if (!layers || n_layers <= 0 || !outs || !ldos || !sq || B <= 0 || T <= 0) return DP_ERR_INVALID_ARG;
   if (dt != DP_F32 && dt != DP_BF16) return DP_ERR_INVALID_ARG;
   if (!(beta == 0.f || beta == 1.f) || !finite_pos(C)) return DP_ERR_INVALID_ARG;
@@ -254,13 +255,43 @@ dp_status dp_clip_accumulate_grouped(const dp_linear_desc* layers, int32_t n_lay
       s = launch_clip_accumulate_fma(layers[l].A, layers[l].lda, layers[l].G, layers[l].ldg, dt, B, T,
                                      layers[l].d, layers[l].p, clip_ws, outs[l], ldos[l], beta, st);
       if (s != DP_OK) return s;
+      if (noise) {
+        s = launch_add_noise(outs[l], layers[l].p, layers[l].d, ldos[l], false, noise->amp,
+                             noise->scale, noise->seed, noise->tensor_ids[l], noise->step, st);
+        if (s != DP_OK) return s;
+      }
     }
     return DP_OK;
   }
   float* partial = reinterpret_cast<float*>(static_cast<char*>(ws) +
                                             align_up(size_t(B) * sizeof(float), 256));
-  return launch_clip_accumulate_tc(layers, n_layers, B, T, clip_ws, outs, ldos, beta, partial,
+  return launch_clip_accumulate_tc(layers, n_layers, B, T, clip_ws, outs, ldos, beta, noise, partial,
                                    dev_status, st);
+}
+
+dp_status dp_clip_accumulate_grouped(const dp_linear_desc* layers, int32_t n_layers, dp_dtype dt,
+                                     int32_t B, int32_t T, const float* sq, float C, float* clip,
+                                     float* const* outs, const int64_t* ldos, float beta, void* ws,
+                                     size_t ws_bytes, int32_t* dev_status, void* stream) {
+  return clip_accumulate_impl(layers, n_layers, dt, B, T, sq, C, clip, outs, ldos, beta, nullptr, ws,
+                              ws_bytes, dev_status, stream);
+}
+
+static bool noise_args_ok(float sigma, float C, float scale) {
+  return std::isfinite(sigma) && sigma >= 0.f && finite_pos(C) && std::isfinite(scale);
+}
+
+dp_status dp_clip_accumulate_noise_grouped(const dp_linear_desc* layers, int32_t n_layers,
+                                           dp_dtype dt, int32_t B, int32_t T, const float* sq,
+                                           float C, float* clip, float* const* outs,
+                                           const int64_t* ldos, float beta, float sigma, float scale,
+                                           uint64_t seed, const uint32_t* tensor_ids, uint32_t step,
+                                           void* ws, size_t ws_bytes, int32_t* dev_status,
+                                           void* stream) {
+  if (!tensor_ids || !noise_args_ok(sigma, C, scale)) return DP_ERR_INVALID_ARG;
+  const GtaNoise noise{sigma * C, scale, seed, step, tensor_ids};
+  return clip_accumulate_impl(layers, n_layers, dt, B, T, sq, C, clip, outs, ldos, beta, &noise, ws,
+                              ws_bytes, dev_status, stream);
 }
 
 static dp_linear_desc one_layer(const void* A, int64_t lda, const void* G, int64_t ldg, int32_t d,
@@ -312,11 +343,14 @@ size_t dp_clip_accumulate_embed_ws_bytes(int32_t B, int32_t T, int32_t d, int32_
   return total;
 }
 
-dp_status dp_clip_accumulate_embed(const int32_t* ids, const void* G, int64_t ldg, dp_dtype dt,
-                                   int32_t B, int32_t T, int32_t d, int32_t V, const float* sq,
-                                   float C, float* clip, float* out, int64_t ldo, float beta,
-                                   int32_t* perm, int32_t* seg, void* ws, size_t ws_bytes,
-                                   int32_t* dev_status, void* stream) {
+struct EmbedNoise { float amp, scale; uint64_t seed; uint32_t tensor_id, step; };
+
+static dp_status clip_accumulate_embed_impl(const int32_t* ids, const void* G, int64_t ldg,
+                                            dp_dtype dt, int32_t B, int32_t T, int32_t d, int32_t V,
+                                            const float* sq, float C, float* clip, float* out,
+                                            int64_t ldo, float beta, const EmbedNoise* noise,
+                                            int32_t* perm, int32_t* seg, void* ws, size_t ws_bytes,
+                                            int32_t* dev_status, void* stream) {
   if (!ids || !G || !sq || !out || B <= 0 || T <= 0 || d <= 0 || V <= 0) return DP_ERR_INVALID_ARG;
   if (ldg < d || ldo < d) return DP_ERR_INVALID_ARG;
   if (dt != DP_F32 && dt != DP_BF16) return DP_ERR_INVALID_ARG;
@@ -345,8 +379,42 @@ dp_status dp_clip_accumulate_embed(const int32_t* ids, const void* G, int64_t ld
                                        cudaMemcpyDeviceToDevice, st));
   if (seg) DP_CUDA_OK(cudaMemcpyAsync(seg, sw.seg, size_t(V + 1) * sizeof(int),
                                       cudaMemcpyDeviceToDevice, st));
+  // With noise and beta == 0 the table is filled with scale*sigma*C*z (write only) in place of
+  // the zero fill; with beta == 1 the noise was already drawn by whoever wrote the table first.
+  bool clear = true;
+  float scale = 1.f;
+  if (noise) {
+    scale = noise->scale;
+    if (beta == 0.f) {
+      s = launch_add_noise(out, V, d, ldo, true, noise->amp, noise->scale, noise->seed,
+                           noise->tensor_id, noise->step, st);
+      if (s != DP_OK) return s;
+      clear = false;
+    }
+  }
   return launch_embed_scatter(ids, G, ldg, dt, n, T, d, V, clip_ws, sw.perm, sw.seg, out, ldo, beta,
-                              st);
+                              scale, clear, st);
+}
+
+dp_status dp_clip_accumulate_embed(const int32_t* ids, const void* G, int64_t ldg, dp_dtype dt,
+                                   int32_t B, int32_t T, int32_t d, int32_t V, const float* sq,
+                                   float C, float* clip, float* out, int64_t ldo, float beta,
+                                   int32_t* perm, int32_t* seg, void* ws, size_t ws_bytes,
+                                   int32_t* dev_status, void* stream) {
+  return clip_accumulate_embed_impl(ids, G, ldg, dt, B, T, d, V, sq, C, clip, out, ldo, beta, nullptr,
+                                    perm, seg, ws, ws_bytes, dev_status, stream);
+}
+
+dp_status dp_clip_accumulate_embed_noise(const int32_t* ids, const void* G, int64_t ldg, dp_dtype dt,
+                                         int32_t B, int32_t T, int32_t d, int32_t V, const float* sq,
+                                         float C, float* clip, float* out, int64_t ldo, float beta,
+                                         float sigma, float scale, uint64_t seed, uint32_t tensor_id,
+                                         uint32_t step, int32_t* perm, int32_t* seg, void* ws,
+                                         size_t ws_bytes, int32_t* dev_status, void* stream) {
+  if (!noise_args_ok(sigma, C, scale)) return DP_ERR_INVALID_ARG;
+  const EmbedNoise noise{sigma * C, scale, seed, tensor_id, step};
+  return clip_accumulate_embed_impl(ids, G, ldg, dt, B, T, d, V, sq, C, clip, out, ldo, beta, &noise,
+                                    perm, seg, ws, ws_bytes, dev_status, stream);
 }
 
 // ----------------------------------------------------------------------------------- noise
@@ -356,7 +424,18 @@ dp_status dp_add_noise(float* out, int64_t n, float sigma, float C, float scale,
   if (!std::isfinite(sigma) || sigma < 0.f || !finite_pos(C) || !std::isfinite(scale))
     return DP_ERR_INVALID_ARG;
   if (!aligned16(out)) return DP_ERR_ALIGNMENT;
-  return launch_add_noise(out, n, sigma * C, scale, seed, tensor_id, step, (cudaStream_t)stream);
+  // a flat buffer is the (n, 1) tensor with pitch 1
+  return launch_add_noise(out, n, 1, 1, false, sigma * C, scale, seed, tensor_id, step,
+                          (cudaStream_t)stream);
+}
+
+dp_status dp_fill_noise(float* out, int64_t n, float sigma, float C, float scale, uint64_t seed,
+                        uint32_t tensor_id, uint32_t step, void* stream) {
+  if (!out || n < 0) return DP_ERR_INVALID_ARG;
+  if (!noise_args_ok(sigma, C, scale)) return DP_ERR_INVALID_ARG;
+  if (!aligned16(out)) return DP_ERR_ALIGNMENT;
+  return launch_add_noise(out, n, 1, 1, true, sigma * C, scale, seed, tensor_id, step,
+                          (cudaStream_t)stream);
 }
 
 }  // extern "C"

@@ -283,7 +283,7 @@ __global__ void __launch_bounds__(256)
 embed_scatter_kernel(const int* __restrict__ ids, const T* __restrict__ G, long long ldg, int Tn,
                      int d, const float* __restrict__ clip, const int* __restrict__ perm,
                      const int* __restrict__ seg, int V, float* __restrict__ out, long long ldo,
-                     float beta) {
+                     float beta, float scale) {
   __shared__ float part[8][kEmbedColsPerBlock];
   __shared__ int s_pos[kScatStage];
   __shared__ float s_r[kScatStage];
@@ -342,6 +342,7 @@ embed_scatter_kernel(const int* __restrict__ ids, const T* __restrict__ G, long 
 #pragma unroll
       for (int ww = 0; ww < 8; ++ww) s += part[ww][threadIdx.x];
       float* o = out + size_t(v) * ldo + cc;
+      s *= scale;
       *o = (beta != 0.f) ? (*o + s) : s;
     }
   }
@@ -391,20 +392,22 @@ dp_status launch_embed_sort(const int* ids, int n, int V, const EmbedSortWs& ws,
 
 dp_status launch_embed_scatter(const int* ids, const void* G, int64_t ldg, dp_dtype dt, int n,
                                int T, int d, int V, const float* clip, const int* perm,
-                               const int* seg, float* out, int64_t ldo, float beta,
-                               cudaStream_t st) {
-  // beta == 0: clear the table once, then every touched row is written as 0 + sum
-  if (beta == 0.f) {
+                               const int* seg, float* out, int64_t ldo, float beta, float scale,
+                               bool clear, cudaStream_t st) {
+  // beta == 0: the table is cleared once (unless the caller already filled it, e.g. with
+  // noise), then every touched row receives table + scale*sum
+  if (beta == 0.f && clear) {
     DP_CUDA_OK(cudaMemset2DAsync(out, size_t(ldo) * sizeof(float), 0, size_t(d) * sizeof(float),
                                  size_t(V), st));
   }
   dim3 grid(n, ceil_div(d, kEmbedColsPerBlock));
   if (dt == DP_F32)
     embed_scatter_kernel<float><<<grid, 256, 0, st>>>(ids, (const float*)G, ldg, T, d, clip, perm,
-                                                     seg, V, out, ldo, 1.f);
+                                                     seg, V, out, ldo, 1.f, scale);
   else
     embed_scatter_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(ids, (const __nv_bfloat16*)G, ldg, T,
-                                                             d, clip, perm, seg, V, out, ldo, 1.f);
+                                                             d, clip, perm, seg, V, out, ldo, 1.f,
+                                                             scale);
   DP_LAUNCH_OK();
   return DP_OK;
 }

@@ -37,10 +37,13 @@ dp_status launch_embed_sort(const int* ids, int n, int V, const EmbedSortWs& ws,
                             cudaStream_t st);
 dp_status launch_embed_scatter(const int* ids, const void* G, int64_t ldg, dp_dtype dt, int n,
                                int T, int d, int V, const float* clip, const int* perm,
-                               const int* seg, float* out, int64_t ldo, float beta,
-                               cudaStream_t st);
+                               const int* seg, float* out, int64_t ldo, float beta, float scale,
+                               bool clear, cudaStream_t st);
 
-dp_status launch_add_noise(float* out, long long n, float amp, float scale, uint64_t seed,
-                           uint32_t tensor_id, uint32_t step, cudaStream_t st);
+// logical (rows, cols) tensor with row pitch ld; element j = row*cols + col of the stream.
+// fill: write scale*amp*z without reading out.
+dp_status launch_add_noise(float* out, long long rows, int cols, long long ld, bool fill, float amp,
+                           float scale, uint64_t seed, uint32_t tensor_id, uint32_t step,
+                           cudaStream_t st);
 
 }  // namespace dpg

@@ -2,6 +2,7 @@
 #pragma once
 
 #include "dp_common.cuh"
+#include "fma_kernels.cuh"
 #include "ghost_plan.cuh"
 
 namespace dpg {
@@ -20,6 +21,16 @@ struct GtaLayer {
   int item_begin;
   int col_begin;          // square-sum mode: first partial-sum column of this layer
   float beta;
+  float noise_amp;        // sigma*C of the fused noise, negative = none
+  uint32_t tensor_id;     // noise stream id of this output tensor
+};
+
+// Fused Gaussian mechanism of a grouped call (host side).
+struct GtaNoise {
+  float amp, scale;
+  uint64_t seed;
+  uint32_t step;
+  const uint32_t* tensor_ids;   // [n_layers]
 };
 
 int gta_choose_nsplit(const dp_linear_desc* layers, int n_layers, int B, int T, int sms);
@@ -28,8 +39,8 @@ size_t gta_partial_bytes(const dp_linear_desc* layers, int n_layers, int B, int 
 // One persistent launch over the output tiles of all layers (plus split-K reduces if needed).
 dp_status launch_clip_accumulate_tc(const dp_linear_desc* layers, int n_layers, int B, int T,
                                     const float* clip, float* const* outs, const int64_t* ldos,
-                                    float beta, float* partial_ws, int* dev_status,
-                                    cudaStream_t st);
+                                    float beta, const GtaNoise* noise, float* partial_ws,
+                                    int* dev_status, cudaStream_t st);
 
 dp_status launch_direct_norm_tc(const dp_linear_desc* layers, const GhostPlan& plan, int B, int T,
                                 float* partials, int* dev_status, cudaStream_t st);

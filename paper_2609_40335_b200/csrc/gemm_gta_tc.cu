@@ -9,12 +9,14 @@
 // memory holds MN-major tiles: every TMA box is 64 token rows x 64 columns (128-byte rows,
 // 128-byte swizzle).  A K step never straddles two examples (the tensor map is 3-D:
 // column, token, example; the token tail of an example is zero-filled), so one clip factor
-// applies to a whole stage: eight "scaler" warps multiply the G tile by R_i in shared memory
+// applies to a whole stage: four "scaler" warps multiply the G tile by R_i in shared memory
 // (packed bf16 FMAs with R_i split into two bf16 parts) between the TMA-full and MMA-ready
 // barriers.
 //
-// Roles per CTA (448 threads): warp 0 TMA producer, warp 1 MMA issuer, warps 2-9 scalers,
-// warps 10-13 epilogue; two TMEM accumulators overlap the epilogue with the next tile.
+// Roles per CTA (576 threads): warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 scalers,
+// warps 6-17 epilogue (three per TMEM lane quarter, sharing the 256 columns 3+3+2 chunks; they
+// also draw the fused Gaussian noise); two TMEM accumulators overlap the epilogue with the
+// next tile.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -23,6 +25,7 @@
 
 #include "dp_common.cuh"
 #include "gemm_gta.cuh"
+#include "noise_device.cuh"
 #include "ptx_sm100.cuh"
 #include "tma_host.cuh"
 
@@ -39,9 +42,13 @@ constexpr int kStageBytes = kGBytes + kABytes;      // 48 KiB
 #define DPG_GTA_STAGES 4
 #endif
 constexpr int kStages = DPG_GTA_STAGES;
-constexpr int kScalerWarps = 8;
+constexpr int kScalerWarps = 4;
 constexpr int kEpiWarp0 = 2 + kScalerWarps;          // first epilogue warp
-constexpr int kThreads = (kEpiWarp0 + 4) * 32;
+#ifndef DPG_GTA_EPI_WARPS
+#define DPG_GTA_EPI_WARPS 12
+#endif
+constexpr int kEpiWarps = DPG_GTA_EPI_WARPS;         // kEpiWarps/4 per TMEM lane quarter (column groups)
+constexpr int kThreads = (kEpiWarp0 + kEpiWarps) * 32;
 constexpr int kTmemCols = 512;                      // 2 accumulators x 256 columns
 constexpr size_t kSmemBytes = size_t(kStages) * kStageBytes + 1024 + 256;
 
@@ -53,6 +60,8 @@ struct __align__(64) GtaParams {
   int B, T, tsteps;          // tsteps = ceil(T / 64) K steps per example
   int total_items;
   const float* clip;         // [B] R_i (scale mode)
+  uint32_t noise_k0, noise_k1, noise_step;   // Gaussian stream of the fused noise (per-layer id)
+  float noise_scale;
   float* sq_partials;        // [B][n_per] (square-sum mode)
   int n_per;
   int* dev_status;
@@ -98,7 +107,7 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
   uint64_t* acc_empty = acc_full + 2;         // [2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  float* epi_red = reinterpret_cast<float*>(tmem_slot + 2);   // [2][4]
+  float* epi_red = reinterpret_cast<float*>(tmem_slot + 2);   // [2][kEpiWarps]
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -109,7 +118,7 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
       ptx::mbar_init(&ready[s], kScalerWarps);
       ptx::mbar_init(&empty[s], 1);
     }
-    for (int b = 0; b < 2; ++b) { ptx::mbar_init(&acc_full[b], 1); ptx::mbar_init(&acc_empty[b], 4); }
+    for (int b = 0; b < 2; ++b) { ptx::mbar_init(&acc_full[b], 1); ptx::mbar_init(&acc_empty[b], kEpiWarps); }
     *abort_flag = 0;
     ptx::fence_mbar_init();
   }
@@ -234,8 +243,11 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
     }
   } else {
     // ----------------------------------------------------------------- epilogue
-    const int q = warp & 3;
+    const int q = warp & 3;                          // TMEM lane quarter this warp may read
     const int ew = warp - kEpiWarp0;
+    // this warp's 32-column chunks: the 8 chunks are dealt to the kEpiWarps/4 column groups
+    constexpr int kGroups = kEpiWarps / 4;
+    const int c_lo = ((ew >> 2) * (kBN / 32)) / kGroups, c_hi = (((ew >> 2) + 1) * (kBN / 32)) / kGroups;
     uint32_t n_item = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x, ++n_item) {
@@ -249,7 +261,7 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
       if (kSqsum) {
         float acc = 0.f;
 #pragma unroll 1
-        for (int c = 0; c < kBN / 32; ++c) {
+        for (int c = c_lo; c < c_hi; ++c) {
           uint32_t r[32];
           ptx::tmem_ld_32x32b_x32(t0 + c * 32, r);
           ptx::tmem_ld_wait();
@@ -260,11 +272,12 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&acc_empty[buf]);
         acc = warp_sum(acc);
-        if (lane == 0) epi_red[buf * 4 + ew] = acc;
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (lane == 0) epi_red[buf * kEpiWarps + ew] = acc;
+        asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
         if (ew == 0 && lane == 0) {
-          const float s = (epi_red[buf * 4 + 0] + epi_red[buf * 4 + 1]) +
-                          (epi_red[buf * 4 + 2] + epi_red[buf * 4 + 3]);
+          float s = 0.f;
+#pragma unroll
+          for (int e = 0; e < kEpiWarps; ++e) s += epi_red[buf * kEpiWarps + e];
           P.sq_partials[size_t(it.example) * P.n_per + L.col_begin + it.tm * L.tiles_n + it.tn] = s;
         }
       } else {
@@ -275,34 +288,56 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
         if (L.nsplit == 1) { dst = L.out; ld = L.ldo; beta = L.beta; }
         else { dst = L.partial + size_t(it.split) * size_t(L.M) * L.N; ld = L.N; beta = 0.f; }
         const bool vec_ok = ((ld & 3) == 0) && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0);
+        // fused Gaussian mechanism (Eq. 3): only on the final destination, never on a K-split plane
+        const bool noisy = (L.noise_amp >= 0.f) && (L.nsplit == 1);
+        const NoiseKey nkey{P.noise_k0, P.noise_k1, L.tensor_id, P.noise_step};
 #pragma unroll 1
-        for (int c = 0; c < kBN / 32; ++c) {
+        for (int c = c_lo; c < c_hi; ++c) {
           uint32_t r[32];
           ptx::tmem_ld_32x32b_x32(t0 + c * 32, r);
           ptx::tmem_ld_wait();
           const int col0 = it.tn * kBN + c * 32;
           if (row < L.M && col0 < L.N) {
             float* o = dst + size_t(row) * ld + col0;
-            if (vec_ok && col0 + 32 <= L.N) {
+            const bool full32 = col0 + 32 <= L.N;
+            float v[32];
 #pragma unroll
-              for (int j = 0; j < 8; ++j) {
-                float4 v = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
-                                       __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
-                if (beta != 0.f) {
+            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+            if (beta != 0.f) {
+              if (vec_ok && full32) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
                   const float4 old = *reinterpret_cast<const float4*>(o + 4 * j);
-                  v.x += old.x; v.y += old.y; v.z += old.z; v.w += old.w;
+                  v[4 * j] += old.x; v[4 * j + 1] += old.y; v[4 * j + 2] += old.z; v[4 * j + 3] += old.w;
                 }
-                *reinterpret_cast<float4*>(o + 4 * j) = v;
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) if (col0 + j < L.N) v[j] += o[j];
               }
+            }
+            if (noisy) {
+              const unsigned long long j0 = (unsigned long long)row * L.N + col0;   // stream index
+              // N is a multiple of 4 here (the host fuses only such layers), so the Philox
+              // counters of this thread's 32 columns never straddle a row
+#pragma unroll
+              for (int qd = 0; qd < 8; ++qd) {
+                if (col0 + 4 * qd < L.N) {
+                  float z[4];
+                  normals4((j0 >> 2) + qd, nkey, z);
+#pragma unroll
+                  for (int e = 0; e < 4; ++e)
+                    v[4 * qd + e] = noised(v[4 * qd + e], z[e], L.noise_amp, P.noise_scale);
+                }
+              }
+            }
+            if (vec_ok && full32) {
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                *reinterpret_cast<float4*>(o + 4 * j) =
+                    make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
             } else {
 #pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                if (col0 + j < L.N) {
-                  float v = __uint_as_float(r[j]);
-                  if (beta != 0.f) v += o[j];
-                  o[j] = v;
-                }
-              }
+              for (int j = 0; j < 32; ++j) if (col0 + j < L.N) o[j] = v[j];
             }
           }
         }
@@ -382,8 +417,8 @@ size_t gta_partial_bytes(const dp_linear_desc* layers, int n_layers, int B, int 
 
 dp_status launch_clip_accumulate_tc(const dp_linear_desc* layers, int n_layers, int B, int T,
                                     const float* clip, float* const* outs, const int64_t* ldos,
-                                    float beta, float* partial_ws, int* dev_status,
-                                    cudaStream_t st) {
+                                    float beta, const GtaNoise* noise, float* partial_ws,
+                                    int* dev_status, cudaStream_t st) {
   dp_status s = set_attr_once<kClipScale, false>();
   if (s != DP_OK) return s;
   const int sms = sm_count();
@@ -415,7 +450,16 @@ dp_status launch_clip_accumulate_tc(const dp_linear_desc* layers, int n_layers, 
         pw += align_up(size_t(nsplit) * size_t(D.p) * size_t(D.d) * sizeof(float), 256);
       }
       L.item_begin = items; L.col_begin = 0;
+      // noise is drawn in the epilogue when the layer is not K-split and its width is a
+      // multiple of 4; otherwise a stand-alone pass follows (negative amp: no fused noise)
+      const bool fuse = noise && nsplit == 1 && (D.d % 4 == 0);
+      L.noise_amp = fuse ? noise->amp : -1.f;
+      L.tensor_id = noise ? noise->tensor_ids[g] : 0u;
       items += L.tiles_m * L.tiles_n * nsplit;
+    }
+    if (noise) {
+      P.noise_k0 = uint32_t(noise->seed); P.noise_k1 = uint32_t(noise->seed >> 32);
+      P.noise_step = noise->step; P.noise_scale = noise->scale;
     }
     P.n_layers = g1 - g0; P.B = B; P.T = T; P.tsteps = tsteps;
     P.total_items = items;
@@ -424,13 +468,19 @@ dp_status launch_clip_accumulate_tc(const dp_linear_desc* layers, int n_layers, 
     const int grid = std::min(items, sms);
     gemm_gta_kernel<kClipScale, false><<<grid, kThreads, kSmemBytes, st>>>(P);
     DP_LAUNCH_OK();
-    if (nsplit > 1) {
-      for (int g = g0; g < g1; ++g) {
-        const GtaLayer& L = P.layer[g - g0];
+    for (int g = g0; g < g1; ++g) {
+      const GtaLayer& L = P.layer[g - g0];
+      if (nsplit > 1) {
         const size_t total = size_t(L.M) * L.N;
         const int blocks = (int)std::min<size_t>((total + 255) / 256, size_t(sms) * 8);
         splitk_reduce_kernel<<<blocks, 256, 0, st>>>(L.partial, nsplit, L.M, L.N, L.out, L.ldo, beta);
         DP_LAUNCH_OK();
+      }
+      if (noise && L.noise_amp < 0.f) {        // not fused for this layer: stand-alone pass
+        const dp_status ns = launch_add_noise(L.out, L.M, L.N, L.ldo, false, noise->amp,
+                                              noise->scale, noise->seed, noise->tensor_ids[g],
+                                              noise->step, st);
+        if (ns != DP_OK) return ns;
       }
     }
   }

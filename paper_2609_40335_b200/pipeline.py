@@ -51,7 +51,7 @@ class DeviceStep:
     dev_status: torch.Tensor
     outs: Dict[str, torch.Tensor] = field(default_factory=dict)
     ws: Optional[torch.Tensor] = None
-    launches_per_step: int = 0
+    side_stream: Optional[torch.cuda.Stream] = None     # noise fills that overlap the norm phase
 
     def input_bytes(self) -> int:
         n = self.ids.numel() * 4 + self.G_emb.numel() * self.G_emb.element_size()
@@ -155,8 +155,93 @@ def noise_phase(ds: DeviceStep, seed: int, step: int, scale: float = 1.0, stream
         dp.dp_add_noise(ds.outs[name], ds.sigma, ds.C, scale, seed, tid, step, stream=stream)
 
 
-def dp_step(ds: DeviceStep, seed: int = 0, step: int = 0, noise: bool = True, stream=None) -> None:
+def tensor_ids(ds: DeviceStep) -> Dict[str, int]:
+    return {name: tid for tid, name in enumerate(sorted(ds.outs))}
+
+
+def clip_noise_phase(ds: DeviceStep, seed: int, step: int, scale: float = 1.0, stream=None) -> None:
+    """Clipped sums with the noise fused in: same values as clip_phase + noise_phase, but the
+    linear-layer noise is generated in the GEMM epilogue and the embedding table is filled with
+    its noise instead of zeros (single-device use: no exchange between sum and noise)."""
+    kw = dict(ws=ds.ws, dev_status=ds.dev_status, stream=stream)
+    tid = tensor_ids(ds)
+    layers = list(ds.linears)
+    names = [f"linear{k}" for k in range(len(ds.linears))]
+    if ds.lm is not None:
+        layers.append(ds.lm)
+        names.append("wte" if ds.tied else "lm_head")
+    if layers:
+        dp.dp_clip_accumulate_noise_grouped(layers, ds.B, ds.T, ds.sq, ds.C, [ds.outs[n] for n in names],
+                                            ds.sigma, scale, seed, [tid[n] for n in names], step,
+                                            beta=0.0, **kw)
+    dp.dp_clip_accumulate_embed_noise(ds.ids, ds.G_emb, ds.V, ds.sq, ds.C, ds.outs["wte"], ds.sigma,
+                                      scale, seed, tid["wte"], step,
+                                      beta=1.0 if (ds.tied and ds.lm is not None) else 0.0,
+                                      d=ds.d_model, **kw)
+    if ds.positions:
+        dp.dp_clip_accumulate_embed_noise(ds.pos_ids, ds.G_emb, WPE_ROWS, ds.sq, ds.C, ds.outs["wpe"],
+                                          ds.sigma, scale, seed, tid["wpe"], step, beta=0.0,
+                                          d=ds.d_model, **kw)
+
+
+def prefill_embedding_noise(ds: DeviceStep, seed: int, step: int, scale: float = 1.0) -> torch.cuda.Event:
+    """Start the noise fill of the embedding tables on a side stream.  The fill depends on no
+    gradient, so it overlaps the (HBM-bound) norm phase; returns the event to wait for."""
+    if ds.side_stream is None:
+        ds.side_stream = torch.cuda.Stream(device=ds.sq.device)
+    main = torch.cuda.current_stream()
+    tid = tensor_ids(ds)
+    side = ds.side_stream
+    side.wait_stream(main)                       # previous step's readers of the tables are done
+    names = ["wpe"] if ds.positions else []
+    if not (ds.tied and ds.lm is not None):
+        names.append("wte")                      # tied: the head GEMM writes the table first
+    for name in names:
+        dp.dp_fill_noise(ds.outs[name], ds.sigma, ds.C, scale, seed, tid[name], step, stream=side)
+    ev = torch.cuda.Event()
+    ev.record(side)
+    return ev
+
+
+def clip_after_prefill(ds: DeviceStep, seed: int, step: int, filled: torch.cuda.Event,
+                       scale: float = 1.0) -> None:
+    """Clipped sums when the embedding tables already hold their noise (see prefill)."""
+    kw = dict(ws=ds.ws, dev_status=ds.dev_status)
+    tid = tensor_ids(ds)
+    layers = list(ds.linears)
+    names = [f"linear{k}" for k in range(len(ds.linears))]
+    if ds.lm is not None:
+        layers.append(ds.lm)
+        names.append("wte" if ds.tied else "lm_head")
+    if layers:
+        dp.dp_clip_accumulate_noise_grouped(layers, ds.B, ds.T, ds.sq, ds.C, [ds.outs[n] for n in names],
+                                            ds.sigma, scale, seed, [tid[n] for n in names], step,
+                                            beta=0.0, **kw)
+    torch.cuda.current_stream().wait_event(filled)
+    # beta = 1: rows are added onto the noise (untied) or onto head sum + noise (tied)
+    dp.dp_clip_accumulate_embed(ds.ids, ds.G_emb, ds.V, ds.sq, ds.C, ds.outs["wte"], beta=1.0,
+                                d=ds.d_model, **kw)
+    if ds.positions:
+        dp.dp_clip_accumulate_embed(ds.pos_ids, ds.G_emb, WPE_ROWS, ds.sq, ds.C, ds.outs["wpe"],
+                                    beta=1.0, d=ds.d_model, **kw)
+
+
+def dp_step(ds: DeviceStep, seed: int = 0, step: int = 0, noise: bool = True, fused: bool = True,
+            overlap: bool = True, stream=None) -> None:
+    """norms -> clipped sums -> noise.
+
+    fused=True draws the linear-layer noise inside the clipped-sum GEMM; with overlap=True the
+    embedding tables' noise is filled on a side stream while the norms run (scale 1 only).
+    """
+    if noise and fused and overlap and stream is None:
+        filled = prefill_embedding_noise(ds, seed, step)
+        norms_phase(ds)
+        clip_after_prefill(ds, seed, step, filled)
+        return
     norms_phase(ds, stream)
+    if noise and fused:
+        clip_noise_phase(ds, seed, step, stream=stream)
+        return
     clip_phase(ds, stream)
     if noise:
         noise_phase(ds, seed, step, stream=stream)

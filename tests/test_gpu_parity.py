@@ -371,6 +371,88 @@ def test_noise_tail_region_and_scaling():
     assert torch.equal(y3, base)
 
 
+# ------------------------------------------------------------------ fused noise
+@pytest.mark.parametrize("shapes", [
+    [(768, 128 * 100), (768, 768)],      # enough tiles: noise drawn in the GEMM epilogue
+    [(256, 384)],                        # few tiles: K split, noise after the reduce
+    [(50, 128 * 80), (104, 200)],        # widths not a multiple of 4: quads straddle rows
+])
+def test_fused_noise_in_gemm_equals_unfused_calls(shapes):
+    B, T = 4, 128
+    host = [host_linear(B, T, d, p, "bf16", seed=500 + k, ldg=W.round_up(p, 8) if p % 8 else None)
+            for k, (d, p) in enumerate(shapes)]
+    layers = []
+    for (A, G), (d, p) in zip(host, shapes):
+        if d % 8:                                           # pad the activation pitch for TMA
+            a = torch.zeros(B, T, W.round_up(d, 8), dtype=torch.bfloat16, device=dev())
+            a[:, :, :d] = P.to_device(A)
+            layers.append(dp.Linear(a, P.to_device(G), d=d, p=p))
+        else:
+            layers.append(dev_linear(A, G))
+    sq = torch.full((B,), 4.0, device=dev())
+    tids = [7 + k for k in range(len(shapes))]
+    seed, step, sigma, C_, scale = 99, 3, 0.8, 1.0, 0.25
+    fused = [torch.empty(p, d, device=dev()) for d, p in shapes]
+    dp.dp_clip_accumulate_noise_grouped(layers, B, T, sq, C_, fused, sigma, scale, seed, tids, step)
+    plain = [torch.empty(p, d, device=dev()) for d, p in shapes]
+    dp.dp_clip_accumulate_grouped(layers, B, T, sq, C_, plain)
+    sums = [t.clone() for t in plain]
+    for t, tid in zip(plain, tids):
+        dp.dp_add_noise(t, sigma, C_, scale, seed, tid, step)
+    torch.cuda.synchronize()
+    for f, u, s0, tid in zip(fused, plain, sums, tids):
+        assert torch.equal(f, u)                            # same stream, same arithmetic
+        want = NO.add_noise(s0.cpu().numpy().astype(np.float64), sigma, C_, scale, seed, tid, step)
+        assert np.abs(f.cpu().numpy() - want).max() < 1e-6
+
+
+@pytest.mark.parametrize("beta", [0.0, 1.0])
+def test_fused_noise_in_embedding_matches_unfused_calls(beta):
+    B, T, d, V = 3, 128, 768, 5003
+    ids = W.zipf_ids(B, T, V, 1.1, 41)
+    G = W._normal((B, T, d), 1e-2, "bf16", 42)
+    sq = torch.full((B,), 9.0, device=dev())
+    base = torch.randn(V, d, device=dev())
+    seed, tid, step, sigma, C_, scale = 5, 2, 1, 0.8, 1.0, 0.5
+    dids, dG = torch.from_numpy(ids).to(dev()), P.to_device(G)
+    fused = base.clone()
+    dp.dp_clip_accumulate_embed_noise(dids, dG, V, sq, C_, fused, sigma, scale, seed, tid, step, beta=beta)
+    plain = base.clone()
+    dp.dp_clip_accumulate_embed(dids, dG, V, sq, C_, plain, beta=beta)
+    if beta == 0.0:
+        dp.dp_add_noise(plain, sigma, C_, scale, seed, tid, step)
+    else:
+        # tied case: the table already holds noise + head; the call adds scale * row sums
+        plain = base + scale * (plain - base)
+    torch.cuda.synchronize()
+    assert torch.allclose(fused, plain, rtol=1e-5, atol=2e-6)
+
+
+def test_fused_and_unfused_steps_agree():
+    w = W.named_workload("cfg4", B=3, n_blocks=1, V=4099)
+    a, b = P.upload(w), P.upload(w)
+    c = P.upload(w)
+    P.dp_step(a, seed=11, step=2, fused=True)                      # noise prefill on a side stream
+    P.dp_step(b, seed=11, step=2, fused=False)
+    P.dp_step(c, seed=11, step=2, fused=True, overlap=False)
+    torch.cuda.synchronize()
+    check_status(a.dev_status)
+    for k in a.outs:
+        assert torch.allclose(a.outs[k], b.outs[k], rtol=1e-5, atol=2e-6), k
+        assert torch.allclose(c.outs[k], b.outs[k], rtol=1e-5, atol=2e-6), k
+
+
+def test_overlapped_step_untied_with_positions_matches_unfused():
+    w = W.named_workload("cfg3", B=2, T=256, n_blocks=1, V=3001)
+    a, b = P.upload(w), P.upload(w)
+    for step in range(2):                                          # twice: side-stream reuse
+        P.dp_step(a, seed=5, step=step, fused=True)
+        P.dp_step(b, seed=5, step=step, fused=False)
+    torch.cuda.synchronize()
+    for k in a.outs:
+        assert torch.allclose(a.outs[k], b.outs[k], rtol=1e-5, atol=2e-6), k
+
+
 # ---------------------------------------------------------------------------- error paths
 def test_argument_errors_are_reported_before_any_launch():
     B, T, d, p = 2, 16, 64, 64
