@@ -51,7 +51,8 @@ typedef enum {
   DP_ERR_UNSUPPORTED = 2,   /* a size beyond what the kernels were built for */
   DP_ERR_ALIGNMENT = 3,     /* pointer / leading dimension breaks the TMA rules above */
   DP_ERR_WORKSPACE = 4,     /* ws is NULL or smaller than *_ws_bytes reports */
-  DP_ERR_CUDA = 5           /* CUDA runtime / driver error; dp_last_cuda_error() has the code */
+  DP_ERR_CUDA = 5,          /* CUDA runtime / driver error; dp_last_cuda_error() has the code */
+  DP_ERR_SCRATCH_LIMIT = 6  /* dp_embed_norms_static: problem larger than the built-in scratch */
 } dp_status;
 
 typedef enum { DP_F32 = 0, DP_BF16 = 1 } dp_dtype;
@@ -94,6 +95,26 @@ dp_status dp_embed_norms(const int32_t* ids, const void* G, int64_t ldg, dp_dtyp
                          int32_t* first_occ, void* ws, size_t ws_bytes,
                          int32_t* dev_status, void* stream);
 size_t dp_embed_norms_ws_bytes(int32_t B, int32_t T, int32_t d);
+
+/* ---- the same embedding norm without any caller workspace ----
+ * (No counterpart in the paper: this entry point exists for the way the library is hosted.)
+ * For callers that cannot allocate or pass scratch memory -- code running while the host's
+ * allocator is frozen for a step, plug-ins that receive only their input and output tensors,
+ * devices whose memory is already fully committed.  The partial sums of the norm kernel live in
+ * a fixed 64 KiB array inside the library image (every device that loads the library holds it
+ * until the process exits), so B * ceil(d / 256) must not exceed DP_STATIC_SCRATCH_FLOATS,
+ * else DP_ERR_SCRATCH_LIMIT is returned and nothing is enqueued.  Inputs, outputs and results
+ * are those of dp_embed_norms.  No cudaMalloc / cudaFree or other allocating call is made.
+ * The first call on each device looks up the array's device address (a host-side runtime
+ * query); make that first call before starting any stream capture.  All calls on a device
+ * share the one array: it keeps the previous call's contents (each call overwrites every
+ * element it later reads, so nothing needs clearing), and two calls whose kernels may overlap
+ * on the GPU -- different streams, no ordering between them -- race on it and must not be
+ * issued. */
+#define DP_STATIC_SCRATCH_FLOATS 16384
+dp_status dp_embed_norms_static(const int32_t* ids, const void* G, int64_t ldg, dp_dtype dt,
+                                int32_t B, int32_t T, int32_t d, int32_t V, float* sq,
+                                int32_t* first_occ, int32_t* dev_status, void* stream);
 
 /* ---- cross term of a weight-tied embedding / LM head (Eq. 11, Eq. 13) ----
  * Adds 2*<g_in_i, g_out_i> to sq[i], with g_in_i the (V,d) embedding gradient of example i

@@ -35,6 +35,7 @@ class _LinearDesc(C.Structure):
 
 
 EXPORTS = ["dp_ghost_norms", "dp_ghost_norms_ws_bytes", "dp_embed_norms", "dp_embed_norms_ws_bytes",
+           "dp_embed_norms_static",
            "dp_tied_cross_term", "dp_tied_cross_term_ws_bytes", "dp_clip_factors",
            "dp_clip_accumulate", "dp_clip_accumulate_ws_bytes", "dp_clip_accumulate_grouped",
            "dp_clip_accumulate_grouped_ws_bytes", "dp_clip_accumulate_noise_grouped",
@@ -60,6 +61,7 @@ def load():
     L.dp_ghost_norms_ws_bytes.argtypes = [C.POINTER(_LinearDesc), i32, i32, i32, i32]
     L.dp_ghost_norms_ws_bytes.restype = sz
     L.dp_embed_norms.argtypes = [vp, vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, sz, vp, vp]
+    L.dp_embed_norms_static.argtypes = [vp, vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, vp]
     L.dp_embed_norms_ws_bytes.argtypes = [i32, i32, i32]
     L.dp_embed_norms_ws_bytes.restype = sz
     L.dp_tied_cross_term.argtypes = [vp, vp, i64, vp, i64, vp, i64, i32, i32, i32, i32, i32, vp, vp,
@@ -208,6 +210,19 @@ def dp_embed_norms(ids: torch.Tensor, G: torch.Tensor, V: int, sq: torch.Tensor,
                           _ptr(first_occ), _ptr(ws), ws.numel() * ws.element_size(),
                           _ptr(dev_status), _stream(stream))
     _check(st, "dp_embed_norms")
+
+
+def dp_embed_norms_static(ids: torch.Tensor, G: torch.Tensor, V: int, sq: torch.Tensor, d=None,
+                          first_occ=None, dev_status=None, stream=None):
+    """dp_embed_norms for callers that cannot allocate: no workspace is passed or created here;
+    the kernel's scratch is a fixed array inside the library (B * ceil(d/256) <= 16384, else
+    status 6).  Calls that may overlap on the GPU must not be issued (they share that array)."""
+    L = load()
+    B, T = ids.shape
+    d = d if d is not None else G.shape[-1]
+    st = L.dp_embed_norms_static(_ptr(ids), _ptr(G), _rows_ld(G), _dt(G), B, T, d, V, _ptr(sq),
+                                 _ptr(first_occ), _ptr(dev_status), _stream(stream))
+    _check(st, "dp_embed_norms_static")
 
 
 def dp_tied_cross_term(ids, G_emb, A_lm, G_lm, V: int, sq=None, cross=None, d=None, ws=None,

@@ -105,6 +105,9 @@ const char* dp_status_string(dp_status s) {
     case DP_ERR_ALIGNMENT: return "pointer or leading dimension not aligned for TMA";
     case DP_ERR_WORKSPACE: return "workspace missing or too small";
     case DP_ERR_CUDA: return "CUDA error (see dp_last_cuda_error)";
+    case DP_ERR_SCRATCH_LIMIT:
+      return "problem needs more scratch than the library's built-in array holds "
+             "(B * ceil(d/256) > DP_STATIC_SCRATCH_FLOATS); use dp_embed_norms with a workspace";
   }
   return "unknown status";
 }
