@@ -199,11 +199,16 @@ def run_ours(args):
 
     def step(k, ev=None):
         if ev: ev[0].record(stream)
-        if fused:
+        if fused and args.prefill:
+            filled = P.prefill_all_noise(ds, args.seed, k)           # side stream, overlaps the norms
+        elif fused:
             filled = P.prefill_embedding_noise(ds, args.seed, k)     # side stream, overlaps the norms
         P.norms_phase(ds)
         if ev: ev[1].record(stream)
-        if fused:
+        if fused and args.prefill:
+            P.clip_onto_noise(ds, filled)
+            if ev: ev[2].record(stream)
+        elif fused:
             P.clip_after_prefill(ds, args.seed, k, filled)
             if ev: ev[2].record(stream)
         else:
@@ -406,6 +411,7 @@ def main():
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--prefill", action="store_true", help="noise of every tensor filled beside the norms")
     ap.add_argument("--unfused", action="store_true",
                     help="separate noise pass (what the multi-GPU path uses) instead of fused noise")
     args = ap.parse_args()

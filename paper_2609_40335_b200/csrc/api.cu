@@ -115,6 +115,7 @@ const char* dp_status_string(dp_status s) {
 int32_t dp_last_cuda_error(void) { return g_last_cuda_error; }
 const char* dp_version(void) { return "dp_ghost 0.1.0 (sm_100a)"; }
 int64_t dp_kernel_launches(void) { return g_kernel_launches; }
+int32_t dp_debug_max_active_pairs(void) { return gta_max_active_pairs(); }
 int32_t dp_debug_force_fma(int32_t on) {
   const int prev = g_force_fma;
   g_force_fma = on ? 1 : 0;

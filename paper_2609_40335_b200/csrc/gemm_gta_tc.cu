@@ -9,14 +9,20 @@
 // memory holds MN-major tiles: every TMA box is 64 token rows x 64 columns (128-byte rows,
 // 128-byte swizzle).  A K step never straddles two examples (the tensor map is 3-D:
 // column, token, example; the token tail of an example is zero-filled), so one clip factor
-// applies to a whole stage: four "scaler" warps multiply the G tile by R_i in shared memory
+// applies to a whole stage: a "scaler" warp multiplies the G tile by R_i in shared memory
 // (packed bf16 FMAs with R_i split into two bf16 parts) between the TMA-full and MMA-ready
-// barriers.
+// barriers; four such warps work on four consecutive stages at once.
 //
-// Roles per CTA (576 threads): warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 scalers,
-// warps 6-17 epilogue (three per TMEM lane quarter, sharing the 256 columns 3+3+2 chunks; they
-// also draw the fused Gaussian noise); two TMEM accumulators overlap the epilogue with the
-// next tile.
+// Roles per CTA (704 threads): warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 scalers,
+// warps 6-21 epilogue (four per TMEM lane quarter, two 32-column chunks each; they also draw
+// the fused Gaussian noise, which is latency-bound per warp -- hence so many); two TMEM
+// accumulators overlap the epilogue with the next tile.
+//
+// Clipped sums run on CTA PAIRS (cta_group::2, cluster of 2): a 256 x 256 output tile per pair,
+// each CTA loading its own 128 G rows and half of the A tile's columns, rank 0 issuing the MMAs
+// for both, stage-free and accumulator-ready signals multicast to both CTAs by tcgen05.commit,
+// scaler and epilogue warps of rank 1 arriving on rank 0's barriers.  The DIRECT-norm variant
+// stays on single CTAs.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -35,22 +41,29 @@ namespace {
 
 constexpr int kBM = 128, kBN = 256, kBK = 64;
 constexpr int kBoxBytes = 64 * 128;                 // 64 token rows x 128 bytes
-constexpr int kGBytes = (kBM / 64) * kBoxBytes;     // 16 KiB
-constexpr int kABytes = (kBN / 64) * kBoxBytes;     // 32 KiB
-constexpr int kStageBytes = kGBytes + kABytes;      // 48 KiB
-#ifndef DPG_GTA_STAGES
-#define DPG_GTA_STAGES 4
-#endif
-constexpr int kStages = DPG_GTA_STAGES;
+constexpr int kGBytes = (kBM / 64) * kBoxBytes;     // 16 KiB: this CTA's 128 rows of the G tile
+
+// Tile geometry.  Single CTA: 128 x 256 output tile, the CTA loads all 256 columns of the A
+// tile (48 KiB per stage, 4 stages).  CTA pair (cta_group::2): 256 x 256 output tile per pair;
+// each CTA loads its own 128 G rows and HALF of the A tile's columns (32 KiB per stage, 6
+// stages), the pair's MMA reads both halves -- a third less operand traffic per flop.
+template <bool kPair>
+struct Geo {
+  static constexpr int kAColsPerCta = kPair ? kBN / 2 : kBN;
+  static constexpr int kABytes = (kAColsPerCta / 64) * kBoxBytes;
+  static constexpr int kStageBytes = kGBytes + kABytes;
+  static constexpr int kStages = kPair ? 6 : 4;
+  static constexpr int kTileM = kPair ? 2 * kBM : kBM;       // output rows per work item
+  static constexpr size_t kSmemBytes = size_t(kStages) * kStageBytes + 1024 + 256;
+};
 constexpr int kScalerWarps = 4;
 constexpr int kEpiWarp0 = 2 + kScalerWarps;          // first epilogue warp
 #ifndef DPG_GTA_EPI_WARPS
-#define DPG_GTA_EPI_WARPS 12
+#define DPG_GTA_EPI_WARPS 16
 #endif
 constexpr int kEpiWarps = DPG_GTA_EPI_WARPS;         // kEpiWarps/4 per TMEM lane quarter (column groups)
 constexpr int kThreads = (kEpiWarp0 + kEpiWarps) * 32;
 constexpr int kTmemCols = 512;                      // 2 accumulators x 256 columns
-constexpr size_t kSmemBytes = size_t(kStages) * kStageBytes + 1024 + 256;
 
 struct __align__(64) GtaParams {
   CUtensorMap tmG[kGtaMaxLayers];
@@ -93,9 +106,17 @@ __device__ __forceinline__ Item decode_item(const GtaParams& P, int item) {
   return it;
 }
 
-template <bool kScale, bool kSqsum>
+template <bool kScale, bool kSqsum, bool kPair>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_gta_kernel(const __grid_constant__ GtaParams P) {
+  constexpr int kStages = Geo<kPair>::kStages;
+  constexpr int kStageBytes = Geo<kPair>::kStageBytes;
+  constexpr int kTileM = Geo<kPair>::kTileM;
+  constexpr int kPeers = kPair ? 2 : 1;
+  // pair: rank 0 issues the MMAs; both CTAs walk the same list of work items
+  const uint32_t rank = kPair ? ptx::cluster_ctarank() : 0u;
+  const int first_item = kPair ? int(blockIdx.x >> 1) : int(blockIdx.x);
+  const int item_stride = kPair ? int(gridDim.x >> 1) : int(gridDim.x);
   extern __shared__ uint8_t smem_raw[];
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                               ~uintptr_t(1023));
@@ -115,19 +136,23 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       ptx::mbar_init(&full[s], 1);
-      ptx::mbar_init(&ready[s], kScalerWarps);
+      ptx::mbar_init(&ready[s], kPeers);                    // one scaler warp per CTA and stage
       ptx::mbar_init(&empty[s], 1);
     }
-    for (int b = 0; b < 2; ++b) { ptx::mbar_init(&acc_full[b], 1); ptx::mbar_init(&acc_empty[b], kEpiWarps); }
+    for (int b = 0; b < 2; ++b) {
+      ptx::mbar_init(&acc_full[b], 1);
+      ptx::mbar_init(&acc_empty[b], kEpiWarps * kPeers);    // epilogue warps of both CTAs
+    }
     *abort_flag = 0;
     ptx::fence_mbar_init();
   }
   if (warp == 1) {
-    ptx::tmem_alloc(tmem_slot, kTmemCols);
-    ptx::tmem_relinquish();
+    if (kPair) { ptx::tmem_alloc_pair(tmem_slot, kTmemCols); ptx::tmem_relinquish_pair(); }
+    else { ptx::tmem_alloc(tmem_slot, kTmemCols); ptx::tmem_relinquish(); }
   }
   ptx::tc_fence_before();
   __syncthreads();
+  if (kPair) ptx::cluster_sync_all();     // the partner's barriers exist before anyone arrives on them
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -136,7 +161,7 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
     if (lane == 0) {
       uint32_t stage = 0, phase = 0;
       bool ok = true;
-      for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x) {
+      for (int item = first_item; item < P.total_items && ok; item += item_stride) {
         const Item it = decode_item<kSqsum>(P, item);
         const CUtensorMap* tg = &P.tmG[it.layer];
         const CUtensorMap* ta = &P.tmA[it.layer];
@@ -145,13 +170,14 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
           const int ex = ks / P.tsteps, t0 = (ks - ex * P.tsteps) * kBK;
           uint8_t* dst = tiles + size_t(stage) * kStageBytes;
           ptx::mbar_arrive_expect_tx(&full[stage], kStageBytes);
+          const int m0 = it.tm * kTileM + int(rank) * kBM;                   // this CTA's G rows
+          const int n0 = it.tn * kBN + int(rank) * Geo<kPair>::kAColsPerCta;   // and A columns
 #pragma unroll
           for (int j = 0; j < kBM / 64; ++j)
-            ptx::tma_load_3d(dst + j * kBoxBytes, tg, &full[stage], it.tm * kBM + j * 64, t0, ex);
+            ptx::tma_load_3d(dst + j * kBoxBytes, tg, &full[stage], m0 + j * 64, t0, ex);
 #pragma unroll
-          for (int j = 0; j < kBN / 64; ++j)
-            ptx::tma_load_3d(dst + kGBytes + j * kBoxBytes, ta, &full[stage],
-                             it.tn * kBN + j * 64, t0, ex);
+          for (int j = 0; j < Geo<kPair>::kAColsPerCta / 64; ++j)
+            ptx::tma_load_3d(dst + kGBytes + j * kBoxBytes, ta, &full[stage], n0 + j * 64, t0, ex);
           if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
       }
@@ -162,36 +188,45 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
     }
   } else if (warp == 1) {
     // --------------------------------------------------------------- MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = ptx::idesc_bf16_f32(kBM, kBN, 1, 1);
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = ptx::idesc_bf16_f32(kTileM, kBN, 1, 1);
       // MN-major, 128-byte swizzle: 64-column chunks are one box (8 KiB) apart, groups of
       // 8 token rows are 1 KiB apart
       constexpr uint64_t dbase = ptx::smem_desc_base(kBoxBytes, 1024, ptx::SWIZZLE_128B);
       uint32_t stage = 0, phase = 0, n_item = 0;
       bool ok = true;
-      for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x, ++n_item) {
+      for (int item = first_item; item < P.total_items && ok; item += item_stride, ++n_item) {
         const Item it = decode_item<kSqsum>(P, item);
         const uint32_t buf = n_item & 1, acc_phase = (n_item >> 1) & 1;
-        if (!ptx::mbar_wait(&acc_empty[buf], acc_phase ^ 1, abort_flag)) { ok = false; break; }
+        if (!(kPair ? ptx::mbar_wait_cluster(&acc_empty[buf], acc_phase ^ 1, abort_flag)
+                    : ptx::mbar_wait(&acc_empty[buf], acc_phase ^ 1, abort_flag))) { ok = false; break; }
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * kBN;
         for (int ks = it.k0; ks < it.k1; ++ks) {
           uint64_t* go = kScale ? &ready[stage] : &full[stage];
-          if (!ptx::mbar_wait(go, phase, abort_flag)) { ok = false; break; }
+          if (!(kPair ? ptx::mbar_wait_cluster(go, phase, abort_flag)
+                      : ptx::mbar_wait(go, phase, abort_flag))) { ok = false; break; }
           ptx::tc_fence_after();
           const uint32_t sg = ptx::smem_u32(tiles + size_t(stage) * kStageBytes);
           const uint32_t sa = sg + kGBytes;
 #pragma unroll
           for (int kk = 0; kk < kBK / 16; ++kk) {
             // 16 token rows further = two 1 KiB row groups
-            ptx::mma_bf16_ss(d_tmem, ptx::smem_desc(dbase, sg + kk * 2048),
-                             ptx::smem_desc(dbase, sa + kk * 2048), idesc,
-                             (ks > it.k0 || kk > 0) ? 1u : 0u);
+            const uint64_t da = ptx::smem_desc(dbase, sg + kk * 2048);
+            const uint64_t db = ptx::smem_desc(dbase, sa + kk * 2048);
+            const uint32_t accum = (ks > it.k0 || kk > 0) ? 1u : 0u;
+            if (kPair) ptx::mma_bf16_ss_pair(d_tmem, da, db, idesc, accum);
+            else ptx::mma_bf16_ss(d_tmem, da, db, idesc, accum);
           }
-          ptx::mma_commit(&empty[stage]);
+          // stage reusable in both CTAs once these MMAs retire
+          if (kPair) ptx::mma_commit_pair(&empty[stage], 3);
+          else ptx::mma_commit(&empty[stage]);
           if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
-        if (ok) ptx::mma_commit(&acc_full[buf]);
+        if (ok) {
+          if (kPair) ptx::mma_commit_pair(&acc_full[buf], 3);
+          else ptx::mma_commit(&acc_full[buf]);
+        }
       }
       if (!ok) {
         *abort_flag = 1;
@@ -201,13 +236,17 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
   } else if (warp < kEpiWarp0) {
     // ------------------------------------------------------------------ scalers
     if (kScale) {
-      constexpr int kScalerThreads = kScalerWarps * 32;
-      const int st = threadIdx.x - 64;                 // 0 .. kScalerThreads-1
-      uint32_t stage = 0, phase = 0;
+      // Each scaler warp owns every kScalerWarps-th K step, so kScalerWarps stages are scaled
+      // concurrently: the per-stage latency (shared-memory round trip, proxy fence, barrier
+      // hand-off) is overlapped instead of serialised.
+      const int sw = warp - 2;
+      uint32_t cnt = 0;
       bool ok = true;
-      for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x) {
+      for (int item = first_item; item < P.total_items && ok; item += item_stride) {
         const Item it = decode_item<kSqsum>(P, item);
-        for (int ks = it.k0; ks < it.k1; ++ks) {
+        for (int ks = it.k0; ks < it.k1; ++ks, ++cnt) {
+          if (int(cnt % kScalerWarps) != sw) continue;
+          const uint32_t stage = cnt % kStages, phase = (cnt / kStages) & 1u;
           if (!ptx::mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
           const int ex = ks / P.tsteps;
           const float r = __ldg(P.clip + ex);
@@ -219,21 +258,27 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
             const __nv_bfloat16 rl = __float2bfloat16_rn(r - __bfloat162float(rh));
             const __nv_bfloat162 rh2 = __halves2bfloat162(rh, rh), rl2 = __halves2bfloat162(rl, rl);
             uint4* g = reinterpret_cast<uint4*>(tiles + size_t(stage) * kStageBytes);
-            uint4 v[kGBytes / 16 / kScalerThreads];
+            constexpr int kChunks = kGBytes / 16 / 32;          // 16-byte chunks per lane
+#pragma unroll 1
+            for (int c0 = 0; c0 < kChunks; c0 += 8) {
+              uint4 v[8];
 #pragma unroll
-            for (int c = 0; c < kGBytes / 16 / kScalerThreads; ++c) v[c] = g[c * kScalerThreads + st];
+              for (int c = 0; c < 8; ++c) v[c] = g[(c0 + c) * 32 + lane];
 #pragma unroll
-            for (int c = 0; c < kGBytes / 16 / kScalerThreads; ++c) {
-              __nv_bfloat162* w = reinterpret_cast<__nv_bfloat162*>(&v[c]);
+              for (int c = 0; c < 8; ++c) {
+                __nv_bfloat162* w = reinterpret_cast<__nv_bfloat162*>(&v[c]);
 #pragma unroll
-              for (int e = 0; e < 4; ++e) w[e] = __hfma2(w[e], rh2, __hmul2(w[e], rl2));
-              g[c * kScalerThreads + st] = v[c];
+                for (int e = 0; e < 4; ++e) w[e] = __hfma2(w[e], rh2, __hmul2(w[e], rl2));
+                g[(c0 + c) * 32 + lane] = v[c];
+              }
             }
             ptx::fence_proxy_async_smem();
           }
           __syncwarp();
-          if (lane == 0) ptx::mbar_arrive(&ready[stage]);
-          if (++stage == kStages) { stage = 0; phase ^= 1; }
+          if (lane == 0) {
+            if (kPair) ptx::mbar_arrive_cluster(&ready[stage], 0);   // the MMA issuer lives in rank 0
+            else ptx::mbar_arrive(&ready[stage]);
+          }
         }
       }
       if (!ok && lane == 0) {
@@ -250,14 +295,14 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
     const int c_lo = ((ew >> 2) * (kBN / 32)) / kGroups, c_hi = (((ew >> 2) + 1) * (kBN / 32)) / kGroups;
     uint32_t n_item = 0;
     bool ok = true;
-    for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x, ++n_item) {
+    for (int item = first_item; item < P.total_items && ok; item += item_stride, ++n_item) {
       const Item it = decode_item<kSqsum>(P, item);
       const GtaLayer& L = P.layer[it.layer];
       const uint32_t buf = n_item & 1, acc_phase = (n_item >> 1) & 1;
       if (!ptx::mbar_wait(&acc_full[buf], acc_phase, abort_flag)) { ok = false; break; }
       ptx::tc_fence_after();
       const uint32_t t0 = tmem_base + (uint32_t(q * 32) << 16) + buf * kBN;
-      const int row = it.tm * kBM + q * 32 + lane;
+      const int row = it.tm * kTileM + int(rank) * kBM + q * 32 + lane;
       if (kSqsum) {
         float acc = 0.f;
 #pragma unroll 1
@@ -270,7 +315,10 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
         }
         ptx::tc_fence_before();
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&acc_empty[buf]);
+        if (lane == 0) {
+          if (kPair) ptx::mbar_arrive_cluster(&acc_empty[buf], 0);
+          else ptx::mbar_arrive(&acc_empty[buf]);
+        }
         acc = warp_sum(acc);
         if (lane == 0) epi_red[buf * kEpiWarps + ew] = acc;
         asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
@@ -343,7 +391,10 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
         }
         ptx::tc_fence_before();
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&acc_empty[buf]);
+        if (lane == 0) {
+          if (kPair) ptx::mbar_arrive_cluster(&acc_empty[buf], 0);
+          else ptx::mbar_arrive(&acc_empty[buf]);
+        }
       }
     }
     if (!ok && lane == 0) {
@@ -354,9 +405,13 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
 
   ptx::tc_fence_before();
   __syncthreads();
+  // pair: neither CTA may leave while the partner can still read its shared memory or arrive on
+  // its barriers (every wait above is bounded, so both always get here)
+  if (kPair) ptx::cluster_sync_all();
   if (warp == 1) {
     ptx::tc_fence_after();
-    ptx::tmem_dealloc(tmem_base, kTmemCols);
+    if (kPair) ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
+    else ptx::tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 
@@ -380,14 +435,46 @@ constexpr bool kClipScale = false;   // experiment only: clip factors are ignore
 constexpr bool kClipScale = true;
 #endif
 
-template <bool kScale, bool kSqsum>
+#ifdef DPG_GTA_SINGLE_CTA
+constexpr bool kUsePair = false;     // experiment only: clipped sums on the single-CTA tiles
+#else
+constexpr bool kUsePair = true;
+#endif
+
+template <bool kScale, bool kSqsum, bool kPair>
 dp_status set_attr_once() {
   static bool done = false;
   if (!done) {
-    DP_CUDA_OK(cudaFuncSetAttribute(gemm_gta_kernel<kScale, kSqsum>,
-                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
+    DP_CUDA_OK(cudaFuncSetAttribute(gemm_gta_kernel<kScale, kSqsum, kPair>,
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)Geo<kPair>::kSmemBytes));
     done = true;
   }
+  return DP_OK;
+}
+
+// Launch on `units` persistent CTAs (single) or CTA pairs (cluster of 2).
+template <bool kScale, bool kSqsum, bool kPair>
+dp_status launch_gta(const GtaParams& P, int units, cudaStream_t st) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(kPair ? 2 * units : units, 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = Geo<kPair>::kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = kPair ? 2 : 1;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+#ifdef DPG_GTA_POLICY_LB
+  attr[1].id = cudaLaunchAttributeClusterSchedulingPolicyPreference;
+  attr[1].val.clusterSchedulingPolicyPreference = cudaClusterSchedulingPolicyLoadBalancing;
+  cfg.numAttrs = 2;
+#endif
+  DP_CUDA_OK(cudaLaunchKernelEx(&cfg, gemm_gta_kernel<kScale, kSqsum, kPair>, P));
+  ++g_kernel_launches;
   return DP_OK;
 }
 
@@ -398,10 +485,11 @@ dp_status set_attr_once() {
 int gta_choose_nsplit(const dp_linear_desc* layers, int n_layers, int B, int T, int sms) {
   long long tiles = 0;
   for (int l = 0; l < n_layers; ++l)
-    tiles += (long long)ceil_div(layers[l].p, kBM) * ceil_div(layers[l].d, kBN);
+    tiles += (long long)ceil_div(layers[l].p, Geo<kUsePair>::kTileM) * ceil_div(layers[l].d, kBN);
   const int ksteps = B * ceil_div(T, kBK);
-  if (tiles >= 2LL * sms) return 1;
-  long long ns = std::max<long long>(1, (2LL * sms) / std::max<long long>(tiles, 1));
+  const int units = kUsePair ? sms / 2 : sms;          // persistent CTAs or CTA pairs
+  if (tiles >= 2LL * units) return 1;
+  long long ns = std::max<long long>(1, (2LL * units) / std::max<long long>(tiles, 1));
   ns = std::min<long long>(ns, std::max(1, ksteps / 4));
   return (int)std::max<long long>(1, ns);
 }
@@ -419,7 +507,7 @@ dp_status launch_clip_accumulate_tc(const dp_linear_desc* layers, int n_layers, 
                                     const float* clip, float* const* outs, const int64_t* ldos,
                                     float beta, const GtaNoise* noise, float* partial_ws,
                                     int* dev_status, cudaStream_t st) {
-  dp_status s = set_attr_once<kClipScale, false>();
+  dp_status s = set_attr_once<kClipScale, false, kUsePair>();
   if (s != DP_OK) return s;
   const int sms = sm_count();
   const int tsteps = ceil_div(T, kBK);
@@ -442,7 +530,7 @@ dp_status launch_clip_accumulate_tc(const dp_linear_desc* layers, int n_layers, 
       GtaLayer& L = P.layer[g - g0];
       L.out = outs[g]; L.ldo = ldos[g]; L.beta = beta;
       L.M = D.p; L.N = D.d;
-      L.tiles_m = ceil_div(D.p, kBM); L.tiles_n = ceil_div(D.d, kBN);
+      L.tiles_m = ceil_div(D.p, Geo<kUsePair>::kTileM); L.tiles_n = ceil_div(D.d, kBN);
       L.nsplit = nsplit; L.ksteps_per_split = kps;
       L.partial = nullptr;
       if (nsplit > 1) {
@@ -465,9 +553,9 @@ dp_status launch_clip_accumulate_tc(const dp_linear_desc* layers, int n_layers, 
     P.total_items = items;
     P.clip = clip;
     P.dev_status = dev_status;
-    const int grid = std::min(items, sms);
-    gemm_gta_kernel<kClipScale, false><<<grid, kThreads, kSmemBytes, st>>>(P);
-    DP_LAUNCH_OK();
+    const int units = std::min(items, kUsePair ? sms / 2 : sms);
+    s = launch_gta<kClipScale, false, kUsePair>(P, units, st);
+    if (s != DP_OK) return s;
     for (int g = g0; g < g1; ++g) {
       const GtaLayer& L = P.layer[g - g0];
       if (nsplit > 1) {
@@ -487,9 +575,26 @@ dp_status launch_clip_accumulate_tc(const dp_linear_desc* layers, int n_layers, 
   return DP_OK;
 }
 
+// Diagnostic: how many CTA pairs of the clipped-sum kernel the device can hold at once.
+int gta_max_active_pairs() {
+  if (set_attr_once<kClipScale, false, true>() != DP_OK) return -1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * 74, 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = Geo<true>::kSmemBytes;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  int n = -1;
+  if (cudaOccupancyMaxActiveClusters(&n, gemm_gta_kernel<kClipScale, false, true>, &cfg) != cudaSuccess)
+    return -2;
+  return n;
+}
+
 dp_status launch_direct_norm_tc(const dp_linear_desc* layers, const GhostPlan& plan, int B, int T,
                                 float* partials, int* dev_status, cudaStream_t st) {
-  dp_status s = set_attr_once<false, true>();
+  dp_status s = set_attr_once<false, true, false>();
   if (s != DP_OK) return s;
   const int sms = sm_count();
   for (size_t g0 = 0; g0 < plan.direct_layers.size(); g0 += kGtaMaxLayers) {
@@ -517,9 +622,8 @@ dp_status launch_direct_norm_tc(const dp_linear_desc* layers, const GhostPlan& p
     P.total_items = items;
     P.sq_partials = partials; P.n_per = plan.n_per;
     P.dev_status = dev_status;
-    const int grid = std::min(items, sms);
-    gemm_gta_kernel<false, true><<<grid, kThreads, kSmemBytes, st>>>(P);
-    DP_LAUNCH_OK();
+    s = launch_gta<false, true, false>(P, std::min(items, sms), st);
+    if (s != DP_OK) return s;
   }
   return DP_OK;
 }

@@ -203,6 +203,39 @@ def prefill_embedding_noise(ds: DeviceStep, seed: int, step: int, scale: float =
     return ev
 
 
+def prefill_all_noise(ds: DeviceStep, seed: int, step: int) -> torch.cuda.Event:
+    """Fill EVERY output tensor with its noise on the side stream (scale 1).  The fills are
+    ALU-bound and depend on no gradient, the norm phase is HBM-bound: they share the SMs."""
+    if ds.side_stream is None:
+        ds.side_stream = torch.cuda.Stream(device=ds.sq.device)
+    side = ds.side_stream
+    side.wait_stream(torch.cuda.current_stream())
+    for tid, name in enumerate(sorted(ds.outs)):
+        dp.dp_fill_noise(ds.outs[name], ds.sigma, ds.C, 1.0, seed, tid, step, stream=side)
+    ev = torch.cuda.Event()
+    ev.record(side)
+    return ev
+
+
+def clip_onto_noise(ds: DeviceStep, filled: torch.cuda.Event) -> None:
+    """Clipped sums accumulated (beta = 1) onto tensors that already hold their noise."""
+    kw = dict(ws=ds.ws, dev_status=ds.dev_status)
+    layers = list(ds.linears)
+    names = [f"linear{k}" for k in range(len(ds.linears))]
+    if ds.lm is not None:
+        layers.append(ds.lm)
+        names.append("wte" if ds.tied else "lm_head")
+    torch.cuda.current_stream().wait_event(filled)
+    if layers:
+        dp.dp_clip_accumulate_grouped(layers, ds.B, ds.T, ds.sq, ds.C, [ds.outs[n] for n in names],
+                                      beta=1.0, **kw)
+    dp.dp_clip_accumulate_embed(ds.ids, ds.G_emb, ds.V, ds.sq, ds.C, ds.outs["wte"], beta=1.0,
+                                d=ds.d_model, **kw)
+    if ds.positions:
+        dp.dp_clip_accumulate_embed(ds.pos_ids, ds.G_emb, WPE_ROWS, ds.sq, ds.C, ds.outs["wpe"],
+                                    beta=1.0, d=ds.d_model, **kw)
+
+
 def clip_after_prefill(ds: DeviceStep, seed: int, step: int, filled: torch.cuda.Event,
                        scale: float = 1.0) -> None:
     """Clipped sums when the embedding tables already hold their noise (see prefill)."""

@@ -49,6 +49,26 @@ def case_ghost(reps):
         dp.dp_ghost_norms(layers, B, T, sq)
 
 
+def case_ghost_long(reps):
+    """Tensor-bound regime of the ghost norm: T = 512 (10 tile pairs per example and layer)."""
+    B, T = 64, 512
+    layers = [dp.Linear(_randn_bf16(B, T, 1024), _randn_bf16(B, T, 4096, std=1e-2)) for _ in range(2)]
+    sq = torch.zeros(B, device="cuda")
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    dp.dp_ghost_norms(layers, B, T, sq)
+    e0.record()
+    for _ in range(reps):
+        dp.dp_ghost_norms(layers, B, T, sq)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    tiles = 10 * B * len(layers)                       # 128 x 128 tile pairs
+    flops = tiles * 2 * 128 * 128 * (1024 + 4096)
+    nbytes = B * len(layers) * 2 * T * (1024 + 4096)
+    print(f"ghost T=512: {ms:.4f} ms per call, {flops / ms / 1e9:.1f} TFLOP/s issued, "
+          f"{nbytes / ms / 1e6:.0f} GB/s algorithmic")
+
+
 def case_noise(reps):
     x = torch.zeros(50257 * 768, device="cuda")
     for k in range(reps):
@@ -81,7 +101,7 @@ def main():
     which = sys.argv[1] if len(sys.argv) > 1 else "gemm"
     reps = int(sys.argv[2]) if len(sys.argv) > 2 else 3
     torch.manual_seed(0)
-    {"gemm": case_gemm, "gemm1": case_gemm_unclipped, "ghost": case_ghost, "noise": case_noise, "embed": case_embed,
+    {"gemm": case_gemm, "gemm1": case_gemm_unclipped, "ghost512": case_ghost_long, "ghost": case_ghost, "noise": case_noise, "embed": case_embed,
      "cross": case_cross}[which](reps)
     torch.cuda.synchronize()
     print("done", which, reps)
