@@ -24,6 +24,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one grouped GEMM launch, from the ncu capture
+# summarised in profiles/gemm_gta_kernel_pair.md (scaled to the full launch as described there)
+GEMM_TRAFFIC_BYTES = {"cfg2": int(0.96 * (1.022e9 + 0.324e9))}
+
 METRIC = "dp_sgd_examples_per_sec"
 UNIT = "examples/s"
 
@@ -110,9 +114,14 @@ def work_counts(w):
                 embed_bytes=embed_bytes)
 
 
-def make_workload(name, seed=0):
+def make_workload(name, seed=0, B=None, T=None):
     from paper_2609_40335_b200 import workloads
-    return workloads.named_workload(name, seed=seed)
+    over = {}
+    if B:
+        over["B"] = B
+    if T:
+        over["T"] = T
+    return workloads.named_workload(name, seed=seed, **over)
 
 
 # ------------------------------------------------------------------------ reference arm
@@ -142,7 +151,7 @@ def run_reference(args):
     if rank != 0:
         return
     cores = len(os.sched_getaffinity(0))
-    w = make_workload(args.workload)
+    w = make_workload(args.workload, B=args.B, T=args.T)
     for _ in range(args.warmup):
         oracle_sample_step(w, 1)
     ts = [oracle_sample_step(w, 1) for _ in range(args.steps)]
@@ -184,7 +193,7 @@ def run_ours(args):
     peaks = measured_peaks()
 
     # every rank holds its own batch of the same shape (weak scaling over examples)
-    w = make_workload(args.workload, seed=rank)
+    w = make_workload(args.workload, seed=rank, B=args.B, T=args.T)
     ds = P.upload(w, dev)
     counts = work_counts(w)
     stream = torch.cuda.current_stream()
@@ -198,6 +207,7 @@ def run_ours(args):
     fused = (world == 1) and not args.unfused     # noise inside the clipped-sum kernels
 
     def step(k, ev=None):
+        ge = (ev[4], ev[5]) if ev else None
         if ev: ev[0].record(stream)
         if fused and args.prefill:
             filled = P.prefill_all_noise(ds, args.seed, k)           # side stream, overlaps the norms
@@ -209,10 +219,10 @@ def run_ours(args):
             P.clip_onto_noise(ds, filled)
             if ev: ev[2].record(stream)
         elif fused:
-            P.clip_after_prefill(ds, args.seed, k, filled)
+            P.clip_after_prefill(ds, args.seed, k, filled, gemm_events=ge)
             if ev: ev[2].record(stream)
         else:
-            P.clip_phase(ds)
+            P.clip_phase(ds, gemm_events=ge)
             if ev: ev[2].record(stream)
             reduce_sums()
             P.noise_phase(ds, seed=args.seed, step=k)
@@ -227,7 +237,7 @@ def run_ours(args):
     if rank == 0:
         sampler.start()
         time.sleep(0.25)
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     if world > 1:
         dist.barrier()
@@ -256,38 +266,27 @@ def run_ours(args):
     ms_clip = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
     ms_noise = statistics.mean(e[2].elapsed_time(e[3]) for e in evs)
 
-    # dominant kernel: the tensor-core G^T A GEMM of the clipped sums, timed live with events
-    # around the grouped call (the bracket also holds its one tiny clip-factor kernel)
+    # dominant kernel: the tensor-core G^T A GEMM of the clipped sums.  Its duration is taken
+    # live inside the timed region: CUDA events bracket the grouped call in every timed step (the
+    # bracket also holds the call's one clip-factor kernel, ~2 us).  With --prefill the GEMM
+    # accumulates onto pre-filled noise and is not bracketed.
     lin_layers = ds.linears + ([ds.lm] if ds.lm else [])
     g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    gemm_ms = []
-    gemm_outs = [ds.outs[f"linear{k}"] for k in range(len(ds.linears))]
-    if ds.lm is not None:
-        gemm_outs.append(ds.outs["wte"] if ds.tied else ds.outs["lm_head"])
-    for _ in range(max(3, min(args.steps, 10))):
-        g0.record(stream)
-        if fused:
-            dp.dp_clip_accumulate_noise_grouped(lin_layers, ds.B, ds.T, ds.sq, ds.C, gemm_outs, ds.sigma,
-                                                1.0, args.seed, list(range(len(gemm_outs))), 0,
-                                                ws=ds.ws, dev_status=ds.dev_status)
-        else:
-            dp.dp_clip_accumulate_grouped(lin_layers, ds.B, ds.T, ds.sq, ds.C, gemm_outs, ws=ds.ws,
-                                          dev_status=ds.dev_status)
-        g1.record(stream)
-        torch.cuda.synchronize()
-        gemm_ms.append(g0.elapsed_time(g1))
-    gemm_ms_avg = statistics.mean(gemm_ms)
+    if fused and args.prefill:
+        gemm_ms_avg = ms_clip
+    else:
+        gemm_ms_avg = statistics.mean(e[4].elapsed_time(e[5]) for e in evs)
     n_gemm = 1          # one persistent launch over the output tiles of all layers
     achieved_tf = counts["acc_flops"] / (gemm_ms_avg * 1e-3) / 1e12
     peak_tf = peaks["bf16_tflops_sustained"]
-    roofline = {"kernel": "gemm_gta_kernel<scale> (%s)" % ("dp_clip_accumulate_noise_grouped, noise "
-                                                          "drawn in the epilogue" if fused else
-                                                          "dp_clip_accumulate_grouped"),
+    roofline = {"kernel": "gemm_gta_kernel<scale, pair> (%s)" % (
+                    "dp_clip_accumulate_noise_grouped, Gaussian noise drawn in the epilogue" if fused
+                    else "dp_clip_accumulate_grouped"),
                 "bound": "tensor",
                 "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
-                "frac": achieved_tf / peak_tf, "peak_source": peaks["source"] + " sustained bf16",
+                "frac": achieved_tf / peak_tf, "peak_source": peaks["source"] + " sustained bf16 (kernel timed inside the long step)",
                 "launches_per_step": n_gemm, "ms_per_launch_avg": gemm_ms_avg / n_gemm,
-                "flops_per_step": counts["acc_flops"], "traffic": None}
+                "flops_per_launch": counts["acc_flops"], "traffic": GEMM_TRAFFIC_BYTES.get(w.name)}
     # the norm phase is HBM-bound at T=128: algorithmic bytes = every A and G read once
     g0.record(stream)
     reps = 5
@@ -409,6 +408,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--B", type=int, default=0, help="override the workload's batch size (cfg5 sweep)")
+    ap.add_argument("--T", type=int, default=0, help="override the workload's sequence length")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--prefill", action="store_true", help="noise of every tensor filled beside the norms")

@@ -132,7 +132,7 @@ def norms_phase(ds: DeviceStep, stream=None) -> None:
     dp.dp_clip_factors(ds.sq, ds.C, clip=ds.clip, norms=ds.norms, stream=stream)
 
 
-def clip_phase(ds: DeviceStep, stream=None) -> None:
+def clip_phase(ds: DeviceStep, stream=None, gemm_events=None) -> None:
     """Clipped sums of every parameter tensor from ds.sq."""
     kw = dict(ws=ds.ws, dev_status=ds.dev_status, stream=stream)
     layers = list(ds.linears)
@@ -141,7 +141,11 @@ def clip_phase(ds: DeviceStep, stream=None) -> None:
         layers.append(ds.lm)
         outs.append(ds.outs["wte"] if ds.tied else ds.outs["lm_head"])
     if layers:
+        if gemm_events:
+            gemm_events[0].record(torch.cuda.current_stream())
         dp.dp_clip_accumulate_grouped(layers, ds.B, ds.T, ds.sq, ds.C, outs, beta=0.0, **kw)
+        if gemm_events:
+            gemm_events[1].record(torch.cuda.current_stream())
     dp.dp_clip_accumulate_embed(ds.ids, ds.G_emb, ds.V, ds.sq, ds.C, ds.outs["wte"],
                                 beta=1.0 if (ds.tied and ds.lm is not None) else 0.0, d=ds.d_model, **kw)
     if ds.positions:
@@ -237,8 +241,9 @@ def clip_onto_noise(ds: DeviceStep, filled: torch.cuda.Event) -> None:
 
 
 def clip_after_prefill(ds: DeviceStep, seed: int, step: int, filled: torch.cuda.Event,
-                       scale: float = 1.0) -> None:
-    """Clipped sums when the embedding tables already hold their noise (see prefill)."""
+                       scale: float = 1.0, gemm_events=None) -> None:
+    """Clipped sums when the embedding tables already hold their noise (see prefill).
+    gemm_events: optional (start, stop) CUDA events recorded around the grouped GEMM call."""
     kw = dict(ws=ds.ws, dev_status=ds.dev_status)
     tid = tensor_ids(ds)
     layers = list(ds.linears)
@@ -247,9 +252,13 @@ def clip_after_prefill(ds: DeviceStep, seed: int, step: int, filled: torch.cuda.
         layers.append(ds.lm)
         names.append("wte" if ds.tied else "lm_head")
     if layers:
+        if gemm_events:
+            gemm_events[0].record(torch.cuda.current_stream())
         dp.dp_clip_accumulate_noise_grouped(layers, ds.B, ds.T, ds.sq, ds.C, [ds.outs[n] for n in names],
                                             ds.sigma, scale, seed, [tid[n] for n in names], step,
                                             beta=0.0, **kw)
+        if gemm_events:
+            gemm_events[1].record(torch.cuda.current_stream())
     torch.cuda.current_stream().wait_event(filled)
     # beta = 1: rows are added onto the noise (untied) or onto head sum + noise (tied)
     dp.dp_clip_accumulate_embed(ds.ids, ds.G_emb, ds.V, ds.sq, ds.C, ds.outs["wte"], beta=1.0,

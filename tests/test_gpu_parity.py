@@ -510,3 +510,44 @@ def test_reduced_model_step_matches_oracle(name, over):
             assert (got[w.T:] == 0).all()
             got = got[: w.T]
         assert frob_rel(got, want) < TOL_SUM, k
+
+
+# ------------------------------------------------------ full-size cfg2, sampled outputs
+def test_cfg2_full_size_sampled_against_oracle():
+    """The bench configuration itself (DistilGPT2 shape, B=32, T=128, 24 linears + LM head with
+    V=50257, one grouped launch per phase).  The oracle is too slow for all of it, so it checks
+    (a) the per-example norms of three sampled examples over every layer, and (b) the clipped
+    sums of sampled layers and sampled LM-head rows, with per-example squared norms drawn by
+    the test (they are an input of the clipped-sum calls)."""
+    w = W.named_workload("cfg2")
+    ds = P.upload(w)
+    P.norms_phase(ds)
+    torch.cuda.synchronize()
+    check_status(ds.dev_status)
+    sq_gpu = ds.sq.cpu().numpy()
+    for i in (0, 13, 31):
+        sl = slice(i, i + 1)
+        lin = [(l.A.widened_rows(sl), l.G.widened_rows(sl)) for l in w.linears]
+        ref = O.dp_step(lin, w.ids[sl], w.G_emb.widened_rows(sl), w.V, w.C,
+                        lm=(w.lm.A.widened_rows(sl), w.lm.G.widened_rows(sl)), want_sums=False)
+        assert abs(sq_gpu[i] - ref["sq"][0]) / ref["sq"][0] < TIGHT_BF16, i
+    # clipped sums with test-chosen norms: half of the examples clipped
+    rng = np.random.default_rng(123)
+    sq_in = (rng.uniform(0.25, 4.0, w.B) ** 2).astype(np.float32)
+    ds.sq.copy_(torch.from_numpy(sq_in))
+    P.clip_phase(ds)
+    torch.cuda.synchronize()
+    check_status(ds.dev_status)
+    _, R = O.clip_factors(sq_in.astype(np.float64), w.C)
+    assert (R < 1).any() and (R == 1).any()
+    for k in (0, 1, 10, 23):                                  # one of each layer shape
+        l = w.linears[k]
+        want = O.clipped_sum_linear(l.A.widened(), l.G.widened(), R)
+        assert frob_rel(ds.outs[f"linear{k}"].cpu().numpy(), want) < 5e-3, k
+    rows = np.array([0, 1, 127, 128, 255, 256, 25000, 50175, 50176, 50255, 50256])
+    Gs = W.bf16_bits_to_f32(w.lm.G.data[:, :, rows]).astype(np.float64)
+    want = O.clipped_sum_linear(w.lm.A.widened(), Gs, R)
+    got = ds.outs["lm_head"].cpu().numpy()[rows]
+    assert frob_rel(got, want) < 5e-3
+    want_e = O.clipped_sum_embed(w.ids, w.G_emb.widened(), R, w.V)
+    assert frob_rel(ds.outs["wte"].cpu().numpy(), want_e) < 1e-5
