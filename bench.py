@@ -211,9 +211,10 @@ def run_ours(args):
         if ev: ev[0].record(stream)
         if fused and args.prefill:
             filled = P.prefill_all_noise(ds, args.seed, k)           # side stream, overlaps the norms
-        elif fused:
-            filled = P.prefill_embedding_noise(ds, args.seed, k)     # side stream, overlaps the norms
-        P.norms_phase(ds)
+        if fused and not args.prefill:
+            filled = P.overlapped_norms(ds, args.seed, k)            # noise fill beside the norm kernel
+        else:
+            P.norms_phase(ds)
         if ev: ev[1].record(stream)
         if fused and args.prefill:
             P.clip_onto_noise(ds, filled)

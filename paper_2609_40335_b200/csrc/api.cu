@@ -63,6 +63,15 @@ GhostPlan plan_ghost_norms(const dp_linear_desc* layers, int n_layers, int B, in
     if (items >= 2LL * sms || budget <= 8 || plan.ghost_layers.empty()) break;
     budget /= 2;
   }
+  // longest items first: with a static round-robin split the last, partly filled wave then
+  // holds the cheapest items
+  std::stable_sort(plan.ghost_layers.begin(), plan.ghost_layers.end(), [&](int a, int b) {
+    auto cost = [&](int l) {
+      const GhostLayerPlan& L = plan.layer[l];
+      return std::min(L.a_steps, L.g_steps) + L.chunk_steps;
+    };
+    return cost(a) > cost(b);
+  });
   int col = 0;
   for (int l = 0; l < n_layers; ++l) {
     if (plan.mode_used[l] == DP_NORM_GHOST) {

@@ -271,12 +271,15 @@ sort_place_kernel(const int* __restrict__ ids, int n, int V, const int* __restri
 }
 
 // ------------------------------------------------------------------ segmented row sum
-// grid = (sorted positions, 256-column slabs); only the block sitting on the first sorted
-// position of a token id works.  Rows of the segment are staged 64 at a time (position and clip
-// factor into shared memory), warp w takes rows w, w+8, ... of each stage with all its 16-byte
-// loads in flight together; the 8 per-warp sums are combined in warp order, so the result does
-// not depend on timing.
-constexpr int kScatStage = 64;
+// grid = (64-position chunks of the sorted order, 256-column slabs).  A block finds the segment
+// heads (first sorted position of a token id) inside its chunk and sums each head's rows:
+//   * short segments (<= 32 rows): one warp per segment, lanes own 8 columns, rows are added in
+//     sorted order with 8 row loads in flight;
+//   * long segments (a frequent token): the whole block, rows staged 64 at a time, warp w taking
+//     rows w, w+8, ... of each stage, the 8 per-warp sums combined in warp order.
+// Both orders are fixed, so the result does not depend on timing (no floating-point atomics).
+constexpr int kScatChunk = 64;
+constexpr int kScatShort = 32;
 
 template <typename T>
 __global__ void __launch_bounds__(256)
@@ -285,66 +288,140 @@ embed_scatter_kernel(const int* __restrict__ ids, const T* __restrict__ G, long 
                      const int* __restrict__ seg, int V, float* __restrict__ out, long long ldo,
                      float beta, float scale) {
   __shared__ float part[8][kEmbedColsPerBlock];
-  __shared__ int s_pos[kScatStage];
-  __shared__ float s_r[kScatStage];
-  const int k0 = blockIdx.x;
-  if (k0 >= seg[V]) return;
-  const int pos0 = perm[k0];
-  const int v = ids[pos0];
-  if (seg[v] != k0) return;                    // not the head of its segment
-  const int n = seg[v + 1] - k0;
+  __shared__ int s_pos[kScatChunk];
+  __shared__ float s_r[kScatChunk];
+  __shared__ int s_hk[kScatChunk], s_hv[kScatChunk], s_hn[kScatChunk];
+  __shared__ unsigned s_mask[2];
+  const int n_valid = seg[V];
+  const int kc = blockIdx.x * kScatChunk;
+  if (kc >= n_valid) return;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+
+  // ---- heads of this chunk
+  int my_v = -1, my_n = 0;
+  bool head = false;
+  if (threadIdx.x < kScatChunk) {
+    const int k = kc + threadIdx.x;
+    if (k < n_valid) {
+      my_v = ids[perm[k]];
+      head = (k == 0) || (ids[perm[k - 1]] != my_v);
+      if (head) my_n = seg[my_v + 1] - k;
+    }
+    const unsigned m = __ballot_sync(0xffffffffu, head);
+    if (lane == 0) s_mask[w] = m;
+  }
+  __syncthreads();
+  const int n_heads = __popc(s_mask[0]) + __popc(s_mask[1]);
+  if (threadIdx.x < kScatChunk && head) {
+    const int slot = (w == 1 ? __popc(s_mask[0]) : 0) + __popc(s_mask[w] & ((1u << lane) - 1u));
+    s_hk[slot] = kc + threadIdx.x;
+    s_hv[slot] = my_v;
+    s_hn[slot] = my_n;
+  }
+  __syncthreads();
+
   const int c = blockIdx.y * kEmbedColsPerBlock + lane * 8;
   const int nvalid = min(8, d - c);
   const bool vec = ((reinterpret_cast<uintptr_t>(G) & 15) == 0) && ((ldg * sizeof(T)) % 16 == 0);
-  float acc[8];
+  const bool ovec = ((reinterpret_cast<uintptr_t>(out) & 15) == 0) && ((ldo & 3) == 0);
+
+  // ---- short segments: one warp each
+  for (int h = w; h < n_heads; h += 8) {
+    const int n = s_hn[h];
+    if (n > kScatShort || nvalid <= 0) continue;
+    const int k0 = s_hk[h], v = s_hv[h];
+    float acc[8];
 #pragma unroll
-  for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-  for (int base = 0; base < n; base += kScatStage) {
-    const int m = min(kScatStage, n - base);
-    __syncthreads();
-    if (threadIdx.x < m) {
-      const int pos = perm[k0 + base + threadIdx.x];
-      s_pos[threadIdx.x] = pos;
-      s_r[threadIdx.x] = clip[pos / Tn];
-    }
-    __syncthreads();
-    if (nvalid > 0) {
-      float vals[kScatStage / 8][8];
+    for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+    for (int b0 = 0; b0 < n; b0 += 8) {
+      float vals[8][8];
+      float r[8];
 #pragma unroll
-      for (int b = 0; b < kScatStage / 8; ++b) {
-        const int k = w + 8 * b;
-        if (k < m) {
-          load8<T>(G + size_t(s_pos[k]) * ldg + c, nvalid, vec, vals[b]);
+      for (int b = 0; b < 8; ++b) {
+        if (b0 + b < n) {
+          const int pos = perm[k0 + b0 + b];
+          r[b] = clip[pos / Tn];
+          load8<T>(G + size_t(pos) * ldg + c, nvalid, vec, vals[b]);
         } else {
+          r[b] = 0.f;
 #pragma unroll
           for (int e = 0; e < 8; ++e) vals[b][e] = 0.f;
         }
       }
 #pragma unroll
-      for (int b = 0; b < kScatStage / 8; ++b) {
-        const int k = w + 8 * b;
-        if (k < m) {
-          const float r = s_r[k];
+      for (int b = 0; b < 8; ++b)
 #pragma unroll
-          for (int e = 0; e < 8; ++e) acc[e] = fmaf(r, vals[b][e], acc[e]);
+        for (int e = 0; e < 8; ++e) acc[e] = fmaf(r[b], vals[b][e], acc[e]);
+    }
+    float* o = out + size_t(v) * ldo + c;
+    if (ovec && nvalid == 8) {
+      float4 a = make_float4(acc[0] * scale, acc[1] * scale, acc[2] * scale, acc[3] * scale);
+      float4 b = make_float4(acc[4] * scale, acc[5] * scale, acc[6] * scale, acc[7] * scale);
+      if (beta != 0.f) {
+        const float4 oa = *reinterpret_cast<const float4*>(o), ob = *reinterpret_cast<const float4*>(o + 4);
+        a.x += oa.x; a.y += oa.y; a.z += oa.z; a.w += oa.w;
+        b.x += ob.x; b.y += ob.y; b.z += ob.z; b.w += ob.w;
+      }
+      *reinterpret_cast<float4*>(o) = a;
+      *reinterpret_cast<float4*>(o + 4) = b;
+    } else {
+      for (int e = 0; e < nvalid; ++e) o[e] = (beta != 0.f ? o[e] : 0.f) + acc[e] * scale;
+    }
+  }
+
+  // ---- long segments: the whole block, one after another
+  for (int h = 0; h < n_heads; ++h) {
+    const int n = s_hn[h];
+    if (n <= kScatShort) continue;
+    const int k0 = s_hk[h], v = s_hv[h];
+    float acc[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+    for (int base = 0; base < n; base += kScatChunk) {
+      const int m = min(kScatChunk, n - base);
+      __syncthreads();
+      if (threadIdx.x < m) {
+        const int pos = perm[k0 + base + threadIdx.x];
+        s_pos[threadIdx.x] = pos;
+        s_r[threadIdx.x] = clip[pos / Tn];
+      }
+      __syncthreads();
+      if (nvalid > 0) {
+        float vals[kScatChunk / 8][8];
+#pragma unroll
+        for (int b = 0; b < kScatChunk / 8; ++b) {
+          const int k = w + 8 * b;
+          if (k < m) {
+            load8<T>(G + size_t(s_pos[k]) * ldg + c, nvalid, vec, vals[b]);
+          } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) vals[b][e] = 0.f;
+          }
+        }
+#pragma unroll
+        for (int b = 0; b < kScatChunk / 8; ++b) {
+          const int k = w + 8 * b;
+          if (k < m) {
+            const float r = s_r[k];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = fmaf(r, vals[b][e], acc[e]);
+          }
         }
       }
     }
-  }
 #pragma unroll
-  for (int e = 0; e < 8; ++e) part[w][lane * 8 + e] = acc[e];
-  __syncthreads();
-  {
+    for (int e = 0; e < 8; ++e) part[w][lane * 8 + e] = acc[e];
+    __syncthreads();
     const int cc = blockIdx.y * kEmbedColsPerBlock + threadIdx.x;
     if (cc < d) {
-      float s = 0.f;
+      float sum = 0.f;
 #pragma unroll
-      for (int ww = 0; ww < 8; ++ww) s += part[ww][threadIdx.x];
+      for (int ww = 0; ww < 8; ++ww) sum += part[ww][threadIdx.x];
       float* o = out + size_t(v) * ldo + cc;
-      s *= scale;
-      *o = (beta != 0.f) ? (*o + s) : s;
+      sum *= scale;
+      *o = (beta != 0.f) ? (*o + sum) : sum;
     }
+    __syncthreads();
   }
 }
 
@@ -400,7 +477,7 @@ dp_status launch_embed_scatter(const int* ids, const void* G, int64_t ldg, dp_dt
     DP_CUDA_OK(cudaMemset2DAsync(out, size_t(ldo) * sizeof(float), 0, size_t(d) * sizeof(float),
                                  size_t(V), st));
   }
-  dim3 grid(n, ceil_div(d, kEmbedColsPerBlock));
+  dim3 grid(ceil_div(n, kScatChunk), ceil_div(d, kEmbedColsPerBlock));
   if (dt == DP_F32)
     embed_scatter_kernel<float><<<grid, 256, 0, st>>>(ids, (const float*)G, ldg, T, d, clip, perm,
                                                      seg, V, out, ldo, 1.f, scale);

@@ -159,7 +159,7 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
   if (warp == 0) {
     // ------------------------------------------------------------- TMA producer
     if (lane == 0) {
-      uint32_t stage = 0, phase = 0;
+      uint32_t stage = 0, phase = 0, issued = 0;
       bool ok = true;
       for (int item = first_item; item < P.total_items && ok; item += item_stride) {
         const Item it = decode_item<kSqsum>(P, item);
@@ -178,12 +178,14 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
 #pragma unroll
           for (int j = 0; j < Geo<kPair>::kAColsPerCta / 64; ++j)
             ptx::tma_load_3d(dst + kGBytes + j * kBoxBytes, ta, &full[stage], n0 + j * 64, t0, ex);
+          ++issued;
           if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
       }
       if (!ok) {
         *abort_flag = 1;
         if (P.dev_status) atomicOr(P.dev_status, DP_DEV_TIMEOUT);
+        ptx::drain_issued_copies(full, kStages, issued);   // copies in flight land before exit
       }
     }
   } else if (warp == 1) {

@@ -30,11 +30,17 @@ namespace {
 constexpr int kTile = 128;                       // Gram tile edge (rows of A_i / G_i)
 constexpr int kKStep = 64;                       // bf16 columns per stage row (128 bytes)
 constexpr int kTileBytes = kTile * kKStep * 2;   // 16 KiB
-constexpr int kStageBytes = 2 * kTileBytes;      // row tile ti and row tile tj
-constexpr int kStages = 6;
+// A stage holds row tile ti and, for off-diagonal tile pairs, row tile tj.  When T <= 128 every
+// pair is diagonal, so stages shrink to one tile and twice as many are kept in flight (the
+// kernel is HBM-bound there: bytes in flight are what counts).
+template <bool kDiagOnly>
+struct GhostGeo {
+  static constexpr int kStageBytes = kDiagOnly ? kTileBytes : 2 * kTileBytes;
+  static constexpr int kStages = kDiagOnly ? 12 : 6;
+  static constexpr size_t kSmemBytes = size_t(kStages) * kStageBytes + 1024 /*alignment slack*/ + 512;
+};
 constexpr int kThreads = 192;
 constexpr int kTmemCols = 512;                   // 2 buffers x (S_A 128 + S_G 128) columns
-constexpr size_t kSmemBytes = size_t(kStages) * kStageBytes + 1024 /*alignment slack*/ + 256;
 
 struct __align__(64) GhostParams {
   CUtensorMap tmA[kGhostMaxLayers];
@@ -78,8 +84,11 @@ __device__ __forceinline__ Item decode_item(const GhostParams& P, int item) {
   return it;
 }
 
+template <bool kDiagOnly>
 __global__ void __launch_bounds__(kThreads, 1)
 ghost_norm_tc_kernel(const __grid_constant__ GhostParams P) {
+  constexpr int kStages = GhostGeo<kDiagOnly>::kStages;
+  constexpr int kStageBytes = GhostGeo<kDiagOnly>::kStageBytes;
   extern __shared__ uint8_t smem_raw[];
   // 128-byte swizzled tiles need 1024-byte alignment
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
@@ -114,11 +123,11 @@ ghost_norm_tc_kernel(const __grid_constant__ GhostParams P) {
   if (warp == 0) {
     // ------------------------------------------------------------- TMA producer
     if (lane == 0) {
-      uint32_t stage = 0, phase = 0;
+      uint32_t stage = 0, phase = 0, issued = 0;
       bool ok = true;
       for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x) {
         const Item it = decode_item(P, item);
-        const bool diag = (it.ti == it.tj);
+        const bool diag = kDiagOnly || (it.ti == it.tj);
         const uint32_t bytes = diag ? kTileBytes : kStageBytes;
         for (int pass = 0; pass < 2 && ok; ++pass) {
           const CUtensorMap* tm = pass == 0 ? &P.tmA[it.layer] : &P.tmG[it.layer];
@@ -131,6 +140,7 @@ ghost_norm_tc_kernel(const __grid_constant__ GhostParams P) {
             if (!diag)
               ptx::tma_load_3d(dst + kTileBytes, tm, &full[stage], k * kKStep, it.tj * kTile,
                                it.example);
+            ++issued;
             if (++stage == kStages) { stage = 0; phase ^= 1; }
           }
         }
@@ -138,10 +148,7 @@ ghost_norm_tc_kernel(const __grid_constant__ GhostParams P) {
       if (!ok) {
         *abort_flag = 1;
         if (P.dev_status) atomicOr(P.dev_status, DP_DEV_TIMEOUT);
-        // let copies already in flight land before the CTA may exit
-        for (int s = 0; s < kStages; ++s) {
-          (void)ptx::mbar_wait(&full[s], 0, abort_flag + 0 * s);   // bounded
-        }
+        ptx::drain_issued_copies(full, kStages, issued);   // copies in flight land before exit
       }
     }
   } else if (warp == 1) {
@@ -154,7 +161,7 @@ ghost_norm_tc_kernel(const __grid_constant__ GhostParams P) {
       bool ok = true;
       for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x, ++n_item) {
         const Item it = decode_item(P, item);
-        const bool diag = (it.ti == it.tj);
+        const bool diag = kDiagOnly || (it.ti == it.tj);
         const uint32_t buf = n_item & 1, acc_phase = (n_item >> 1) & 1;
         if (!ptx::mbar_wait(&acc_empty[buf], acc_phase ^ 1, abort_flag)) { ok = false; break; }
         ptx::tc_fence_after();
@@ -264,8 +271,12 @@ dp_status launch_ghost_norm_tc(const dp_linear_desc* layers, const GhostPlan& pl
                                float* partials, int* dev_status, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
-    DP_CUDA_OK(cudaFuncSetAttribute(ghost_norm_tc_kernel,
-                                    cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
+    DP_CUDA_OK(cudaFuncSetAttribute(ghost_norm_tc_kernel<true>,
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)GhostGeo<true>::kSmemBytes));
+    DP_CUDA_OK(cudaFuncSetAttribute(ghost_norm_tc_kernel<false>,
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)GhostGeo<false>::kSmemBytes));
     attr_set = true;
   }
   const int nt = ceil_div(T, kTile);
@@ -294,7 +305,10 @@ dp_status launch_ghost_norm_tc(const dp_linear_desc* layers, const GhostPlan& pl
     P.partials = partials;
     P.dev_status = dev_status;
     const int grid = std::min(items, sm_count());
-    ghost_norm_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(P);
+    if (nt == 1)
+      ghost_norm_tc_kernel<true><<<grid, kThreads, GhostGeo<true>::kSmemBytes, st>>>(P);
+    else
+      ghost_norm_tc_kernel<false><<<grid, kThreads, GhostGeo<false>::kSmemBytes, st>>>(P);
     DP_LAUNCH_OK();
   }
   return DP_OK;

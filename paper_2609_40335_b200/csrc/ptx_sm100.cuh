@@ -67,6 +67,20 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
   return true;
 }
 
+// After a producer gave up: wait (bounded, ~0.1 s per stage) until the copies it had already
+// issued have landed, so that the CTA does not exit with TMA writes to its shared memory in
+// flight.  `issued` counts all stages armed so far on the ring of `n_stages` full-barriers.
+__device__ __forceinline__ void drain_issued_copies(uint64_t* full, int n_stages, uint32_t issued) {
+  const uint32_t first = issued > (uint32_t)n_stages ? issued - n_stages : 0u;
+  for (uint32_t i = first; i < issued; ++i) {
+    const uint32_t stage = i % n_stages, parity = (i / n_stages) & 1u;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(&full[stage], parity)) {
+      if (clock64() - t0 > 150000000LL) break;
+    }
+  }
+}
+
 // ----------------------------------------------------------------------- TMA
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* m) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");

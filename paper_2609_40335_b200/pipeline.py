@@ -116,12 +116,16 @@ def allocate(ds: DeviceStep) -> None:
     ds.ws = torch.empty(need, dtype=torch.uint8, device=dev)
 
 
-def norms_phase(ds: DeviceStep, stream=None) -> None:
-    """Per-example squared norms into ds.sq (zeroed first), then norms and clip factors."""
+def norms_phase(ds: DeviceStep, stream=None, after_first_launch=None) -> None:
+    """Per-example squared norms into ds.sq (zeroed first), then norms and clip factors.
+    after_first_launch: called right after the big norm kernel has been enqueued (used to start
+    side-stream work that should share the SMs with it rather than run ahead of it)."""
     ds.sq.zero_()
     every = ds.linears + ([ds.lm] if ds.lm else [])
     if every:
         dp.dp_ghost_norms(every, ds.B, ds.T, ds.sq, ws=ds.ws, dev_status=ds.dev_status, stream=stream)
+    if after_first_launch is not None:
+        after_first_launch()
     dp.dp_embed_norms(ds.ids, ds.G_emb, ds.V, ds.sq, ws=ds.ws, dev_status=ds.dev_status, stream=stream)
     if ds.positions:
         dp.dp_embed_norms(ds.pos_ids, ds.G_emb, ds.T, ds.sq, ws=ds.ws, dev_status=ds.dev_status,
@@ -188,15 +192,21 @@ def clip_noise_phase(ds: DeviceStep, seed: int, step: int, scale: float = 1.0, s
                                           d=ds.d_model, **kw)
 
 
-def prefill_embedding_noise(ds: DeviceStep, seed: int, step: int, scale: float = 1.0) -> torch.cuda.Event:
+def prefill_embedding_noise(ds: DeviceStep, seed: int, step: int, scale: float = 1.0,
+                            after: Optional[torch.cuda.Event] = None) -> torch.cuda.Event:
     """Start the noise fill of the embedding tables on a side stream.  The fill depends on no
-    gradient, so it overlaps the (HBM-bound) norm phase; returns the event to wait for."""
+    gradient, so it overlaps the (HBM-bound) norm phase; returns the event to wait for.
+    after: event that orders the fill behind the previous users of the tables (default: all
+    work enqueued so far on the current stream)."""
     if ds.side_stream is None:
         ds.side_stream = torch.cuda.Stream(device=ds.sq.device)
     main = torch.cuda.current_stream()
     tid = tensor_ids(ds)
     side = ds.side_stream
-    side.wait_stream(main)                       # previous step's readers of the tables are done
+    if after is not None:
+        side.wait_event(after)
+    else:
+        side.wait_stream(main)                   # previous step's readers of the tables are done
     names = ["wpe"] if ds.positions else []
     if not (ds.tied and ds.lm is not None):
         names.append("wte")                      # tied: the head GEMM writes the table first
@@ -268,6 +278,21 @@ def clip_after_prefill(ds: DeviceStep, seed: int, step: int, filled: torch.cuda.
                                     beta=1.0, d=ds.d_model, **kw)
 
 
+def overlapped_norms(ds: DeviceStep, seed: int, step: int) -> torch.cuda.Event:
+    """Norm phase with the embedding tables' noise fill beside it.  The fill is enqueued right
+    AFTER the big norm kernel: measured on B200, a fill that is already resident keeps the norm
+    kernel's CTAs out until it ends, while a fill that arrives second shares the SMs."""
+    start = torch.cuda.Event()
+    start.record(torch.cuda.current_stream())
+    box = {}
+
+    def launch_fill():
+        box["ev"] = prefill_embedding_noise(ds, seed, step, after=start)
+
+    norms_phase(ds, after_first_launch=launch_fill)
+    return box["ev"]
+
+
 def dp_step(ds: DeviceStep, seed: int = 0, step: int = 0, noise: bool = True, fused: bool = True,
             overlap: bool = True, stream=None) -> None:
     """norms -> clipped sums -> noise.
@@ -276,8 +301,7 @@ def dp_step(ds: DeviceStep, seed: int = 0, step: int = 0, noise: bool = True, fu
     embedding tables' noise is filled on a side stream while the norms run (scale 1 only).
     """
     if noise and fused and overlap and stream is None:
-        filled = prefill_embedding_noise(ds, seed, step)
-        norms_phase(ds)
+        filled = overlapped_norms(ds, seed, step)
         clip_after_prefill(ds, seed, step, filled)
         return
     norms_phase(ds, stream)

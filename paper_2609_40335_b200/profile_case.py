@@ -69,6 +69,39 @@ def case_ghost_long(reps):
           f"{nbytes / ms / 1e6:.0f} GB/s algorithmic")
 
 
+def case_overlap(reps):
+    """Does the ALU-bound noise fill share the SMs with the HBM-bound norm kernel?"""
+    B, T = 32, 128
+    layers = [dp.Linear(_randn_bf16(B, T, 768), _randn_bf16(B, T, 3072, std=1e-2)) for _ in range(18)]
+    sq = torch.zeros(B, device="cuda")
+    x = torch.empty(50257 * 768, device="cuda")
+    side = torch.cuda.Stream()
+    main = torch.cuda.current_stream()
+    ws = torch.empty(dp.dp_ghost_norms_ws_bytes(layers, B, T), dtype=torch.uint8, device="cuda")
+
+    def run(mode):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(main)
+        for k in range(reps):
+            if mode in ("fill", "fill_first"):
+                side.wait_stream(main)
+                dp.dp_fill_noise(x, 0.8, 1.0, 1.0, 1, 0, k, stream=side)
+            if mode != "fill":
+                dp.dp_ghost_norms(layers, B, T, sq, ws=ws)
+            if mode == "ghost_first":
+                side.wait_stream(main) if False else None
+                dp.dp_fill_noise(x, 0.8, 1.0, 1.0, 1, 0, k, stream=side)
+            main.wait_stream(side)
+        e1.record(main)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    for mode in ("ghost", "fill", "fill_first", "ghost_first"):
+        run(mode)
+        print(f"overlap[{mode}]: {run(mode):.4f} ms per iteration")
+
+
 def case_noise(reps):
     x = torch.zeros(50257 * 768, device="cuda")
     for k in range(reps):
@@ -101,7 +134,7 @@ def main():
     which = sys.argv[1] if len(sys.argv) > 1 else "gemm"
     reps = int(sys.argv[2]) if len(sys.argv) > 2 else 3
     torch.manual_seed(0)
-    {"gemm": case_gemm, "gemm1": case_gemm_unclipped, "ghost512": case_ghost_long, "ghost": case_ghost, "noise": case_noise, "embed": case_embed,
+    {"gemm": case_gemm, "gemm1": case_gemm_unclipped, "ghost512": case_ghost_long, "overlap": case_overlap, "ghost": case_ghost, "noise": case_noise, "embed": case_embed,
      "cross": case_cross}[which](reps)
     torch.cuda.synchronize()
     print("done", which, reps)
