@@ -3,6 +3,7 @@
 #include <cmath>
 #include <cstring>
 
+#include "cross_term.cuh"
 #include "dp_common.cuh"
 #include "fma_kernels.cuh"
 #include "gemm_gta.cuh"
@@ -202,7 +203,9 @@ dp_status dp_embed_norms(const int32_t* ids, const void* G, int64_t ldg, dp_dtyp
 size_t dp_tied_cross_term_ws_bytes(int32_t B, int32_t T, int32_t d, int32_t V) {
   (void)d; (void)V;
   if (B <= 0 || T <= 0) return 0;
-  return align_up(size_t(B) * ceil_div(T, 16) * sizeof(float), 256);
+  // enough for either kernel: one partial per 16-token slab (fp32 path) or per 128 x 128 tile
+  const int per = std::max(ceil_div(T, 16), cross_term_tc_partials_per_example(T));
+  return align_up(size_t(B) * per * sizeof(float), 256);
 }
 
 dp_status dp_tied_cross_term(const int32_t* ids, const void* G_emb, int64_t ldge, const void* A_lm,
@@ -214,13 +217,24 @@ dp_status dp_tied_cross_term(const int32_t* ids, const void* G_emb, int64_t ldge
   if (!sq && !cross) return DP_ERR_INVALID_ARG;
   if (ldge < d || ldal < d || ldgl < V) return DP_ERR_INVALID_ARG;
   if (dt != DP_F32 && dt != DP_BF16) return DP_ERR_INVALID_ARG;
+  const bool tc = (dt == DP_BF16) && !g_force_fma;
+  if (tc && (!aligned16(G_emb) || !aligned16(A_lm) || (ldge % 8) || (ldal % 8))) return DP_ERR_ALIGNMENT;
   if (!ws || ws_bytes < dp_tied_cross_term_ws_bytes(B, T, d, V)) return DP_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   float* partials = static_cast<float*>(ws);
-  dp_status s = launch_cross_term_fma(ids, G_emb, ldge, A_lm, ldal, G_lm, ldgl, dt, B, T, d, V,
-                                      partials, dev_status, st);
+  dp_status s;
+  int per;
+  if (tc) {
+    s = launch_cross_term_tc(ids, G_emb, ldge, A_lm, ldal, G_lm, ldgl, B, T, d, V, partials,
+                             dev_status, st);
+    per = cross_term_tc_partials_per_example(T);
+  } else {
+    s = launch_cross_term_fma(ids, G_emb, ldge, A_lm, ldal, G_lm, ldgl, dt, B, T, d, V, partials,
+                              dev_status, st);
+    per = ceil_div(T, 16);
+  }
   if (s != DP_OK) return s;
-  return launch_reduce_partials(partials, ceil_div(T, 16), B, sq, 2.f, cross, st);
+  return launch_reduce_partials(partials, per, B, sq, 2.f, cross, st);
 }
 
 // --------------------------------------------------------------------------- clip factors

@@ -317,12 +317,14 @@ def test_clip_accumulate_embed(dtype, B, T, d, V, beta):
 
 # --------------------------------------------------------------------------- tied cross term
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-@pytest.mark.parametrize("B,T,d,V", [(3, 16, 64, 1000), (2, 128, 768, 50257), (2, 70, 100, 33)])
+@pytest.mark.parametrize("B,T,d,V", [(3, 16, 64, 1000), (2, 128, 768, 50257), (2, 70, 100, 33),
+                                     (2, 300, 136, 4099)])
 def test_tied_cross_term(dtype, B, T, d, V):
     g_std = 1.0 if dtype == "f32" else 1e-2
     ids = W.zipf_ids(B, T, V, 1.1, 31)
-    G_emb = W._normal((B, T, d), g_std, dtype, 32)
-    A_lm = W._normal((B, T, d), 1.0, dtype, 33)
+    ldd = W.round_up(d, 8) if (dtype == "bf16" and d % 8) else None     # TMA pitch, NaN padding
+    G_emb = W._normal((B, T, d), g_std, dtype, 32, ld=ldd)
+    A_lm = W._normal((B, T, d), 1.0, dtype, 33, ld=ldd)
     ld = W.round_up(V, 8) if dtype == "bf16" else V
     G_lm = W._normal((B, T, V), g_std, dtype, 34, ld=ld if ld != V else None)
     ref = O.tied_sq_norms(ids, G_emb.widened(), A_lm.widened(), G_lm.widened(), V)
