@@ -193,8 +193,19 @@ def run_ours(args):
     peaks = measured_peaks()
 
     # every rank holds its own batch of the same shape (weak scaling over examples)
-    w = make_workload(args.workload, seed=rank, B=args.B, T=args.T)
-    ds = P.upload(w, dev)
+    if args.device_inputs:
+        # large sweep cells: inputs drawn on the device (host generation would take minutes)
+        import types
+        assert args.workload == "cfg5", "--device-inputs is for the GPT-2-medium sweep"
+        B_, T_ = args.B or 16, args.T or 128
+        ds = P.synthesize_on_device("cfg5", B_, T_, 1024, 24, seed=rank, device=dev)
+        w = types.SimpleNamespace(
+            name="cfg5", dtype="bf16", B=B_, T=T_, V=50257, d_model=1024, tied=False, positions=False,
+            linears=[types.SimpleNamespace(d=l.d, p=l.p) for l in ds.linears],
+            lm=types.SimpleNamespace(d=ds.lm.d, p=ds.lm.p))
+    else:
+        w = make_workload(args.workload, seed=rank, B=args.B, T=args.T)
+        ds = P.upload(w, dev)
     counts = work_counts(w)
     stream = torch.cuda.current_stream()
 
@@ -324,7 +335,8 @@ def run_ours(args):
     # from pinned host memory and reads the per-example norms and clip factors back
     host_in, dev_in = [], []
     seen = set()
-    for t in [ds.ids, ds.G_emb] + [x for l in lin_layers for x in (l.A, l.G)]:
+    e2e_enabled = ds.input_bytes() < 8e9 and not args.device_inputs
+    for t in ([ds.ids, ds.G_emb] + [x for l in lin_layers for x in (l.A, l.G)]) if e2e_enabled else []:
         if t.data_ptr() in seen:
             continue
         seen.add(t.data_ptr())
@@ -343,7 +355,7 @@ def run_ours(args):
         host_out[1].copy_(ds.clip, non_blocking=True)
         torch.cuda.synchronize()
 
-    e2e_steps = max(3, min(args.steps, 10))
+    e2e_steps = max(3, min(args.steps, 10)) if e2e_enabled else 1
     e2e_step(0)
     if world > 1:
         dist.barrier()
@@ -365,7 +377,7 @@ def run_ours(args):
 
     # CPU baseline: the oracle on a bounded sample, on this machine's host cores (rank 0, N=1 only)
     cpu = None
-    if world == 1 and not args.no_cpu_baseline:
+    if world == 1 and not args.no_cpu_baseline and not args.device_inputs:
         n_ex = 4
         t_ex = oracle_sample_step(w, n_ex)
         n_noise = 4_000_000
@@ -392,8 +404,8 @@ def run_ours(args):
         "clocks": clocks,
         "roofline": roofline,
         "roofline_other": others,
-        "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
-                "d2h_bytes_per_step": int(d2h), "steps": e2e_steps},
+        "e2e": ({"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+                 "d2h_bytes_per_step": int(d2h), "steps": e2e_steps} if e2e_enabled else None),
         "cpu_baseline": cpu,
         "peaks": peaks,
     }
@@ -411,6 +423,8 @@ def main():
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--B", type=int, default=0, help="override the workload's batch size (cfg5 sweep)")
     ap.add_argument("--T", type=int, default=0, help="override the workload's sequence length")
+    ap.add_argument("--device-inputs", action="store_true",
+                    help="cfg5 only: draw the inputs on the device (big cells)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--prefill", action="store_true", help="noise of every tensor filled beside the norms")

@@ -225,6 +225,13 @@ int64_t dp_kernel_launches(void);
  * instead of the tensor-core ones (used to cross-check the two on the device).  Returns
  * the previous value.  Off by default; not meant for production use. */
 int32_t dp_debug_force_fma(int32_t on);
+/* Diagnostics.  dp_debug_noise_error_scan: exhaustive float64 check of the fp32 Box-Muller
+ * factors over all 2^24 inputs; out4 [dev, 4 doubles] = {max relative error of the radius for
+ * r^2 <= t_max (t_max <= 0: the threshold in use), max absolute error of cos/sin, largest radius
+ * seen, the compiled r^2 threshold}.  dp_debug_max_active_pairs: CTA pairs of the clipped-sum
+ * kernel the device can hold. */
+dp_status dp_debug_noise_error_scan(float t_max, double* out4, void* stream);
+int32_t dp_debug_max_active_pairs(void);
 
 #ifdef __cplusplus
 }

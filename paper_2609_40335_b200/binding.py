@@ -41,7 +41,8 @@ EXPORTS = ["dp_ghost_norms", "dp_ghost_norms_ws_bytes", "dp_embed_norms", "dp_em
            "dp_clip_accumulate_grouped_ws_bytes", "dp_clip_accumulate_noise_grouped",
            "dp_clip_accumulate_embed_noise", "dp_clip_accumulate_embed",
            "dp_clip_accumulate_embed_ws_bytes", "dp_add_noise", "dp_fill_noise", "dp_status_string",
-           "dp_last_cuda_error", "dp_version", "dp_kernel_launches", "dp_debug_force_fma"]
+           "dp_last_cuda_error", "dp_version", "dp_kernel_launches", "dp_debug_force_fma",
+           "dp_debug_noise_error_scan", "dp_debug_max_active_pairs"]
 
 
 def lib_path() -> str:
@@ -95,6 +96,8 @@ def load():
     L.dp_last_cuda_error.restype = i32
     L.dp_version.restype = C.c_char_p
     L.dp_kernel_launches.restype = C.c_int64
+    L.dp_debug_noise_error_scan.argtypes = [f32, vp, vp]
+    L.dp_debug_max_active_pairs.restype = i32
     L.dp_debug_force_fma.argtypes = [i32]
     L.dp_debug_force_fma.restype = i32
     for name in EXPORTS:

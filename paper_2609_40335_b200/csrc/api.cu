@@ -126,6 +126,10 @@ int32_t dp_last_cuda_error(void) { return g_last_cuda_error; }
 const char* dp_version(void) { return "dp_ghost 0.1.0 (sm_100a)"; }
 int64_t dp_kernel_launches(void) { return g_kernel_launches; }
 int32_t dp_debug_max_active_pairs(void) { return gta_max_active_pairs(); }
+dp_status dp_debug_noise_error_scan(float t_max, double* out3, void* stream) {
+  if (!out3) return DP_ERR_INVALID_ARG;
+  return launch_noise_error_scan(t_max, out3, (cudaStream_t)stream);
+}
 int32_t dp_debug_force_fma(int32_t on) {
   const int prev = g_force_fma;
   g_force_fma = on ? 1 : 0;

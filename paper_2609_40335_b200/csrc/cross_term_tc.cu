@@ -141,7 +141,7 @@ cross_term_tc_kernel(const __grid_constant__ CrossParams P) {
         }
       }
       const __nv_bfloat16* gcol = P.Glm + size_t(ex) * P.T * P.ldgl + (id >= 0 ? id : 0);
-      if (!ptx::mbar_wait(&acc_full[buf], acc_phase, abort_flag)) { ok = false; break; }
+      if (!ptx::mbar_wait_relaxed(&acc_full[buf], acc_phase, abort_flag)) { ok = false; break; }
       ptx::tc_fence_after();
       const uint32_t t0 = tmem_base + (uint32_t(q * 32) << 16) + buf * kTile;
       float acc = 0.f;

@@ -46,4 +46,6 @@ dp_status launch_add_noise(float* out, long long rows, int cols, long long ld, b
                            float scale, uint64_t seed, uint32_t tensor_id, uint32_t step,
                            cudaStream_t st);
 
+dp_status launch_noise_error_scan(float t_max, double* out3, cudaStream_t st);
+
 }  // namespace dpg

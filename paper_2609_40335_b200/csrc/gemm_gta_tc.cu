@@ -301,7 +301,7 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
       const Item it = decode_item<kSqsum>(P, item);
       const GtaLayer& L = P.layer[it.layer];
       const uint32_t buf = n_item & 1, acc_phase = (n_item >> 1) & 1;
-      if (!ptx::mbar_wait(&acc_full[buf], acc_phase, abort_flag)) { ok = false; break; }
+      if (!ptx::mbar_wait_relaxed(&acc_full[buf], acc_phase, abort_flag)) { ok = false; break; }
       ptx::tc_fence_after();
       const uint32_t t0 = tmem_base + (uint32_t(q * 32) << 16) + buf * kBN;
       const int row = it.tm * kTileM + int(rank) * kBM + q * 32 + lane;

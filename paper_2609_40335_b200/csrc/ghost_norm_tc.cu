@@ -200,7 +200,7 @@ ghost_norm_tc_kernel(const __grid_constant__ GhostParams P) {
     for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x, ++n_item) {
       const Item it = decode_item(P, item);
       const uint32_t buf = n_item & 1, acc_phase = (n_item >> 1) & 1;
-      if (!ptx::mbar_wait(&acc_full[buf], acc_phase, abort_flag)) { ok = false; break; }
+      if (!ptx::mbar_wait_relaxed(&acc_full[buf], acc_phase, abort_flag)) { ok = false; break; }
       ptx::tc_fence_after();
       const uint32_t t0 = tmem_base + (uint32_t(q * 32) << 16) + buf * 256;
       float acc = 0.f;

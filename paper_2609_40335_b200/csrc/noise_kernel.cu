@@ -41,7 +41,43 @@ add_noise_kernel(float* __restrict__ out, long long n, int cols, long long ld, f
   }
 }
 
+// Exhaustive error scan of the fp32 Box-Muller factors.  k runs over all 2^24 values of the
+// 24-bit integer that feeds the factor.  out[0] = max relative error of r = sqrt(-2 ln u1) over
+// the inputs with r^2 <= t_max, out[1] = max absolute error of cos / sin(2 pi u2), out[2] = the
+// largest r seen, all against float64; out[3] = the r^2 threshold compiled into box_muller.
+__global__ void noise_error_scan_kernel(float t_max, double* out) {
+  double er = 0.0, ed = 0.0, rmax = 0.0;
+  for (uint32_t k = blockIdx.x * blockDim.x + threadIdx.x; k < (1u << 24); k += gridDim.x * blockDim.x) {
+    const float t = bm_t_f32(k);
+    if (t <= t_max) {
+      const double r32 = (double)__fsqrt_rn(t);
+      const double r64 = sqrt(-2.0 * log(double(k + 1u) * 5.9604644775390625e-08));
+      if (r64 > 0.0) er = fmax(er, fabs(r32 - r64) / r64);
+      rmax = fmax(rmax, r64);
+    }
+    float s, c;
+    bm_dir_f32(k, s, c);
+    double s64, c64;
+    sincospi(double(k) * 1.1920928955078125e-07, &s64, &c64);
+    ed = fmax(ed, fmax(fabs((double)s - s64), fabs((double)c - c64)));
+  }
+  // block-free reduction: doubles compare as integers when non-negative
+  atomicMax(reinterpret_cast<unsigned long long*>(out + 0), (unsigned long long)__double_as_longlong(er));
+  atomicMax(reinterpret_cast<unsigned long long*>(out + 1), (unsigned long long)__double_as_longlong(ed));
+  atomicMax(reinterpret_cast<unsigned long long*>(out + 2), (unsigned long long)__double_as_longlong(rmax));
+}
+
 }  // namespace
+
+dp_status launch_noise_error_scan(float t_max, double* out3 /*4 doubles*/, cudaStream_t st) {
+  DP_CUDA_OK(cudaMemsetAsync(out3, 0, 3 * sizeof(double), st));
+  if (t_max <= 0.f) t_max = DPG_NOISE_TAIL_T;             // scan exactly the fp32 path in use
+  noise_error_scan_kernel<<<sm_count() * 8, 256, 0, st>>>(t_max, out3);
+  DP_LAUNCH_OK();
+  const double thr = DPG_NOISE_TAIL_T;
+  DP_CUDA_OK(cudaMemcpyAsync(out3 + 3, &thr, sizeof(double), cudaMemcpyHostToDevice, st));
+  return DP_OK;
+}
 
 dp_status launch_add_noise(float* out, long long rows, int cols, long long ld, bool fill, float amp,
                            float scale, uint64_t seed, uint32_t tensor_id, uint32_t step,

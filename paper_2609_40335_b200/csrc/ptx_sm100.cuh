@@ -67,6 +67,24 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
   return true;
 }
 
+// Same bounded wait for roles that can afford latency (an epilogue waiting a whole tile for its
+// accumulator): sleeps between polls so that many waiting warps do not take issue slots from
+// the few latency-critical ones (TMA producer, MMA issuer, scalers).
+__device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity,
+                                                  volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  uint32_t spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    __nanosleep(spins < 64 ? 64 : 512);
+    if ((++spins & 255u) == 0) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > 1500000000LL) return false;
+    }
+  }
+  return true;
+}
+
 // After a producer gave up: wait (bounded, ~0.1 s per stage) until the copies it had already
 // issued have landed, so that the CTA does not exit with TMA writes to its shared memory in
 // flight.  `issued` counts all stages armed so far on the ring of `n_stages` full-barriers.

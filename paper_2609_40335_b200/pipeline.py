@@ -54,6 +54,7 @@ class DeviceStep:
     side_stream: Optional[torch.cuda.Stream] = None     # noise fills that overlap the norm phase
 
     def input_bytes(self) -> int:
+        """Bytes of input one step reads (a tensor shared by several layers counts every time)."""
         n = self.ids.numel() * 4 + self.G_emb.numel() * self.G_emb.element_size()
         for l in self.linears + ([self.lm] if self.lm else []):
             n += l.A.numel() * l.A.element_size() + l.G.numel() * l.G.element_size()
@@ -84,6 +85,46 @@ def upload(w: Workload, device="cuda", share_by_identity: bool = True) -> Device
         clip=torch.zeros(w.B, dtype=torch.float32, device=device),
         norms=torch.zeros(w.B, dtype=torch.float32, device=device),
         cross=torch.zeros(w.B, dtype=torch.float32, device=device) if w.tied else None,
+        dev_status=torch.zeros(1, dtype=torch.int32, device=device))
+    allocate(ds)
+    return ds
+
+
+def synthesize_on_device(name: str, B: int, T: int, d_model: int, n_blocks: int, V: int = 50257,
+                         tied: bool = False, positions: bool = False, C: float = 1.0,
+                         sigma: float = 1.0, seed: int = 0, device="cuda") -> DeviceStep:
+    """Benchmark-only inputs drawn on the device (torch generator), for shapes whose host-side
+    generation would take minutes: A ~ N(0,1), G ~ N(0,1e-4), Zipf(1.1) token ids, one tensor set
+    per distinct layer shape shared by all blocks, LM-head pitch padded to a multiple of 8."""
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+
+    def normal(rows, cols, std, ld=None):
+        ld = ld or cols
+        t = torch.empty(B, rows, ld, dtype=torch.bfloat16, device=device)
+        step = max(1, (1 << 28) // (rows * ld))          # bounded fp32 staging buffer
+        for b0 in range(0, B, step):
+            b1 = min(B, b0 + step)
+            x = torch.randn(b1 - b0, rows, ld, generator=g, device=device, dtype=torch.float32)
+            t[b0:b1] = (x * std).to(torch.bfloat16)
+        return t
+
+    shapes = [(d_model, 3 * d_model), (d_model, d_model), (d_model, 4 * d_model), (4 * d_model, d_model)]
+    sets = [(normal(T, d, 1.0), normal(T, p, 1e-2)) for d, p in shapes]
+    linears = [dp.Linear(sets[k][0], sets[k][1], d=shapes[k][0], p=shapes[k][1])
+               for _ in range(n_blocks) for k in range(4)]
+    ldv = (V + 7) // 8 * 8
+    lm = dp.Linear(normal(T, d_model, 1.0), normal(T, V, 1e-2, ld=ldv), d=d_model, p=V)
+    w = torch.arange(1, V + 1, device=device, dtype=torch.float64) ** -1.1
+    ids = torch.multinomial(w / w.sum(), B * T, replacement=True, generator=g).to(torch.int32).view(B, T)
+    pos = torch.arange(T, dtype=torch.int32, device=device).repeat(B, 1).contiguous() if positions else None
+    ds = DeviceStep(
+        B=B, T=T, V=V, C=C, sigma=sigma, tied=tied, positions=positions, linears=linears, lm=lm,
+        ids=ids, pos_ids=pos, G_emb=normal(T, d_model, 1e-2), d_model=d_model,
+        sq=torch.zeros(B, dtype=torch.float32, device=device),
+        clip=torch.zeros(B, dtype=torch.float32, device=device),
+        norms=torch.zeros(B, dtype=torch.float32, device=device),
+        cross=torch.zeros(B, dtype=torch.float32, device=device) if tied else None,
         dev_status=torch.zeros(1, dtype=torch.int32, device=device))
     allocate(ds)
     return ds

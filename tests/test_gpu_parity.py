@@ -455,6 +455,20 @@ def test_overlapped_step_untied_with_positions_matches_unfused():
         assert torch.allclose(a.outs[k], b.outs[k], rtol=1e-5, atol=2e-6), k
 
 
+def test_noise_fp32_path_error_bound_exhaustive():
+    """The fp32 Box-Muller path is used up to r^2 = threshold; beyond it float64 takes over.  An
+    exhaustive device scan of both fp32 factors against float64 (all 2^24 inputs each) must keep
+    the worst-case error of z = r * cos/sin below the 1e-6 tolerance at that threshold."""
+    L = dp.load()
+    out = torch.zeros(4, dtype=torch.float64, device=dev())
+    assert L.dp_debug_noise_error_scan(0.0, out.data_ptr(), None) == 0
+    torch.cuda.synchronize()
+    err_r, err_dir, r_max, thr = out.tolist()
+    assert 3.3 ** 2 <= thr <= 34.0 and r_max <= thr ** 0.5 + 1e-6
+    bound = (err_r + err_dir + 2.0 ** -24) * r_max          # relative r, absolute direction, product rounding
+    assert bound < 1e-6, (err_r, err_dir, r_max, bound)
+
+
 # ---------------------------------------------------------------------------- error paths
 def test_argument_errors_are_reported_before_any_launch():
     B, T, d, p = 2, 16, 64, 64
