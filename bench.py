@@ -378,7 +378,7 @@ def run_ours(args):
     # CPU baseline: the oracle on a bounded sample, on this machine's host cores (rank 0, N=1 only)
     cpu = None
     if world == 1 and not args.no_cpu_baseline and not args.device_inputs:
-        n_ex = 4
+        n_ex = min(w.B, 16)
         t_ex = oracle_sample_step(w, n_ex)
         n_noise = 4_000_000
         t_noise = oracle_noise_seconds(n_noise)
