@@ -352,9 +352,9 @@ dp_status dp_clip_accumulate(const void* A, int64_t lda, const void* G, int64_t 
 }
 
 // ------------------------------------------------------------------ clip accumulate, embedding
-static void embed_ws_layout(int B, int T, int V, size_t* off_clip, size_t* off_counts,
-                            size_t* off_seg, size_t* off_perm, size_t* off_blk, size_t* total,
-                            int* chunks) {
+static void embed_ws_layout(int B, int T, int d, int V, size_t* off_clip, size_t* off_counts,
+                            size_t* off_seg, size_t* off_perm, size_t* off_blk, size_t* off_part,
+                            size_t* total, int* chunks) {
   const size_t n = size_t(B) * T;
   *chunks = int((n + kSortChunk - 1) / kSortChunk);
   size_t o = 0;
@@ -363,14 +363,14 @@ static void embed_ws_layout(int B, int T, int V, size_t* off_clip, size_t* off_c
   *off_seg = o;    o += align_up(size_t(V + 1) * sizeof(int), 256);
   *off_perm = o;   o += align_up(n * sizeof(int), 256);
   *off_blk = o;    o += align_up(size_t(ceil_div(V, 1024)) * sizeof(int), 256);
+  *off_part = o;   o += embed_scatter_partial_bytes((long long)n, d);
   *total = o;
 }
 
 size_t dp_clip_accumulate_embed_ws_bytes(int32_t B, int32_t T, int32_t d, int32_t V) {
-  (void)d;
-  if (B <= 0 || T <= 0 || V <= 0) return 0;
-  size_t a, b, c, e, f, total; int chunks;
-  embed_ws_layout(B, T, V, &a, &b, &c, &e, &f, &total, &chunks);
+  if (B <= 0 || T <= 0 || V <= 0 || d <= 0) return 0;
+  size_t a, b, c, e, f, g, total; int chunks;
+  embed_ws_layout(B, T, d, V, &a, &b, &c, &e, &f, &g, &total, &chunks);
   return total;
 }
 
@@ -387,8 +387,8 @@ static dp_status clip_accumulate_embed_impl(const int32_t* ids, const void* G, i
   if (dt != DP_F32 && dt != DP_BF16) return DP_ERR_INVALID_ARG;
   if (!(beta == 0.f || beta == 1.f) || !finite_pos(C)) return DP_ERR_INVALID_ARG;
   if ((long long)B * T > 0x7fffffffLL) return DP_ERR_UNSUPPORTED;
-  size_t o_clip, o_counts, o_seg, o_perm, o_blk, total; int chunks;
-  embed_ws_layout(B, T, V, &o_clip, &o_counts, &o_seg, &o_perm, &o_blk, &total, &chunks);
+  size_t o_clip, o_counts, o_seg, o_perm, o_blk, o_part, total; int chunks;
+  embed_ws_layout(B, T, d, V, &o_clip, &o_counts, &o_seg, &o_perm, &o_blk, &o_part, &total, &chunks);
   if (!ws || ws_bytes < total) return DP_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   char* w = static_cast<char*>(ws);
@@ -424,7 +424,7 @@ static dp_status clip_accumulate_embed_impl(const int32_t* ids, const void* G, i
     }
   }
   return launch_embed_scatter(ids, G, ldg, dt, n, T, d, V, clip_ws, sw.perm, sw.seg, out, ldo, beta,
-                              scale, clear, st);
+                              scale, clear, reinterpret_cast<float*>(w + o_part), st);
 }
 
 dp_status dp_clip_accumulate_embed(const int32_t* ids, const void* G, int64_t ldg, dp_dtype dt,

@@ -62,10 +62,11 @@ __global__ void __launch_bounds__(kEmbedNormThreads)
 embed_norm_kernel(const int* __restrict__ ids, const T* __restrict__ G, long long ldg, int Tn, int d,
                   int V, int slabs, float* __restrict__ partials, int* __restrict__ first_occ,
                   int* __restrict__ dev_status) {
-  extern __shared__ int sm_i[];
+  extern __shared__ __align__(16) int sm_i[];
+  const int Tp = (Tn + 3) & ~3;  // padded so that every array starts on a 16-byte boundary
   int* s_id = sm_i;              // token id, -1 if out of range
-  int* s_fo = sm_i + Tn;         // first occurrence
-  int* s_ord = sm_i + 2 * Tn;    // rows ordered by (first occurrence, position); sign bit = group end
+  int* s_fo = sm_i + Tp;         // first occurrence
+  int* s_ord = sm_i + 2 * Tp;    // rows ordered by (first occurrence, position); sign bit = group end
   __shared__ float red[32];
   const int i = blockIdx.x / slabs, slab = blockIdx.x % slabs;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -81,21 +82,32 @@ embed_norm_kernel(const int* __restrict__ ids, const T* __restrict__ G, long lon
   }
   __syncthreads();
 
-  // first occurrence: match inside the warp's 32-token window, leaders scan earlier windows
+  // First occurrence and position in the grouped order.  Tokens are ordered by (first
+  // occurrence, position); a token's rank is the number of tokens ordered before it.  Inside
+  // the warp's own 32-token window the ids are matched with __match_any_sync (the peers with a
+  // lower lane come first); all windows are then walked once through shared memory, four ids
+  // per 128-bit load, updating the earliest equal id and nothing else -- the rank needs the
+  // first occurrences of ALL tokens, so it is taken in a second, equally short walk.
   const int t_round = (Tn + 31) & ~31;
+  const int Tn4 = Tn & ~3;
   for (int t = threadIdx.x; t < t_round; t += blockDim.x) {
     const bool live = t < Tn;
     const int id = live ? s_id[t] : -2 - lane;             // unique sentinel for padding lanes
     const int key = (id == -1) ? -2 - 64 - lane : id;      // bad ids never match anything
     const unsigned peers = __match_any_sync(0xffffffffu, key);
-    const int leader = __ffs(peers) - 1;
     const int base = t - lane;
-    int fo = base + leader;
-    if (lane == leader && live && id >= 0) {
-      for (int s = 0; s < base; ++s)
-        if (s_id[s] == id) { fo = s; break; }
+    int fo = base + (__ffs(peers) - 1);                    // earliest equal id in this window
+    if (live && id >= 0) {
+      const int4* v4 = reinterpret_cast<const int4*>(s_id);
+      for (int s4 = 0; s4 < (base >> 2); ++s4) {           // windows before this one
+        const int4 q = v4[s4];
+        const int s = s4 << 2;
+        if (q.w == id) fo = min(fo, s + 3);
+        if (q.z == id) fo = min(fo, s + 2);
+        if (q.y == id) fo = min(fo, s + 1);
+        if (q.x == id) fo = min(fo, s);
+      }
     }
-    fo = __shfl_sync(0xffffffffu, fo, leader);
     if (live) s_fo[t] = (id >= 0) ? fo : t;
   }
   __syncthreads();
@@ -104,7 +116,16 @@ embed_norm_kernel(const int* __restrict__ ids, const T* __restrict__ G, long lon
   for (int t = threadIdx.x; t < Tn; t += blockDim.x) {
     const int fo = s_fo[t];
     int rank = 0;
-    for (int s = 0; s < Tn; ++s) {
+    const int4* f4 = reinterpret_cast<const int4*>(s_fo);
+    for (int s4 = 0; s4 < (Tn4 >> 2); ++s4) {
+      const int4 q = f4[s4];
+      const int s = s4 << 2;
+      rank += (q.x < fo) || (q.x == fo && s < t);
+      rank += (q.y < fo) || (q.y == fo && s + 1 < t);
+      rank += (q.z < fo) || (q.z == fo && s + 2 < t);
+      rank += (q.w < fo) || (q.w == fo && s + 3 < t);
+    }
+    for (int s = Tn4; s < Tn; ++s) {
       const int f = s_fo[s];
       rank += (f < fo) || (f == fo && s < t);
     }
@@ -271,49 +292,69 @@ sort_place_kernel(const int* __restrict__ ids, int n, int V, const int* __restri
 }
 
 // ------------------------------------------------------------------ segmented row sum
-// grid = (64-position chunks of the sorted order, 256-column slabs).  A block finds the segment
-// heads (first sorted position of a token id) inside its chunk and sums each head's rows:
-//   * short segments (<= 32 rows): one warp per segment, lanes own 8 columns, rows are added in
-//     sorted order with 8 row loads in flight;
-//   * long segments (a frequent token): the whole block, rows staged 64 at a time, warp w taking
-//     rows w, w+8, ... of each stage, the 8 per-warp sums combined in warp order.
-// Both orders are fixed, so the result does not depend on timing (no floating-point atomics).
-constexpr int kScatChunk = 64;
-constexpr int kScatShort = 32;
+// The sorted order is cut into 32-position chunks; grid = (chunks, 256-column slabs).
+//   pass 1 (embed_scatter_kernel): a block finds the segments (runs of one token id) that meet
+//     its chunk.  Short segments (<= 32 rows) are summed by one warp each, from their head, in
+//     sorted order, and written to the table.  Rows of LONG segments (a frequent token) are
+//     summed per chunk by the whole block -- warp w takes rows w, w+8, ... and the eight warp
+//     sums are added in warp order -- into a partial buffer [chunk][slot][column]; slot 0 is the
+//     segment that continues from the previous chunk, slot 1 the one that starts in this chunk
+//     (a 32-position chunk can meet at most one of each).
+//   pass 2 (embed_scatter_combine_kernel): the block whose chunk holds a long segment's head
+//     adds that segment's partials in chunk order and writes the table row.
+// Every order is fixed, so the result does not depend on timing (no floating-point atomics),
+// and a very frequent token is spread over as many blocks as it has chunks.
+constexpr int kScatChunk = 32;     // sorted positions per block
+constexpr int kScatShort = 32;     // longest segment handled by a single warp
+constexpr int kScatBatch = 4;      // row loads in flight per lane
 
 template <typename T>
 __global__ void __launch_bounds__(256)
 embed_scatter_kernel(const int* __restrict__ ids, const T* __restrict__ G, long long ldg, int Tn,
                      int d, const float* __restrict__ clip, const int* __restrict__ perm,
                      const int* __restrict__ seg, int V, float* __restrict__ out, long long ldo,
-                     float beta, float scale) {
+                     float beta, float scale, float* __restrict__ long_part) {
   __shared__ float part[8][kEmbedColsPerBlock];
-  __shared__ int s_pos[kScatChunk];
-  __shared__ float s_r[kScatChunk];
+  __shared__ int s_pos[kScatChunk + kScatShort];
+  __shared__ float s_r[kScatChunk + kScatShort];
   __shared__ int s_hk[kScatChunk], s_hv[kScatChunk], s_hn[kScatChunk];
-  __shared__ unsigned s_mask[2];
+  __shared__ unsigned s_mask, s_long0, s_long1;
   const int n_valid = seg[V];
   const int kc = blockIdx.x * kScatChunk;
   if (kc >= n_valid) return;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
 
-  // ---- heads of this chunk
+  // ---- classify the chunk's positions (warp 0) and stage positions / clip factors of the
+  //      chunk and of the kScatShort rows after it (threads 0..63)
   int my_v = -1, my_n = 0;
   bool head = false;
   if (threadIdx.x < kScatChunk) {
     const int k = kc + threadIdx.x;
+    int s0 = 0;
     if (k < n_valid) {
       my_v = ids[perm[k]];
-      head = (k == 0) || (ids[perm[k - 1]] != my_v);
-      if (head) my_n = seg[my_v + 1] - k;
+      s0 = seg[my_v];
+      my_n = seg[my_v + 1] - s0;
+      head = (s0 == k);
     }
+    const bool is_long = my_n > kScatShort;
     const unsigned m = __ballot_sync(0xffffffffu, head);
-    if (lane == 0) s_mask[w] = m;
+    const unsigned l0 = __ballot_sync(0xffffffffu, is_long && s0 < kc);     // continues from before
+    const unsigned l1 = __ballot_sync(0xffffffffu, is_long && s0 >= kc);    // starts in this chunk
+    if (lane == 0) { s_mask = m; s_long0 = l0; s_long1 = l1; }
+  }
+  if (threadIdx.x < kScatChunk + kScatShort) {
+    const int k = kc + threadIdx.x;
+    if (k < n_valid) {
+      const int pos = perm[k];
+      s_pos[threadIdx.x] = pos;
+      s_r[threadIdx.x] = clip[pos / Tn];
+    }
   }
   __syncthreads();
-  const int n_heads = __popc(s_mask[0]) + __popc(s_mask[1]);
+  const int n_heads = __popc(s_mask);
   if (threadIdx.x < kScatChunk && head) {
-    const int slot = (w == 1 ? __popc(s_mask[0]) : 0) + __popc(s_mask[w] & ((1u << lane) - 1u));
+    const int slot = __popc(s_mask & ((1u << lane) - 1u));
     s_hk[slot] = kc + threadIdx.x;
     s_hv[slot] = my_v;
     s_hn[slot] = my_n;
@@ -325,23 +366,22 @@ embed_scatter_kernel(const int* __restrict__ ids, const T* __restrict__ G, long 
   const bool vec = ((reinterpret_cast<uintptr_t>(G) & 15) == 0) && ((ldg * sizeof(T)) % 16 == 0);
   const bool ovec = ((reinterpret_cast<uintptr_t>(out) & 15) == 0) && ((ldo & 3) == 0);
 
-  // ---- short segments: one warp each
+  // ---- short segments: one warp each, rows in sorted order
   for (int h = w; h < n_heads; h += 8) {
     const int n = s_hn[h];
     if (n > kScatShort || nvalid <= 0) continue;
-    const int k0 = s_hk[h], v = s_hv[h];
+    const int o0 = s_hk[h] - kc, v = s_hv[h];          // rows o0 .. o0+n-1 of the staged window
     float acc[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-    for (int b0 = 0; b0 < n; b0 += 8) {
-      float vals[8][8];
-      float r[8];
+    for (int b0 = 0; b0 < n; b0 += kScatBatch) {
+      float vals[kScatBatch][8];
+      float r[kScatBatch];
 #pragma unroll
-      for (int b = 0; b < 8; ++b) {
+      for (int b = 0; b < kScatBatch; ++b) {
         if (b0 + b < n) {
-          const int pos = perm[k0 + b0 + b];
-          r[b] = clip[pos / Tn];
-          load8<T>(G + size_t(pos) * ldg + c, nvalid, vec, vals[b]);
+          r[b] = s_r[o0 + b0 + b];
+          load8<T>(G + size_t(s_pos[o0 + b0 + b]) * ldg + c, nvalid, vec, vals[b]);
         } else {
           r[b] = 0.f;
 #pragma unroll
@@ -349,7 +389,7 @@ embed_scatter_kernel(const int* __restrict__ ids, const T* __restrict__ G, long 
         }
       }
 #pragma unroll
-      for (int b = 0; b < 8; ++b)
+      for (int b = 0; b < kScatBatch; ++b)
 #pragma unroll
         for (int e = 0; e < 8; ++e) acc[e] = fmaf(r[b], vals[b][e], acc[e]);
     }
@@ -369,43 +409,34 @@ embed_scatter_kernel(const int* __restrict__ ids, const T* __restrict__ G, long 
     }
   }
 
-  // ---- long segments: the whole block, one after another
-  for (int h = 0; h < n_heads; ++h) {
-    const int n = s_hn[h];
-    if (n <= kScatShort) continue;
-    const int k0 = s_hk[h], v = s_hv[h];
+  // ---- rows of long segments inside this chunk: per-chunk partial sums
+#pragma unroll 1
+  for (int slot = 0; slot < 2; ++slot) {
+    const unsigned m = slot == 0 ? s_long0 : s_long1;
+    if (m == 0u) continue;                               // uniform over the block
+    const int a = __ffs(m) - 1, b = 32 - __clz(m);       // the rows form one run [a, b)
     float acc[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-    for (int base = 0; base < n; base += kScatChunk) {
-      const int m = min(kScatChunk, n - base);
-      __syncthreads();
-      if (threadIdx.x < m) {
-        const int pos = perm[k0 + base + threadIdx.x];
-        s_pos[threadIdx.x] = pos;
-        s_r[threadIdx.x] = clip[pos / Tn];
-      }
-      __syncthreads();
-      if (nvalid > 0) {
-        float vals[kScatChunk / 8][8];
+    if (nvalid > 0) {
+      float vals[kScatBatch][8];
 #pragma unroll
-        for (int b = 0; b < kScatChunk / 8; ++b) {
-          const int k = w + 8 * b;
-          if (k < m) {
-            load8<T>(G + size_t(s_pos[k]) * ldg + c, nvalid, vec, vals[b]);
-          } else {
+      for (int j = 0; j < kScatBatch; ++j) {
+        const int k = a + w + 8 * j;
+        if (k < b) {
+          load8<T>(G + size_t(s_pos[k]) * ldg + c, nvalid, vec, vals[j]);
+        } else {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) vals[b][e] = 0.f;
-          }
+          for (int e = 0; e < 8; ++e) vals[j][e] = 0.f;
         }
+      }
 #pragma unroll
-        for (int b = 0; b < kScatChunk / 8; ++b) {
-          const int k = w + 8 * b;
-          if (k < m) {
-            const float r = s_r[k];
+      for (int j = 0; j < kScatBatch; ++j) {
+        const int k = a + w + 8 * j;
+        if (k < b) {
+          const float r = s_r[k];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] = fmaf(r, vals[b][e], acc[e]);
-          }
+          for (int e = 0; e < 8; ++e) acc[e] = fmaf(r, vals[j][e], acc[e]);
         }
       }
     }
@@ -417,12 +448,49 @@ embed_scatter_kernel(const int* __restrict__ ids, const T* __restrict__ G, long 
       float sum = 0.f;
 #pragma unroll
       for (int ww = 0; ww < 8; ++ww) sum += part[ww][threadIdx.x];
-      float* o = out + size_t(v) * ldo + cc;
-      sum *= scale;
-      *o = (beta != 0.f) ? (*o + sum) : sum;
+      long_part[(size_t(blockIdx.x) * 2 + slot) * d + cc] = sum;
     }
     __syncthreads();
   }
+}
+
+// pass 2: table row of every long segment = beta*row + scale * (its partials in chunk order)
+__global__ void __launch_bounds__(256)
+embed_scatter_combine_kernel(const int* __restrict__ ids, const int* __restrict__ perm,
+                             const int* __restrict__ seg, int V, int d,
+                             const float* __restrict__ long_part, float* __restrict__ out,
+                             long long ldo, float beta, float scale) {
+  __shared__ int s_v, s_k0, s_n;
+  const int n_valid = seg[V];
+  const int kc = blockIdx.x * kScatChunk;
+  if (kc >= n_valid) return;
+  if (threadIdx.x < 32) {                                // at most one long head per chunk
+    const int k = kc + threadIdx.x;
+    int v = -1, n = 0;
+    bool long_head = false;
+    if (k < n_valid) {
+      v = ids[perm[k]];
+      const int s0 = seg[v];
+      n = seg[v + 1] - s0;
+      long_head = (s0 == k) && (n > kScatShort);
+    }
+    const unsigned m = __ballot_sync(0xffffffffu, long_head);
+    if (threadIdx.x == 0) s_n = 0;
+    __syncwarp();
+    if (long_head) { s_v = v; s_k0 = k; s_n = n; }
+    (void)m;
+  }
+  __syncthreads();
+  const int n = s_n;
+  if (n == 0) return;
+  const int cc = blockIdx.y * kEmbedColsPerBlock + threadIdx.x;
+  if (cc >= d) return;
+  const int c0 = blockIdx.x, c1 = (s_k0 + n - 1) / kScatChunk;
+  float sum = long_part[(size_t(c0) * 2 + 1) * d + cc];            // starts in its own chunk
+  for (int cch = c0 + 1; cch <= c1; ++cch) sum += long_part[(size_t(cch) * 2 + 0) * d + cc];
+  float* o = out + size_t(s_v) * ldo + cc;
+  sum *= scale;
+  *o = (beta != 0.f) ? (*o + sum) : sum;
 }
 
 }  // namespace
@@ -431,7 +499,7 @@ dp_status launch_embed_norms(const int* ids, const void* G, int64_t ldg, dp_dtyp
                              int d, int V, float* partials, int* first_occ, int* dev_status,
                              cudaStream_t st) {
   const int slabs = ceil_div(d, kEmbedColsPerBlock);
-  const size_t smem = size_t(3) * T * sizeof(int);
+  const size_t smem = size_t(3) * ((T + 3) & ~3) * sizeof(int);
   static bool attr = false;
   if (!attr) {
     DP_CUDA_OK(cudaFuncSetAttribute(embed_norm_kernel<float>,
@@ -467,10 +535,14 @@ dp_status launch_embed_sort(const int* ids, int n, int V, const EmbedSortWs& ws,
   return DP_OK;
 }
 
+size_t embed_scatter_partial_bytes(long long n, int d) {
+  return align_up(size_t((n + kScatChunk - 1) / kScatChunk) * 2 * size_t(d) * sizeof(float), 256);
+}
+
 dp_status launch_embed_scatter(const int* ids, const void* G, int64_t ldg, dp_dtype dt, int n,
                                int T, int d, int V, const float* clip, const int* perm,
                                const int* seg, float* out, int64_t ldo, float beta, float scale,
-                               bool clear, cudaStream_t st) {
+                               bool clear, float* long_part, cudaStream_t st) {
   // beta == 0: the table is cleared once (unless the caller already filled it, e.g. with
   // noise), then every touched row receives table + scale*sum
   if (beta == 0.f && clear) {
@@ -480,11 +552,14 @@ dp_status launch_embed_scatter(const int* ids, const void* G, int64_t ldg, dp_dt
   dim3 grid(ceil_div(n, kScatChunk), ceil_div(d, kEmbedColsPerBlock));
   if (dt == DP_F32)
     embed_scatter_kernel<float><<<grid, 256, 0, st>>>(ids, (const float*)G, ldg, T, d, clip, perm,
-                                                     seg, V, out, ldo, 1.f, scale);
+                                                     seg, V, out, ldo, 1.f, scale, long_part);
   else
     embed_scatter_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(ids, (const __nv_bfloat16*)G, ldg, T,
                                                              d, clip, perm, seg, V, out, ldo, 1.f,
-                                                             scale);
+                                                             scale, long_part);
+  DP_LAUNCH_OK();
+  embed_scatter_combine_kernel<<<grid, 256, 0, st>>>(ids, perm, seg, V, d, long_part, out, ldo, 1.f,
+                                                     scale);
   DP_LAUNCH_OK();
   return DP_OK;
 }

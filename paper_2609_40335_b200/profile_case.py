@@ -108,8 +108,8 @@ def case_noise(reps):
         dp.dp_add_noise(x, 0.8, 1.0, 1.0, 1234, 0, k)
 
 
-def case_embed(reps):
-    B, T, d, V = 256, 512, 1024, 50257
+def case_embed(reps, B=256, T=512, d=1024):
+    V = 50257
     w = torch.arange(1, V + 1, device="cuda", dtype=torch.float64) ** -1.1
     ids = torch.multinomial(w / w.sum(), B * T, replacement=True).to(torch.int32).view(B, T)
     G = _randn_bf16(B, T, d, std=1e-2)
@@ -118,6 +118,10 @@ def case_embed(reps):
     for _ in range(reps):
         dp.dp_embed_norms(ids, G, V, sq)
         dp.dp_clip_accumulate_embed(ids, G, V, sq, 1.0, out)
+
+
+def case_embed_small(reps):
+    case_embed(reps, B=32, T=128, d=768)
 
 
 def case_cross(reps):
@@ -134,7 +138,7 @@ def main():
     which = sys.argv[1] if len(sys.argv) > 1 else "gemm"
     reps = int(sys.argv[2]) if len(sys.argv) > 2 else 3
     torch.manual_seed(0)
-    {"gemm": case_gemm, "gemm1": case_gemm_unclipped, "ghost512": case_ghost_long, "overlap": case_overlap, "ghost": case_ghost, "noise": case_noise, "embed": case_embed,
+    {"gemm": case_gemm, "gemm1": case_gemm_unclipped, "ghost512": case_ghost_long, "overlap": case_overlap, "ghost": case_ghost, "noise": case_noise, "embed": case_embed, "embed_small": case_embed_small,
      "cross": case_cross}[which](reps)
     torch.cuda.synchronize()
     print("done", which, reps)
