@@ -28,6 +28,7 @@ import numpy as np
 __all__ = [
     "linear_example_grad", "linear_sq_norms", "embed_example_grad", "embed_sq_norms",
     "tied_sq_norms", "clip_factors", "clipped_sum_linear", "clipped_sum_embed",
+    "vector_example_grad", "vector_sq_norms", "clipped_sum_vector",
     "first_occurrence", "stable_token_sort", "dp_step",
 ]
 
@@ -81,6 +82,40 @@ def embed_sq_norms(ids, G, V):
         E = embed_example_grad(ids[i], G[i], V)
         out[i] = np.sum(E * E)
     return out
+
+
+# ------------------------------------------------- vector parameters (bias, LayerNorm)
+def vector_example_grad(G_i, X_i=None):
+    """Per-example gradient of a parameter that acts element-wise along the feature axis.
+
+    A bias b in z = W a + b receives delta_t per token (Eq. 4 with a constant input 1), so the
+    example's gradient is sum_t G_i[t, :].  A LayerNorm gain gamma in y = gamma * xhat + beta
+    receives sum_t G_i[t, :] * xhat_i[t, :] (G = gradient w.r.t. y); its beta is a bias.
+    G_i: (T, p); X_i: (T, p) multiplier or None -> (p,).
+    """
+    G_i = _f64(G_i)
+    out = np.zeros(G_i.shape[1], dtype=np.float64)
+    for t in range(G_i.shape[0]):
+        out += G_i[t] if X_i is None else G_i[t] * _f64(X_i[t])
+    return out
+
+
+def vector_sq_norms(G, X=None):
+    """(B,) squared norms of the materialised per-example vector gradients."""
+    B = G.shape[0]
+    out = np.zeros(B, dtype=np.float64)
+    for i in range(B):
+        v = vector_example_grad(G[i], None if X is None else X[i])
+        out[i] = np.sum(v * v)
+    return out
+
+
+def clipped_sum_vector(G, X, R):
+    """sum_i R_i g_i for a vector parameter, (p,)."""
+    acc = np.zeros(G.shape[2], dtype=np.float64)
+    for i in range(G.shape[0]):
+        acc += float(R[i]) * vector_example_grad(G[i], None if X is None else X[i])
+    return acc
 
 
 # ----------------------------------------------------------------------------- tied
@@ -179,7 +214,7 @@ def stable_token_sort(ids, V):
 
 # ------------------------------------------------------------------------ whole step
 def dp_step(linears, ids, G_emb, V, C, lm=None, tied=False, positions=False,
-            want_sums=True):
+            want_sums=True, vectors=()):
     """One DP-SGD clipping step over the parameter blocks it is handed.
 
     linears: list of (A, G) with A (B,T,d), G (B,T,p): the block linear layers.
@@ -188,6 +223,8 @@ def dp_step(linears, ids, G_emb, V, C, lm=None, tied=False, positions=False,
     embedding matrix (Eq. 8); then the embedding and head contributions enter
     through ||g_in + g_out||^2 (Eq. 13) and their clipped sums share one matrix.
     positions: also treat a learned position table (row t receives G_emb[i, t]).
+    vectors: list of (G, X or None): biases and LayerNorm gains / shifts (see
+    vector_example_grad); their clipped sums are returned as 'vector<k>'.
 
     Squared norms add over disjoint parameter blocks (Eq. 6, Eq. 10).
     Returns dict with 'sq', 'norms', 'clip', and (if want_sums) 'sums': a dict
@@ -198,6 +235,8 @@ def dp_step(linears, ids, G_emb, V, C, lm=None, tied=False, positions=False,
     sq = np.zeros(B, dtype=np.float64)
     for (A, G) in linears:
         sq += linear_sq_norms(A, G)
+    for (G, X) in vectors:
+        sq += vector_sq_norms(G, X)
     pos_ids = np.broadcast_to(np.arange(T), (B, T))
     if positions:
         sq += embed_sq_norms(pos_ids, G_emb, T)
@@ -217,6 +256,8 @@ def dp_step(linears, ids, G_emb, V, C, lm=None, tied=False, positions=False,
         sums = {}
         for k, (A, G) in enumerate(linears):
             sums[f"linear{k}"] = clipped_sum_linear(A, G, R)
+        for k, (G, X) in enumerate(vectors):
+            sums[f"vector{k}"] = clipped_sum_vector(G, X, R)
         if positions:
             sums["wpe"] = clipped_sum_embed(pos_ids, G_emb, R, T)
         wte = clipped_sum_embed(ids, G_emb, R, V)

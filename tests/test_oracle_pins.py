@@ -282,3 +282,84 @@ def test_workload_shapes_reproduce_table1_counts():
         if tied == "0":
             n += GPT2_VOCAB * d
         assert n == int(count), (model, tied)
+
+
+# ------------------------------------------- vector parameters: biases and LayerNorm
+class TinyFull(torch.nn.Module):
+    """wte -> LayerNorm -> linear1 (+bias) -> tanh -> linear2 (+bias) -> untied head (no bias)."""
+
+    def __init__(self, V, d, h):
+        super().__init__()
+        g = torch.Generator().manual_seed(11)
+        mk = lambda *s: torch.nn.Parameter(torch.randn(*s, generator=g, dtype=torch.float64) * 0.5)
+        self.wte, self.gamma, self.beta = mk(V, d), mk(d), mk(d)
+        self.w1, self.b1, self.w2, self.b2, self.head = mk(h, d), mk(h), mk(d, h), mk(d), mk(V, d)
+
+    def forward(self, ids, keep):
+        h0 = self.wte[ids]
+        keep["h0"] = h0
+        mu = h0.mean(-1, keepdim=True)
+        var = ((h0 - mu) ** 2).mean(-1, keepdim=True)
+        xhat = (h0 - mu) / torch.sqrt(var + 1e-5)
+        keep["xhat"] = xhat
+        y = self.gamma * xhat + self.beta
+        keep["y"] = y
+        z1 = y @ self.w1.T + self.b1
+        keep["z1"] = z1
+        a1 = torch.tanh(z1)
+        keep["a1"] = a1
+        z2 = a1 @ self.w2.T + self.b2
+        keep["z2"] = z2
+        logits = z2 @ self.head.T
+        keep["logits"] = logits
+        return logits
+
+
+def test_oracle_vector_parameters_match_per_example_autograd():
+    V, d, h, T, B = 9, 6, 5, 7, 4
+    model = TinyFull(V, d, h)
+    g = torch.Generator().manual_seed(4)
+    ids = torch.randint(0, V, (B, T), generator=g)
+    labels = torch.randint(0, V, (B, T), generator=g)
+    params = list(model.parameters())
+    names = [n for n, _ in model.named_parameters()]
+
+    def losses(idx, keep):
+        logits = model(ids[idx], keep)
+        n = logits.shape[0]
+        return torch.nn.functional.cross_entropy(logits.reshape(n * T, V), labels[idx].reshape(-1),
+                                                 reduction="none").reshape(n, T).sum(1)
+
+    per_ex = [torch.autograd.grad(losses(slice(i, i + 1), {})[0], params) for i in range(B)]
+    sq_true = np.array([sum(float((x ** 2).sum()) for x in gs) for gs in per_ex])
+    keep = {}
+    total = losses(slice(0, B), keep).sum()
+    G_h0, G_y, G_z1, G_z2, G_log = torch.autograd.grad(
+        total, [keep["h0"], keep["y"], keep["z1"], keep["z2"], keep["logits"]])
+    npy = lambda t: t.detach().numpy()
+    linears = [(npy(keep["y"]), npy(G_z1)), (npy(keep["a1"]), npy(G_z2))]
+    vectors = [(npy(G_y), npy(keep["xhat"])), (npy(G_y), None), (npy(G_z1), None), (npy(G_z2), None)]
+    Cc = float(np.median(np.sqrt(sq_true)))
+    res = O.dp_step(linears, ids.numpy(), npy(G_h0), V, Cc, lm=(npy(keep["z2"]), npy(G_log)),
+                    vectors=vectors)
+    np.testing.assert_allclose(res["sq"], sq_true, rtol=1e-10)
+    R = np.minimum(1.0, Cc / np.sqrt(sq_true))
+    want = {n: sum(R[i] * per_ex[i][k].numpy() for i in range(B)) for k, n in enumerate(names)}
+    for key, name in [("vector0", "gamma"), ("vector1", "beta"), ("vector2", "b1"), ("vector3", "b2"),
+                      ("linear0", "w1"), ("linear1", "w2"), ("lm_head", "head"), ("wte", "wte")]:
+        np.testing.assert_allclose(res["sums"][key], want[name], rtol=1e-9, atol=1e-12)
+
+
+def test_vector_gradient_special_cases():
+    B, T, p = 3, 5, 4
+    G, X = RNG.standard_normal((B, T, p)), RNG.standard_normal((B, T, p))
+    np.testing.assert_allclose(O.vector_sq_norms(G), (G.sum(1) ** 2).sum(1), rtol=1e-12)
+    np.testing.assert_allclose(O.vector_sq_norms(G, X), ((G * X).sum(1) ** 2).sum(1), rtol=1e-12)
+    np.testing.assert_allclose(O.vector_sq_norms(G, np.ones_like(G)), O.vector_sq_norms(G), rtol=1e-12)
+    # a bias is a linear layer whose input is the constant 1 (Eq. 4 with a_t = 1)
+    ones = np.ones((B, T, 1))
+    np.testing.assert_allclose(O.vector_sq_norms(G), O.linear_sq_norms(ones, G), rtol=1e-12)
+    R = np.array([0.5, 1.0, 0.25])
+    np.testing.assert_allclose(O.clipped_sum_vector(G, X, R), np.einsum("i,itp,itp->p", R, G, X), rtol=1e-12)
+    np.testing.assert_allclose(O.clipped_sum_vector(G, None, R),
+                               O.clipped_sum_linear(ones, G, R)[:, 0], rtol=1e-12)
