@@ -114,9 +114,9 @@ def work_counts(w):
                 embed_bytes=embed_bytes)
 
 
-def make_workload(name, seed=0, B=None, T=None):
+def make_workload(name, seed=0, B=None, T=None, full_model=False):
     from paper_2609_40335_b200 import workloads
-    over = {}
+    over = {"full_model": True} if full_model else {}
     if B:
         over["B"] = B
     if T:
@@ -204,7 +204,7 @@ def run_ours(args):
             linears=[types.SimpleNamespace(d=l.d, p=l.p) for l in ds.linears],
             lm=types.SimpleNamespace(d=ds.lm.d, p=ds.lm.p))
     else:
-        w = make_workload(args.workload, seed=rank, B=args.B, T=args.T)
+        w = make_workload(args.workload, seed=rank, B=args.B, T=args.T, full_model=args.full_model)
         ds = P.upload(w, dev)
     counts = work_counts(w)
     stream = torch.cuda.current_stream()
@@ -395,6 +395,7 @@ def run_ours(args):
         "vs_baseline": None, "dtype": w.dtype if w.dtype != "f32" else "f32", "data": "synthetic",
         "config": {"workload": w.name, "B_per_gpu": w.B, "T": w.T, "V": w.V, "layers": len(w.linears),
                    "lm_head": bool(w.lm), "tied": w.tied, "positions": w.positions,
+                   "bias_and_layernorm_params": len(getattr(w, "vectors", []) or []),
                    "accumulate": "fp32", "input_bytes_per_step": ds.input_bytes(),
                    "l2": "inputs (%.2f GB per step) are larger than the 126 MB L2" % (ds.input_bytes() / 1e9)},
         "phases_ms": {"norms": ms_norm, "clip_accumulate": ms_clip, "noise": ms_noise,
@@ -423,6 +424,8 @@ def main():
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--B", type=int, default=0, help="override the workload's batch size (cfg5 sweep)")
     ap.add_argument("--T", type=int, default=0, help="override the workload's sequence length")
+    ap.add_argument("--full-model", action="store_true",
+                    help="also clip the biases and LayerNorm parameters of every block (whole GPT-2 model)")
     ap.add_argument("--device-inputs", action="store_true",
                     help="cfg5 only: draw the inputs on the device (big cells)")
     ap.add_argument("--seed", type=int, default=0)

@@ -116,6 +116,35 @@ dp_status dp_embed_norms_static(const int32_t* ids, const void* G, int64_t ldg, 
                                 int32_t B, int32_t T, int32_t d, int32_t V, float* sq,
                                 int32_t* first_occ, int32_t* dev_status, void* stream);
 
+/* ---- parameters that act element-wise along the feature axis: biases, LayerNorm ----
+ * A bias sees the back-propagated signal of every token (Eq. 4 with a constant input 1): its
+ * per-example gradient is v_i = sum_t G[i,t,:].  A LayerNorm gain has v_i = sum_t G[i,t,:] *
+ * X[i,t,:], X the normalised input and G the gradient at the LayerNorm output; its shift is a
+ * bias.  With these blocks Eq. 6 runs over every parameter of a GPT-2 model.
+ * G, X [dev, (B*T, p)], X may be NULL (bias).  Any alignment works; 16-byte aligned tensors
+ * with pitches that are multiples of 16 bytes take the vector-load path. */
+typedef struct {
+  const void* G;  int64_t ldg;
+  const void* X;  int64_t ldx;      /* NULL / 0 for a bias */
+  int32_t p;
+} dp_vector_desc;
+/* sq[i] += || v_i ||^2 for every parameter in params [host, n entries]. */
+dp_status dp_vector_norms(const dp_vector_desc* params, int32_t n, dp_dtype dt, int32_t B,
+                          int32_t T, float* sq, void* ws, size_t ws_bytes, void* stream);
+size_t dp_vector_norms_ws_bytes(const dp_vector_desc* params, int32_t n, int32_t B, int32_t T);
+/* outs[k] (p_k floats) = beta*outs[k] + sum_i R_i v_i, then, if with_noise, the Gaussian
+ * mechanism outs[k] = scale * (outs[k] + sigma*C*z) with the stream (seed, tensor_ids[k], step)
+ * of dp_add_noise.  outs, tensor_ids [host arrays, n entries; tensor_ids may be NULL without
+ * noise].  clip [dev, B or NULL] receives R. */
+dp_status dp_clip_accumulate_vectors(const dp_vector_desc* params, int32_t n, dp_dtype dt,
+                                     int32_t B, int32_t T, const float* sq, float C, float* clip,
+                                     float* const* outs, float beta, int32_t with_noise,
+                                     float sigma, float scale, uint64_t seed,
+                                     const uint32_t* tensor_ids, uint32_t step,
+                                     void* ws, size_t ws_bytes, void* stream);
+size_t dp_clip_accumulate_vectors_ws_bytes(const dp_vector_desc* params, int32_t n, int32_t B,
+                                           int32_t T);
+
 /* ---- cross term of a weight-tied embedding / LM head (Eq. 11, Eq. 13) ----
  * Adds 2*<g_in_i, g_out_i> to sq[i], with g_in_i the (V,d) embedding gradient of example i
  * and g_out_i = G_lm_i^T A_lm_i, through

@@ -34,7 +34,13 @@ class _LinearDesc(C.Structure):
                 ("mode", C.c_int32), ("mode_used", C.c_int32)]
 
 
-EXPORTS = ["dp_ghost_norms", "dp_ghost_norms_ws_bytes", "dp_embed_norms", "dp_embed_norms_ws_bytes",
+class _VectorDesc(C.Structure):
+    _fields_ = [("G", C.c_void_p), ("ldg", C.c_int64), ("X", C.c_void_p), ("ldx", C.c_int64),
+                ("p", C.c_int32)]
+
+
+EXPORTS = ["dp_vector_norms", "dp_vector_norms_ws_bytes", "dp_clip_accumulate_vectors",
+           "dp_clip_accumulate_vectors_ws_bytes", "dp_ghost_norms", "dp_ghost_norms_ws_bytes", "dp_embed_norms", "dp_embed_norms_ws_bytes",
            "dp_embed_norms_static",
            "dp_tied_cross_term", "dp_tied_cross_term_ws_bytes", "dp_clip_factors",
            "dp_clip_accumulate", "dp_clip_accumulate_ws_bytes", "dp_clip_accumulate_grouped",
@@ -62,6 +68,15 @@ def load():
     L.dp_ghost_norms_ws_bytes.argtypes = [C.POINTER(_LinearDesc), i32, i32, i32, i32]
     L.dp_ghost_norms_ws_bytes.restype = sz
     L.dp_embed_norms.argtypes = [vp, vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, sz, vp, vp]
+    VP = C.POINTER(_VectorDesc)
+    L.dp_vector_norms.argtypes = [VP, i32, i32, i32, i32, vp, vp, sz, vp]
+    L.dp_vector_norms_ws_bytes.argtypes = [VP, i32, i32, i32]
+    L.dp_vector_norms_ws_bytes.restype = sz
+    L.dp_clip_accumulate_vectors.argtypes = [VP, i32, i32, i32, i32, vp, f32, vp, C.POINTER(vp), f32, i32,
+                                             f32, f32, C.c_uint64, C.POINTER(C.c_uint32), C.c_uint32,
+                                             vp, sz, vp]
+    L.dp_clip_accumulate_vectors_ws_bytes.argtypes = [VP, i32, i32, i32]
+    L.dp_clip_accumulate_vectors_ws_bytes.restype = sz
     L.dp_embed_norms_static.argtypes = [vp, vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, vp]
     L.dp_embed_norms_ws_bytes.argtypes = [i32, i32, i32]
     L.dp_embed_norms_ws_bytes.restype = sz
@@ -213,6 +228,67 @@ def dp_embed_norms(ids: torch.Tensor, G: torch.Tensor, V: int, sq: torch.Tensor,
                           _ptr(first_occ), _ptr(ws), ws.numel() * ws.element_size(),
                           _ptr(dev_status), _stream(stream))
     _check(st, "dp_embed_norms")
+
+
+@dataclass
+class Vector:
+    """A bias / LayerNorm parameter: G (B,T,>=p) gradient at its output, X normalised input or None."""
+    G: torch.Tensor
+    X: Optional[torch.Tensor] = None
+    p: Optional[int] = None
+
+
+def _vdescs(params: Sequence[Vector]):
+    arr = (_VectorDesc * len(params))()
+    for k, v in enumerate(params):
+        arr[k].G = _ptr(v.G)
+        arr[k].ldg = _rows_ld(v.G)
+        arr[k].X = _ptr(v.X)
+        arr[k].ldx = _rows_ld(v.X) if v.X is not None else 0
+        arr[k].p = v.p if v.p is not None else v.G.shape[-1]
+    return arr
+
+
+def dp_vector_norms_ws_bytes(params: Sequence[Vector], B: int, T: int) -> int:
+    return int(load().dp_vector_norms_ws_bytes(_vdescs(params), len(params), B, T))
+
+
+def dp_clip_accumulate_vectors_ws_bytes(params: Sequence[Vector], B: int, T: int) -> int:
+    return int(load().dp_clip_accumulate_vectors_ws_bytes(_vdescs(params), len(params), B, T))
+
+
+def dp_vector_norms(params: Sequence[Vector], B: int, T: int, sq: torch.Tensor, ws=None, stream=None):
+    """sq[i] += ||sum_t G[i,t]*X[i,t]||^2 for every bias / LayerNorm parameter."""
+    L = load()
+    arr = _vdescs(params)
+    need = int(L.dp_vector_norms_ws_bytes(arr, len(params), B, T))
+    ws = _ws(need, ws, sq.device)
+    st = L.dp_vector_norms(arr, len(params), _dt(params[0].G), B, T, _ptr(sq), _ptr(ws),
+                           ws.numel() * ws.element_size(), _stream(stream))
+    _check(st, "dp_vector_norms")
+
+
+def dp_clip_accumulate_vectors(params: Sequence[Vector], B: int, T: int, sq, C_: float,
+                               outs: Sequence[torch.Tensor], beta: float = 0.0, noise=None, clip=None,
+                               ws=None, stream=None):
+    """outs[k] = beta*outs[k] + sum_i R_i v_i; noise = (sigma, scale, seed, tensor_ids, step) adds
+    the Gaussian mechanism in the same pass."""
+    L = load()
+    arr = _vdescs(params)
+    n = len(params)
+    optr = (C.c_void_p * n)(*[_ptr(o) for o in outs])
+    need = int(L.dp_clip_accumulate_vectors_ws_bytes(arr, n, B, T))
+    ws = _ws(need, ws, outs[0].device)
+    if noise is None:
+        with_noise, sigma, scale, seed, tids, step = 0, 0.0, 1.0, 0, None, 0
+    else:
+        sigma, scale, seed, ids_, step = noise
+        with_noise, tids = 1, (C.c_uint32 * n)(*[int(t) for t in ids_])
+    st = L.dp_clip_accumulate_vectors(arr, n, _dt(params[0].G), B, T, _ptr(sq), float(C_), _ptr(clip),
+                                      optr, float(beta), with_noise, float(sigma), float(scale),
+                                      int(seed) & (2 ** 64 - 1), tids, int(step), _ptr(ws),
+                                      ws.numel() * ws.element_size(), _stream(stream))
+    _check(st, "dp_clip_accumulate_vectors")
 
 
 def dp_embed_norms_static(ids: torch.Tensor, G: torch.Tensor, V: int, sq: torch.Tensor, d=None,

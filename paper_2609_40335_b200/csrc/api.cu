@@ -8,6 +8,7 @@
 #include "fma_kernels.cuh"
 #include "gemm_gta.cuh"
 #include "ghost_plan.cuh"
+#include "vector_kernels.cuh"
 
 namespace dpg {
 
@@ -239,6 +240,77 @@ dp_status dp_tied_cross_term(const int32_t* ids, const void* G_emb, int64_t ldge
   }
   if (s != DP_OK) return s;
   return launch_reduce_partials(partials, per, B, sq, 2.f, cross, st);
+}
+
+// ------------------------------------------------------- bias / LayerNorm parameters
+static dp_status check_vectors(const dp_vector_desc* prm, int32_t n, int32_t B, int32_t T) {
+  if (!prm || n <= 0 || B <= 0 || T <= 0) return DP_ERR_INVALID_ARG;
+  for (int k = 0; k < n; ++k) {
+    if (!prm[k].G || prm[k].p <= 0 || prm[k].ldg < prm[k].p) return DP_ERR_INVALID_ARG;
+    if (prm[k].X && prm[k].ldx < prm[k].p) return DP_ERR_INVALID_ARG;
+  }
+  return DP_OK;
+}
+
+size_t dp_vector_norms_ws_bytes(const dp_vector_desc* prm, int32_t n, int32_t B, int32_t T) {
+  if (check_vectors(prm, n, B, T) != DP_OK) return 0;
+  return align_up(size_t(B) * vector_total_slabs(prm, n) * sizeof(float), 256);
+}
+
+dp_status dp_vector_norms(const dp_vector_desc* prm, int32_t n, dp_dtype dt, int32_t B, int32_t T,
+                          float* sq, void* ws, size_t ws_bytes, void* stream) {
+  const dp_status c = check_vectors(prm, n, B, T);
+  if (c != DP_OK) return c;
+  if (!sq || (dt != DP_F32 && dt != DP_BF16)) return DP_ERR_INVALID_ARG;
+  if (!ws || ws_bytes < dp_vector_norms_ws_bytes(prm, n, B, T)) return DP_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  float* partials = static_cast<float*>(ws);
+  const int n_per = vector_total_slabs(prm, n);
+  dp_status s = launch_vector_norms(prm, n, dt, B, T, partials, n_per, st);
+  if (s != DP_OK) return s;
+  return launch_reduce_partials(partials, n_per, B, sq, 1.f, nullptr, st);
+}
+
+static size_t vector_partial_bytes(const dp_vector_desc* prm, int32_t n, int32_t B, int32_t T) {
+  size_t worst = 0;
+  for (int n0 = 0; n0 < n; n0 += kVecMaxParams) {
+    const int n1 = std::min(n, n0 + kVecMaxParams);
+    size_t cols = 0;
+    for (int k = n0; k < n1; ++k) cols += size_t(prm[k].p);
+    worst = std::max(worst, cols * vector_row_splits(prm + n0, n1 - n0, B, T, sm_count()));
+  }
+  return align_up(worst * sizeof(float), 256);
+}
+
+size_t dp_clip_accumulate_vectors_ws_bytes(const dp_vector_desc* prm, int32_t n, int32_t B,
+                                           int32_t T) {
+  if (check_vectors(prm, n, B, T) != DP_OK) return 0;
+  return align_up(size_t(B) * sizeof(float), 256) + vector_partial_bytes(prm, n, B, T);
+}
+
+dp_status dp_clip_accumulate_vectors(const dp_vector_desc* prm, int32_t n, dp_dtype dt, int32_t B,
+                                     int32_t T, const float* sq, float C, float* clip,
+                                     float* const* outs, float beta, int32_t with_noise, float sigma,
+                                     float scale, uint64_t seed, const uint32_t* tensor_ids,
+                                     uint32_t step, void* ws, size_t ws_bytes, void* stream) {
+  const dp_status c = check_vectors(prm, n, B, T);
+  if (c != DP_OK) return c;
+  if (!sq || !outs || (dt != DP_F32 && dt != DP_BF16)) return DP_ERR_INVALID_ARG;
+  if (!(beta == 0.f || beta == 1.f) || !finite_pos(C)) return DP_ERR_INVALID_ARG;
+  for (int k = 0; k < n; ++k) if (!outs[k]) return DP_ERR_INVALID_ARG;
+  if (with_noise && (!tensor_ids || !std::isfinite(sigma) || sigma < 0.f || !std::isfinite(scale)))
+    return DP_ERR_INVALID_ARG;
+  if (!ws || ws_bytes < dp_clip_accumulate_vectors_ws_bytes(prm, n, B, T)) return DP_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  float* clip_ws = static_cast<float*>(ws);
+  dp_status s = launch_clip_factors(sq, B, C, clip_ws, nullptr, st);
+  if (s != DP_OK) return s;
+  if (clip) DP_CUDA_OK(cudaMemcpyAsync(clip, clip_ws, size_t(B) * sizeof(float),
+                                       cudaMemcpyDeviceToDevice, st));
+  float* partial = reinterpret_cast<float*>(static_cast<char*>(ws) +
+                                            align_up(size_t(B) * sizeof(float), 256));
+  return launch_vector_sums(prm, n, dt, B, T, clip_ws, outs, beta, with_noise ? 1 : 0, sigma * C,
+                            with_noise ? scale : 1.f, seed, tensor_ids, step, partial, st);
 }
 
 // --------------------------------------------------------------------------- clip factors

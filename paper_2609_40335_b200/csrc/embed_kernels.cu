@@ -12,41 +12,6 @@ namespace dpg {
 
 namespace {
 
-// 8 consecutive columns of one row as floats; `nvalid` columns exist, `vec` says the 16-byte
-// (bf16) / 2 x 16-byte (fp32) vector path is aligned.
-template <typename T>
-__device__ __forceinline__ void load8(const T* p, int nvalid, bool vec, float (&v)[8]);
-
-template <>
-__device__ __forceinline__ void load8<__nv_bfloat16>(const __nv_bfloat16* p, int nvalid, bool vec,
-                                                     float (&v)[8]) {
-  if (vec && nvalid >= 8) {
-    const uint4 q = *reinterpret_cast<const uint4*>(p);
-    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      v[2 * e] = __uint_as_float(w[e] << 16);
-      v[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
-    }
-  } else {
-#pragma unroll
-    for (int e = 0; e < 8; ++e) v[e] = e < nvalid ? __bfloat162float(p[e]) : 0.f;
-  }
-}
-
-template <>
-__device__ __forceinline__ void load8<float>(const float* p, int nvalid, bool vec, float (&v)[8]) {
-  if (vec && nvalid >= 8) {
-    const float4 a = *reinterpret_cast<const float4*>(p);
-    const float4 b = *reinterpret_cast<const float4*>(p + 4);
-    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
-    v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
-  } else {
-#pragma unroll
-    for (int e = 0; e < 8; ++e) v[e] = e < nvalid ? p[e] : 0.f;
-  }
-}
-
 // ------------------------------------------------------------------ norm kernel
 // One block (8 warps) per (example, 256-column slab).  Tokens are grouped by their first
 // occurrence (warp-level id matching, then a scan over earlier tokens for group leaders) and

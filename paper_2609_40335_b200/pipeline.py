@@ -50,6 +50,7 @@ class DeviceStep:
     cross: Optional[torch.Tensor]
     dev_status: torch.Tensor
     outs: Dict[str, torch.Tensor] = field(default_factory=dict)
+    vectors: List[dp.Vector] = field(default_factory=list)      # biases / LayerNorm parameters
     ws: Optional[torch.Tensor] = None
     side_stream: Optional[torch.cuda.Stream] = None     # noise fills that overlap the norm phase
 
@@ -86,6 +87,7 @@ def upload(w: Workload, device="cuda", share_by_identity: bool = True) -> Device
         norms=torch.zeros(w.B, dtype=torch.float32, device=device),
         cross=torch.zeros(w.B, dtype=torch.float32, device=device) if w.tied else None,
         dev_status=torch.zeros(1, dtype=torch.int32, device=device))
+    ds.vectors = [dp.Vector(up(v.G), up(v.X) if v.X is not None else None, p=v.p) for v in w.vectors]
     allocate(ds)
     return ds
 
@@ -141,12 +143,17 @@ def allocate(ds: DeviceStep) -> None:
         ds.outs["lm_head"] = torch.empty(ds.lm.p, ds.lm.d, **f32)
     if ds.positions:
         ds.outs["wpe"] = torch.empty(WPE_ROWS, ds.d_model, **f32)
+    for k, v in enumerate(ds.vectors):
+        ds.outs[f"vector{k}"] = torch.empty(v.p, **f32)
     every = ds.linears + ([ds.lm] if ds.lm else [])
     dt = dp._dt(every[0].A) if every else dp._dt(ds.G_emb)
     need = 256
     if every:
         need = max(need, dp.dp_ghost_norms_ws_bytes(every, ds.B, ds.T))
         need = max(need, dp.dp_clip_accumulate_grouped_ws_bytes(every, ds.B, ds.T))
+    if ds.vectors:
+        need = max(need, dp.dp_vector_norms_ws_bytes(ds.vectors, ds.B, ds.T))
+        need = max(need, dp.dp_clip_accumulate_vectors_ws_bytes(ds.vectors, ds.B, ds.T))
     L = dp.load()
     need = max(need, int(L.dp_embed_norms_ws_bytes(ds.B, ds.T, ds.d_model)))
     need = max(need, int(L.dp_clip_accumulate_embed_ws_bytes(ds.B, ds.T, ds.d_model, ds.V)))
@@ -167,6 +174,8 @@ def norms_phase(ds: DeviceStep, stream=None, after_first_launch=None) -> None:
         dp.dp_ghost_norms(every, ds.B, ds.T, ds.sq, ws=ds.ws, dev_status=ds.dev_status, stream=stream)
     if after_first_launch is not None:
         after_first_launch()
+    if ds.vectors:
+        dp.dp_vector_norms(ds.vectors, ds.B, ds.T, ds.sq, ws=ds.ws, stream=stream)
     dp.dp_embed_norms(ds.ids, ds.G_emb, ds.V, ds.sq, ws=ds.ws, dev_status=ds.dev_status, stream=stream)
     if ds.positions:
         dp.dp_embed_norms(ds.pos_ids, ds.G_emb, ds.T, ds.sq, ws=ds.ws, dev_status=ds.dev_status,
@@ -175,6 +184,20 @@ def norms_phase(ds: DeviceStep, stream=None, after_first_launch=None) -> None:
         dp.dp_tied_cross_term(ds.ids, ds.G_emb, ds.lm.A, ds.lm.G, ds.V, sq=ds.sq, cross=ds.cross,
                               d=ds.d_model, ws=ds.ws, dev_status=ds.dev_status, stream=stream)
     dp.dp_clip_factors(ds.sq, ds.C, clip=ds.clip, norms=ds.norms, stream=stream)
+
+
+def _clip_vectors(ds: DeviceStep, beta: float, noise=None, stream=None) -> None:
+    """Clipped sums of the bias / LayerNorm parameters (noise = (seed, step, scale) fuses Eq. 3)."""
+    if not ds.vectors:
+        return
+    names = [f"vector{k}" for k in range(len(ds.vectors))]
+    args = None
+    if noise is not None:
+        seed, step, scale = noise
+        tid = tensor_ids(ds)
+        args = (ds.sigma, scale, seed, [tid[n] for n in names], step)
+    dp.dp_clip_accumulate_vectors(ds.vectors, ds.B, ds.T, ds.sq, ds.C, [ds.outs[n] for n in names],
+                                  beta=beta, noise=args, ws=ds.ws, stream=stream)
 
 
 def clip_phase(ds: DeviceStep, stream=None, gemm_events=None) -> None:
@@ -196,6 +219,7 @@ def clip_phase(ds: DeviceStep, stream=None, gemm_events=None) -> None:
     if ds.positions:
         dp.dp_clip_accumulate_embed(ds.pos_ids, ds.G_emb, WPE_ROWS, ds.sq, ds.C, ds.outs["wpe"],
                                     beta=0.0, d=ds.d_model, **kw)
+    _clip_vectors(ds, 0.0, stream=stream)
 
 
 def noise_phase(ds: DeviceStep, seed: int, step: int, scale: float = 1.0, stream=None) -> None:
@@ -231,6 +255,7 @@ def clip_noise_phase(ds: DeviceStep, seed: int, step: int, scale: float = 1.0, s
         dp.dp_clip_accumulate_embed_noise(ds.pos_ids, ds.G_emb, WPE_ROWS, ds.sq, ds.C, ds.outs["wpe"],
                                           ds.sigma, scale, seed, tid["wpe"], step, beta=0.0,
                                           d=ds.d_model, **kw)
+    _clip_vectors(ds, 0.0, noise=(seed, step, scale), stream=stream)
 
 
 def prefill_embedding_noise(ds: DeviceStep, seed: int, step: int, scale: float = 1.0,
@@ -289,6 +314,7 @@ def clip_onto_noise(ds: DeviceStep, filled: torch.cuda.Event) -> None:
     if ds.positions:
         dp.dp_clip_accumulate_embed(ds.pos_ids, ds.G_emb, WPE_ROWS, ds.sq, ds.C, ds.outs["wpe"],
                                     beta=1.0, d=ds.d_model, **kw)
+    _clip_vectors(ds, 1.0)
 
 
 def clip_after_prefill(ds: DeviceStep, seed: int, step: int, filled: torch.cuda.Event,
@@ -317,6 +343,7 @@ def clip_after_prefill(ds: DeviceStep, seed: int, step: int, filled: torch.cuda.
     if ds.positions:
         dp.dp_clip_accumulate_embed(ds.pos_ids, ds.G_emb, WPE_ROWS, ds.sq, ds.C, ds.outs["wpe"],
                                     beta=1.0, d=ds.d_model, **kw)
+    _clip_vectors(ds, 0.0, noise=(seed, step, scale))
 
 
 def overlapped_norms(ds: DeviceStep, seed: int, step: int) -> torch.cuda.Event:

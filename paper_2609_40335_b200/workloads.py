@@ -107,6 +107,16 @@ class LinearIO:
 
 
 @dataclasses.dataclass
+class VectorIO:
+    """A bias or LayerNorm parameter: gradient G (B, T, p) at its output and, for a LayerNorm
+    gain, the normalised input X (B, T, p); X is None for biases and LayerNorm shifts."""
+    name: str
+    p: int
+    G: HostTensor
+    X: Optional[HostTensor]
+
+
+@dataclasses.dataclass
 class Workload:
     name: str
     dtype: str
@@ -122,6 +132,7 @@ class Workload:
     lm: Optional[LinearIO]                # LM head (A_lm, G_lm) or None
     tied: bool
     positions: bool
+    vectors: List[VectorIO] = dataclasses.field(default_factory=list)
 
     @property
     def d_model(self) -> int:
@@ -137,14 +148,16 @@ def make_workload(name: str, *, B: int, T: int, dtype: str,
                   V: int, lm_head: bool, tied: bool = False, positions: bool = False,
                   C: float = 1.0, sigma: float = 1.0, id_dist: str = "zipf",
                   a_std: float = 1.0, g_std: float = 1e-2, seed: int = 0,
-                  shared_block_inputs: bool = False) -> Workload:
+                  shared_block_inputs: bool = False, full_model: bool = False) -> Workload:
     """Draw one workload.
 
     block_shapes: the (d, p) of the linear layers inside one transformer block.
     g_std: standard deviation of output gradients ("N(0, 1e-4)" is read as a
     variance, like the paper's N(0, sigma^2 C^2 I)).  shared_block_inputs: draw
     one tensor set per distinct layer shape and reuse it in every block (used
-    only where the full set would not fit in host memory).
+    only where the full set would not fit in host memory).  full_model: also emit the
+    biases of the block linears and the LayerNorm gains / shifts of a GPT-2 block (ln_1, ln_2,
+    final ln_f), so that the parameter blocks cover the whole model.
     """
     linears: List[LinearIO] = []
     cache = {}
@@ -170,8 +183,32 @@ def make_workload(name: str, *, B: int, T: int, dtype: str,
         A_lm = _normal((B, T, d_model), a_std, dtype, _seed_for(seed, name, "A_lm"))
         G_lm = _normal((B, T, V), g_std, dtype, _seed_for(seed, name, "G_lm"), ld=ld)
         lm = LinearIO(f"lm_head_{d_model}x{V}", d_model, V, A_lm, G_lm)
+    vectors: List[VectorIO] = []
+    if full_model:
+        per_block = len(block_shapes)
+
+        ln_cache = {}
+
+        def layer_norm(tag):
+            if tag in ln_cache:
+                return ln_cache[tag]
+            G = _normal((B, T, d_model), g_std, dtype, _seed_for(seed, name, "G_ln", tag))
+            X = _normal((B, T, d_model), 1.0, dtype, _seed_for(seed, name, "X_ln", tag))
+            ln_cache[tag] = [VectorIO(f"{tag}.gamma", d_model, G, X),
+                             VectorIO(f"{tag}.beta", d_model, G, None)]
+            return ln_cache[tag]
+
+        for blk in range(n_blocks):
+            key = 0 if shared_block_inputs else blk
+            vectors += layer_norm(f"h{key}.ln_1")
+            if per_block == 4:
+                vectors += layer_norm(f"h{key}.ln_2")
+            for li in range(per_block):                    # the bias sees the linear layer's G
+                l = linears[blk * per_block + li]
+                vectors.append(VectorIO(f"{l.name}.bias", l.p, l.G, None))
+        vectors += layer_norm("ln_f")
     return Workload(name, dtype, B, T, V, float(C), float(sigma), seed, linears, ids, G_emb,
-                    lm, tied, positions)
+                    lm, tied, positions, vectors)
 
 
 def gpt2_block_shapes(d_model: int) -> List[Tuple[int, int]]:

@@ -567,3 +567,68 @@ def test_cfg2_full_size_sampled_against_oracle():
     assert frob_rel(got, want) < 5e-3
     want_e = O.clipped_sum_embed(w.ids, w.G_emb.widened(), R, w.V)
     assert frob_rel(ds.outs["wte"].cpu().numpy(), want_e) < 1e-5
+
+
+# ------------------------------------------------------ bias / LayerNorm parameters
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("B,T,p,with_x", [(3, 128, 768, True), (2, 100, 300, False), (4, 37, 2304, True),
+                                          (2, 16, 10, True), (5, 300, 1000, False)])
+def test_vector_parameter_norms_and_clipped_sums(dtype, B, T, p, with_x):
+    g_std = 1.0 if dtype == "f32" else 1e-2
+    G = W._normal((B, T, p), g_std, dtype, 61)
+    X = W._normal((B, T, p), 1.0, dtype, 62) if with_x else None
+    Gw, Xw = G.widened(), (X.widened() if with_x else None)
+    prm = [dp.Vector(P.to_device(G), P.to_device(X) if with_x else None, p=p)]
+    sq = torch.zeros(B, device=dev())
+    dp.dp_vector_norms(prm, B, T, sq)
+    torch.cuda.synchronize()
+    sq_true = O.vector_sq_norms(Gw, Xw)
+    tol = TOL_F32 if dtype == "f32" else TIGHT_BF16
+    assert rel(sq.cpu().numpy(), sq_true).max() < tol
+    Cc = float(np.median(np.sqrt(sq_true)))
+    sq_in = torch.from_numpy(sq_true.astype(np.float32)).to(dev())
+    _, R = O.clip_factors(sq_in.cpu().numpy().astype(np.float64), Cc)
+    base = torch.randn(p, device=dev())
+    for beta in (0.0, 1.0):
+        out = base.clone()
+        dp.dp_clip_accumulate_vectors(prm, B, T, sq_in, Cc, [out], beta=beta)
+        torch.cuda.synchronize()
+        want = O.clipped_sum_vector(Gw, Xw, R) + beta * base.cpu().numpy().astype(np.float64)
+        assert frob_rel(out.cpu().numpy(), want) < 1e-5
+    # fused Gaussian mechanism == clipped sum followed by dp_add_noise, same stream
+    fused, plain = torch.empty(p, device=dev()), torch.empty(p, device=dev())
+    dp.dp_clip_accumulate_vectors(prm, B, T, sq_in, Cc, [fused], noise=(0.8, 0.5, 77, [9], 4))
+    dp.dp_clip_accumulate_vectors(prm, B, T, sq_in, Cc, [plain])
+    if p % 4 == 0:
+        dp.dp_add_noise(plain, 0.8, Cc, 0.5, 77, 9, 4)
+        torch.cuda.synchronize()
+        assert torch.equal(fused, plain)
+    want = NO.add_noise(O.clipped_sum_vector(Gw, Xw, R), 0.8, Cc, 0.5, 77, 9, 4)
+    torch.cuda.synchronize()
+    assert np.abs(fused.cpu().numpy() - want).max() < 1e-6 + 1e-5 * np.abs(want).max()
+
+
+def test_full_model_step_with_biases_and_layernorm_matches_oracle():
+    w = W.named_workload("cfg3", B=2, T=128, n_blocks=2, V=3001, full_model=True)
+    assert len(w.vectors) == 2 * (4 + 4) + 2
+    ds = P.upload(w)
+    P.dp_step(ds, noise=False)
+    torch.cuda.synchronize()
+    check_status(ds.dev_status)
+    lin = [(l.A.widened(), l.G.widened()) for l in w.linears]
+    vec = [(v.G.widened(), v.X.widened() if v.X is not None else None) for v in w.vectors]
+    ref = O.dp_step(lin, w.ids, w.G_emb.widened(), w.V, w.C, lm=(w.lm.A.widened(), w.lm.G.widened()),
+                    positions=True, vectors=vec)
+    assert rel(ds.sq.cpu().numpy(), ref["sq"]).max() < TIGHT_BF16
+    for k, want in ref["sums"].items():
+        got = ds.outs[k].cpu().numpy()
+        if k == "wpe":
+            got = got[: w.T]
+        assert frob_rel(got, want) < TOL_SUM, k
+    # fused-noise step agrees with the unfused one on every tensor, vectors included
+    a, b = P.upload(w), P.upload(w)
+    P.dp_step(a, seed=3, step=1, fused=True)
+    P.dp_step(b, seed=3, step=1, fused=False)
+    torch.cuda.synchronize()
+    for k in a.outs:
+        assert torch.allclose(a.outs[k], b.outs[k], rtol=1e-5, atol=2e-6), k
