@@ -261,6 +261,11 @@ int32_t dp_debug_force_fma(int32_t on);
  * kernel the device can hold. */
 dp_status dp_debug_noise_error_scan(float t_max, double* out4, void* stream);
 int32_t dp_debug_max_active_pairs(void);
+/* Test knob for the failure path: device-side barrier waits give up after `cycles` (0: at the
+ * first miss; negative: back to the default of about a second).  A kernel whose wait gives up
+ * ORs DP_DEV_TIMEOUT into dev_status, lets its copies and MMAs in flight finish, frees its
+ * tensor memory and returns; the context stays usable.  Returns the previous limit. */
+int64_t dp_debug_set_wait_limit(int64_t cycles);
 
 #ifdef __cplusplus
 }

@@ -48,7 +48,7 @@ EXPORTS = ["dp_vector_norms", "dp_vector_norms_ws_bytes", "dp_clip_accumulate_ve
            "dp_clip_accumulate_embed_noise", "dp_clip_accumulate_embed",
            "dp_clip_accumulate_embed_ws_bytes", "dp_add_noise", "dp_fill_noise", "dp_status_string",
            "dp_last_cuda_error", "dp_version", "dp_kernel_launches", "dp_debug_force_fma",
-           "dp_debug_noise_error_scan", "dp_debug_max_active_pairs"]
+           "dp_debug_noise_error_scan", "dp_debug_max_active_pairs", "dp_debug_set_wait_limit"]
 
 
 def lib_path() -> str:
@@ -113,6 +113,8 @@ def load():
     L.dp_kernel_launches.restype = C.c_int64
     L.dp_debug_noise_error_scan.argtypes = [f32, vp, vp]
     L.dp_debug_max_active_pairs.restype = i32
+    L.dp_debug_set_wait_limit.argtypes = [i64]
+    L.dp_debug_set_wait_limit.restype = i64
     L.dp_debug_force_fma.argtypes = [i32]
     L.dp_debug_force_fma.restype = i32
     for name in EXPORTS:

@@ -15,6 +15,7 @@ namespace dpg {
 int g_last_cuda_error = 0;
 int g_force_fma = 0;
 long long g_kernel_launches = 0;
+long long g_wait_limit = 1500000000LL;
 
 int sm_count() {
   static int n = 0;
@@ -127,6 +128,11 @@ int32_t dp_last_cuda_error(void) { return g_last_cuda_error; }
 const char* dp_version(void) { return "dp_ghost 0.1.0 (sm_100a)"; }
 int64_t dp_kernel_launches(void) { return g_kernel_launches; }
 int32_t dp_debug_max_active_pairs(void) { return gta_max_active_pairs(); }
+int64_t dp_debug_set_wait_limit(int64_t cycles) {
+  const long long prev = g_wait_limit;
+  g_wait_limit = cycles < 0 ? 1500000000LL : cycles;
+  return prev;
+}
 dp_status dp_debug_noise_error_scan(float t_max, double* out3, void* stream) {
   if (!out3) return DP_ERR_INVALID_ARG;
   return launch_noise_error_scan(t_max, out3, (cudaStream_t)stream);

@@ -41,6 +41,7 @@ struct __align__(64) CrossParams {
   int total_items;           // B * nt * nt
   float* partials;           // [B][nt*nt]
   int* dev_status;
+  long long wait_limit;
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -53,7 +54,8 @@ cross_term_tc_kernel(const __grid_constant__ CrossParams P) {
   uint64_t* empty = bars + kStages;
   uint64_t* acc_full = bars + 2 * kStages;
   uint64_t* acc_empty = acc_full + 2;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  uint64_t* mma_done = acc_empty + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mma_done + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   float* epi_red = reinterpret_cast<float*>(tmem_slot + 2);   // [2][4]
 
@@ -61,6 +63,7 @@ cross_term_tc_kernel(const __grid_constant__ CrossParams P) {
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
     for (int b = 0; b < 2; ++b) { ptx::mbar_init(&acc_full[b], 1); ptx::mbar_init(&acc_empty[b], 4); }
+    ptx::mbar_init(mma_done, 1);
     *abort_flag = 0;
     ptx::fence_mbar_init();
   }
@@ -78,7 +81,7 @@ cross_term_tc_kernel(const __grid_constant__ CrossParams P) {
       for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x) {
         const int ex = item / per_ex, tp = item % per_ex, ti = tp / P.nt, tj = tp % P.nt;
         for (int k = 0; k < P.ksteps; ++k) {
-          if (!ptx::mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+          if (!ptx::mbar_wait(&empty[stage], phase ^ 1, abort_flag, P.wait_limit)) { ok = false; break; }
           uint8_t* dst = tiles + size_t(stage) * kStageBytes;
           ptx::mbar_arrive_expect_tx(&full[stage], kStageBytes);
           ptx::tma_load_3d(dst, &P.tmE, &full[stage], k * kKStep, ti * kTile, ex);
@@ -101,11 +104,11 @@ cross_term_tc_kernel(const __grid_constant__ CrossParams P) {
       bool ok = true;
       for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x, ++n_item) {
         const uint32_t buf = n_item & 1, acc_phase = (n_item >> 1) & 1;
-        if (!ptx::mbar_wait(&acc_empty[buf], acc_phase ^ 1, abort_flag)) { ok = false; break; }
+        if (!ptx::mbar_wait(&acc_empty[buf], acc_phase ^ 1, abort_flag, P.wait_limit)) { ok = false; break; }
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * kTile;
         for (int k = 0; k < P.ksteps; ++k) {
-          if (!ptx::mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
+          if (!ptx::mbar_wait(&full[stage], phase, abort_flag, P.wait_limit)) { ok = false; break; }
           ptx::tc_fence_after();
           const uint32_t se = ptx::smem_u32(tiles + size_t(stage) * kStageBytes);
           const uint32_t sa = se + kTileBytes;
@@ -121,6 +124,7 @@ cross_term_tc_kernel(const __grid_constant__ CrossParams P) {
       if (!ok) {
         *abort_flag = 1;
         if (P.dev_status) atomicOr(P.dev_status, DP_DEV_TIMEOUT);
+        ptx::drain_issued_mmas(mma_done, false);
       }
     }
   } else {
@@ -141,7 +145,7 @@ cross_term_tc_kernel(const __grid_constant__ CrossParams P) {
         }
       }
       const __nv_bfloat16* gcol = P.Glm + size_t(ex) * P.T * P.ldgl + (id >= 0 ? id : 0);
-      if (!ptx::mbar_wait_relaxed(&acc_full[buf], acc_phase, abort_flag)) { ok = false; break; }
+      if (!ptx::mbar_wait_relaxed(&acc_full[buf], acc_phase, abort_flag, P.wait_limit)) { ok = false; break; }
       ptx::tc_fence_after();
       const uint32_t t0 = tmem_base + (uint32_t(q * 32) << 16) + buf * kTile;
       float acc = 0.f;
@@ -213,6 +217,7 @@ dp_status launch_cross_term_tc(const int* ids, const void* Ge, int64_t ldge, con
   P.total_items = B * P.nt * P.nt;
   P.partials = partials;
   P.dev_status = dev_status;
+  P.wait_limit = g_wait_limit;
   const int grid = std::min(P.total_items, sm_count());
   cross_term_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(P);
   DP_LAUNCH_OK();

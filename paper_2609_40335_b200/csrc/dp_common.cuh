@@ -12,7 +12,8 @@ namespace dpg {
 // last CUDA error code seen by an entry point (returned by dp_last_cuda_error)
 extern int g_last_cuda_error;
 extern int g_force_fma;
-extern long long g_kernel_launches;   // kernels enqueued by this library since load
+extern long long g_kernel_launches;
+extern long long g_wait_limit;       // cycles a device-side barrier wait may take (test knob)   // kernels enqueued by this library since load
 
 inline dp_status cuda_fail(cudaError_t e) {
   g_last_cuda_error = (int)e;

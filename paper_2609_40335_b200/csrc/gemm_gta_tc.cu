@@ -78,6 +78,7 @@ struct __align__(64) GtaParams {
   float* sq_partials;        // [B][n_per] (square-sum mode)
   int n_per;
   int* dev_status;
+  long long wait_limit;      // cycles a barrier wait may take before the CTA gives up
 };
 static_assert(sizeof(GtaParams) <= 32000, "kernel parameter block too large");
 
@@ -126,7 +127,8 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
   uint64_t* empty = bars + 2 * kStages;       // MMAs retired
   uint64_t* acc_full = bars + 3 * kStages;    // [2]
   uint64_t* acc_empty = acc_full + 2;         // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  uint64_t* mma_done = acc_empty + 2;         // only used when the MMA issuer gives up
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mma_done + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   float* epi_red = reinterpret_cast<float*>(tmem_slot + 2);   // [2][kEpiWarps]
 
@@ -143,6 +145,7 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
       ptx::mbar_init(&acc_full[b], 1);
       ptx::mbar_init(&acc_empty[b], kEpiWarps * kPeers);    // epilogue warps of both CTAs
     }
+    ptx::mbar_init(mma_done, 1);
     *abort_flag = 0;
     ptx::fence_mbar_init();
   }
@@ -166,7 +169,7 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
         const CUtensorMap* tg = &P.tmG[it.layer];
         const CUtensorMap* ta = &P.tmA[it.layer];
         for (int ks = it.k0; ks < it.k1; ++ks) {
-          if (!ptx::mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+          if (!ptx::mbar_wait(&empty[stage], phase ^ 1, abort_flag, P.wait_limit)) { ok = false; break; }
           const int ex = ks / P.tsteps, t0 = (ks - ex * P.tsteps) * kBK;
           uint8_t* dst = tiles + size_t(stage) * kStageBytes;
           ptx::mbar_arrive_expect_tx(&full[stage], kStageBytes);
@@ -200,14 +203,14 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
       for (int item = first_item; item < P.total_items && ok; item += item_stride, ++n_item) {
         const Item it = decode_item<kSqsum>(P, item);
         const uint32_t buf = n_item & 1, acc_phase = (n_item >> 1) & 1;
-        if (!(kPair ? ptx::mbar_wait_cluster(&acc_empty[buf], acc_phase ^ 1, abort_flag)
-                    : ptx::mbar_wait(&acc_empty[buf], acc_phase ^ 1, abort_flag))) { ok = false; break; }
+        if (!(kPair ? ptx::mbar_wait_cluster(&acc_empty[buf], acc_phase ^ 1, abort_flag, P.wait_limit)
+                    : ptx::mbar_wait(&acc_empty[buf], acc_phase ^ 1, abort_flag, P.wait_limit))) { ok = false; break; }
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * kBN;
         for (int ks = it.k0; ks < it.k1; ++ks) {
           uint64_t* go = kScale ? &ready[stage] : &full[stage];
-          if (!(kPair ? ptx::mbar_wait_cluster(go, phase, abort_flag)
-                      : ptx::mbar_wait(go, phase, abort_flag))) { ok = false; break; }
+          if (!(kPair ? ptx::mbar_wait_cluster(go, phase, abort_flag, P.wait_limit)
+                      : ptx::mbar_wait(go, phase, abort_flag, P.wait_limit))) { ok = false; break; }
           ptx::tc_fence_after();
           const uint32_t sg = ptx::smem_u32(tiles + size_t(stage) * kStageBytes);
           const uint32_t sa = sg + kGBytes;
@@ -233,6 +236,7 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
       if (!ok) {
         *abort_flag = 1;
         if (P.dev_status) atomicOr(P.dev_status, DP_DEV_TIMEOUT);
+        ptx::drain_issued_mmas(mma_done, kPair);
       }
     }
   } else if (warp < kEpiWarp0) {
@@ -249,7 +253,7 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
         for (int ks = it.k0; ks < it.k1; ++ks, ++cnt) {
           if (int(cnt % kScalerWarps) != sw) continue;
           const uint32_t stage = cnt % kStages, phase = (cnt / kStages) & 1u;
-          if (!ptx::mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
+          if (!ptx::mbar_wait(&full[stage], phase, abort_flag, P.wait_limit)) { ok = false; break; }
           const int ex = ks / P.tsteps;
           const float r = __ldg(P.clip + ex);
           if (r != 1.0f) {
@@ -301,7 +305,7 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
       const Item it = decode_item<kSqsum>(P, item);
       const GtaLayer& L = P.layer[it.layer];
       const uint32_t buf = n_item & 1, acc_phase = (n_item >> 1) & 1;
-      if (!ptx::mbar_wait_relaxed(&acc_full[buf], acc_phase, abort_flag)) { ok = false; break; }
+      if (!ptx::mbar_wait_relaxed(&acc_full[buf], acc_phase, abort_flag, P.wait_limit)) { ok = false; break; }
       ptx::tc_fence_after();
       const uint32_t t0 = tmem_base + (uint32_t(q * 32) << 16) + buf * kBN;
       const int row = it.tm * kTileM + int(rank) * kBM + q * 32 + lane;
@@ -555,6 +559,7 @@ dp_status launch_clip_accumulate_tc(const dp_linear_desc* layers, int n_layers, 
     P.total_items = items;
     P.clip = clip;
     P.dev_status = dev_status;
+    P.wait_limit = g_wait_limit;
     const int units = std::min(items, kUsePair ? sms / 2 : sms);
     s = launch_gta<kClipScale, false, kUsePair>(P, units, st);
     if (s != DP_OK) return s;
@@ -624,6 +629,7 @@ dp_status launch_direct_norm_tc(const dp_linear_desc* layers, const GhostPlan& p
     P.total_items = items;
     P.sq_partials = partials; P.n_per = plan.n_per;
     P.dev_status = dev_status;
+    P.wait_limit = g_wait_limit;
     s = launch_gta<false, true, false>(P, std::min(items, sms), st);
     if (s != DP_OK) return s;
   }

@@ -52,6 +52,7 @@ struct __align__(64) GhostParams {
   int n_per;                 // partial sums per example in the workspace
   float* partials;           // [B][n_per]
   int* dev_status;
+  long long wait_limit;      // cycles a barrier wait may take before the CTA gives up
 };
 
 struct Item {
@@ -98,7 +99,8 @@ ghost_norm_tc_kernel(const __grid_constant__ GhostParams P) {
   uint64_t* empty = bars + kStages;        // [kStages]  MMA -> TMA
   uint64_t* acc_full = bars + 2 * kStages; // [2]        MMA -> epilogue
   uint64_t* acc_empty = acc_full + 2;      // [2]        epilogue -> MMA
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  uint64_t* mma_done = acc_empty + 2;      // only used when the MMA issuer gives up
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mma_done + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   float* epi_red = reinterpret_cast<float*>(tmem_slot + 2);   // [2][4]
 
@@ -108,6 +110,7 @@ ghost_norm_tc_kernel(const __grid_constant__ GhostParams P) {
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
     for (int b = 0; b < 2; ++b) { ptx::mbar_init(&acc_full[b], 1); ptx::mbar_init(&acc_empty[b], 4); }
+    ptx::mbar_init(mma_done, 1);
     *abort_flag = 0;
     ptx::fence_mbar_init();
   }
@@ -133,7 +136,7 @@ ghost_norm_tc_kernel(const __grid_constant__ GhostParams P) {
           const CUtensorMap* tm = pass == 0 ? &P.tmA[it.layer] : &P.tmG[it.layer];
           const int k0 = pass == 0 ? it.a0 : it.g0, k1 = pass == 0 ? it.a1 : it.g1;
           for (int k = k0; k < k1; ++k) {
-            if (!ptx::mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+            if (!ptx::mbar_wait(&empty[stage], phase ^ 1, abort_flag, P.wait_limit)) { ok = false; break; }
             uint8_t* dst = tiles + size_t(stage) * kStageBytes;
             ptx::mbar_arrive_expect_tx(&full[stage], bytes);
             ptx::tma_load_3d(dst, tm, &full[stage], k * kKStep, it.ti * kTile, it.example);
@@ -163,13 +166,13 @@ ghost_norm_tc_kernel(const __grid_constant__ GhostParams P) {
         const Item it = decode_item(P, item);
         const bool diag = kDiagOnly || (it.ti == it.tj);
         const uint32_t buf = n_item & 1, acc_phase = (n_item >> 1) & 1;
-        if (!ptx::mbar_wait(&acc_empty[buf], acc_phase ^ 1, abort_flag)) { ok = false; break; }
+        if (!ptx::mbar_wait(&acc_empty[buf], acc_phase ^ 1, abort_flag, P.wait_limit)) { ok = false; break; }
         ptx::tc_fence_after();
         for (int pass = 0; pass < 2 && ok; ++pass) {
           const uint32_t d_tmem = tmem_base + buf * 256 + pass * 128;
           const int nsteps = pass == 0 ? it.a1 - it.a0 : it.g1 - it.g0;
           for (int k = 0; k < nsteps; ++k) {
-            if (!ptx::mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
+            if (!ptx::mbar_wait(&full[stage], phase, abort_flag, P.wait_limit)) { ok = false; break; }
             ptx::tc_fence_after();
             const uint32_t sa = ptx::smem_u32(tiles + size_t(stage) * kStageBytes);
             const uint32_t sb = diag ? sa : sa + kTileBytes;
@@ -189,6 +192,7 @@ ghost_norm_tc_kernel(const __grid_constant__ GhostParams P) {
       if (!ok) {
         *abort_flag = 1;
         if (P.dev_status) atomicOr(P.dev_status, DP_DEV_TIMEOUT);
+        ptx::drain_issued_mmas(mma_done, false);
       }
     }
   } else {
@@ -200,7 +204,7 @@ ghost_norm_tc_kernel(const __grid_constant__ GhostParams P) {
     for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x, ++n_item) {
       const Item it = decode_item(P, item);
       const uint32_t buf = n_item & 1, acc_phase = (n_item >> 1) & 1;
-      if (!ptx::mbar_wait_relaxed(&acc_full[buf], acc_phase, abort_flag)) { ok = false; break; }
+      if (!ptx::mbar_wait_relaxed(&acc_full[buf], acc_phase, abort_flag, P.wait_limit)) { ok = false; break; }
       ptx::tc_fence_after();
       const uint32_t t0 = tmem_base + (uint32_t(q * 32) << 16) + buf * 256;
       float acc = 0.f;
@@ -304,6 +308,7 @@ dp_status launch_ghost_norm_tc(const dp_linear_desc* layers, const GhostPlan& pl
     P.n_per = plan.n_per;
     P.partials = partials;
     P.dev_status = dev_status;
+    P.wait_limit = g_wait_limit;
     const int grid = std::min(items, sm_count());
     if (nt == 1)
       ghost_norm_tc_kernel<true><<<grid, kThreads, GhostGeo<true>::kSmemBytes, st>>>(P);

@@ -53,15 +53,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 
 // Wait for the phase with the given parity to complete; false if ~1.5e9 cycles (about a
 // second) pass first or if `*abort_flag` (shared memory) was raised by another role.
+constexpr long long kDefaultWaitLimit = 1500000000LL;     // cycles, about a second
+
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
-                                          volatile int* abort_flag) {
+                                          volatile int* abort_flag,
+                                          long long limit = kDefaultWaitLimit) {
   if (mbar_try_wait(bar, parity)) return true;
+  if (limit <= 0) return false;                       // test knob: give up at once
   const long long t0 = clock64();
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++spins & 1023u) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > 1500000000LL) return false;
+      if (clock64() - t0 > limit) return false;
     }
   }
   return true;
@@ -71,15 +75,17 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
 // accumulator): sleeps between polls so that many waiting warps do not take issue slots from
 // the few latency-critical ones (TMA producer, MMA issuer, scalers).
 __device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity,
-                                                  volatile int* abort_flag) {
+                                                  volatile int* abort_flag,
+                                                  long long limit = kDefaultWaitLimit) {
   if (mbar_try_wait(bar, parity)) return true;
+  if (limit <= 0) return false;
   const long long t0 = clock64();
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
     __nanosleep(spins < 64 ? 64 : 512);
     if ((++spins & 255u) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > 1500000000LL) return false;
+      if (clock64() - t0 > limit) return false;
     }
   }
   return true;
@@ -222,14 +228,16 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t pa
 // (.acquire/.release at CTA scope) forms are used on both sides: measured on B200, the
 // explicit .cluster-scope forms halved the kernel's throughput.
 __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity,
-                                                  volatile int* abort_flag) {
+                                                  volatile int* abort_flag,
+                                                  long long limit = kDefaultWaitLimit) {
   if (mbar_try_wait_cluster(bar, parity)) return true;
+  if (limit <= 0) return false;
   const long long t0 = clock64();
   uint32_t spins = 0;
   while (!mbar_try_wait_cluster(bar, parity)) {
     if ((++spins & 1023u) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > 1500000000LL) return false;
+      if (clock64() - t0 > limit) return false;
     }
   }
   return true;
@@ -264,6 +272,25 @@ __device__ __forceinline__ void mma_commit_pair(uint64_t* bar, uint16_t cta_mask
       "[%0], %1;" ::"r"(smem_u32(bar)),
       "h"(cta_mask)
       : "memory");
+}
+
+// same, arriving only on this CTA's barrier
+__device__ __forceinline__ void mma_commit_pair_local(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                   smem_u32(bar))
+               : "memory");
+}
+
+// After an MMA issuer gave up: wait (bounded, ~0.1 s) until the MMAs it had already issued have
+// retired, so that the CTA does not free tensor memory or exit under them.  `done` is a barrier
+// used for nothing else (count 1, fresh).
+__device__ __forceinline__ void drain_issued_mmas(uint64_t* done, bool pair) {
+  if (pair) mma_commit_pair_local(done);
+  else mma_commit(done);
+  const long long t0 = clock64();
+  while (!mbar_try_wait(done, 0)) {
+    if (clock64() - t0 > 150000000LL) break;
+  }
 }
 
 // ---- descriptors -------------------------------------------------------------

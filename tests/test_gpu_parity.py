@@ -632,3 +632,109 @@ def test_full_model_step_with_biases_and_layernorm_matches_oracle():
     torch.cuda.synchronize()
     for k in a.outs:
         assert torch.allclose(a.outs[k], b.outs[k], rtol=1e-5, atol=2e-6), k
+
+
+# ------------------------------------------------------------- device-side failure path
+def test_wait_limit_failure_path_leaves_context_usable():
+    """Failure detection without a fault: with the barrier-wait limit set to zero every role of
+    the TMA / tensor-core kernels gives up at its first unsatisfied wait, the kernels flag
+    DP_DEV_TIMEOUT, let their copies in flight land, free their tensor memory and return.  The
+    context stays usable and the same calls give correct results once the limit is restored."""
+    L = dp.load()
+    B, T, d, p, V = 4, 128, 256, 384, 1003
+    A, G = host_linear(B, T, d, p, "bf16", seed=71)
+    lin = dev_linear(A, G, dp.DP_NORM_GHOST)
+    lin_direct = dev_linear(A, G, dp.DP_NORM_DIRECT)
+    ids = torch.from_numpy(W.zipf_ids(B, T, V, 1.1, 72)).to(dev())
+    G_emb, A_lm = P.to_device(W._normal((B, T, d), 1e-2, "bf16", 73)), P.to_device(W._normal((B, T, d), 1.0, "bf16", 74))
+    G_lm = P.to_device(W._normal((B, T, V), 1e-2, "bf16", 75, ld=W.round_up(V, 8)))
+    sq_in = torch.full((B,), 4.0, device=dev())
+
+    def run_all():
+        st = torch.zeros(1, dtype=torch.int32, device=dev())
+        sq, sqd, cr = torch.zeros(B, device=dev()), torch.zeros(B, device=dev()), torch.zeros(B, device=dev())
+        out = torch.zeros(p, d, device=dev())
+        dp.dp_ghost_norms([lin], B, T, sq, dev_status=st)
+        dp.dp_ghost_norms([lin_direct], B, T, sqd, dev_status=st)
+        dp.dp_clip_accumulate(lin.A, lin.G, sq_in, 1.0, out, d=d, p=p, dev_status=st)
+        dp.dp_tied_cross_term(ids, G_emb, A_lm, G_lm, V, cross=cr, d=d, dev_status=st)
+        torch.cuda.synchronize()
+        return int(st.item()), sq, sqd, out, cr
+
+    good = run_all()
+    assert good[0] == 0
+    prev = L.dp_debug_set_wait_limit(0)
+    try:
+        bad = run_all()
+    finally:
+        L.dp_debug_set_wait_limit(prev)
+    assert bad[0] & dp.DP_DEV_TIMEOUT
+    again = run_all()
+    assert again[0] == 0
+    for a, b in zip(good[1:], again[1:]):
+        assert torch.equal(a, b)
+    want = O.linear_sq_norms(A.widened(), G.widened())
+    assert rel(again[1].cpu().numpy(), want).max() < TIGHT_BF16
+
+
+# ------------------------------------------------------------------ guard bands, edge sizes
+def test_outputs_stay_inside_their_buffers():
+    """Every output lives inside a larger allocation filled with a sentinel; after the calls only
+    the output's own elements may have changed (a stand-in for a memory checker)."""
+    B, T, d, p, V = 3, 100, 200, 300, 777
+    A, G = host_linear(B, T, d, p, "bf16", seed=81, ldg=W.round_up(p, 8))     # TMA pitch, NaN padding
+    lin = dev_linear(A, G)
+    ids = torch.from_numpy(W.zipf_ids(B, T, V, 1.1, 82)).to(dev())
+    G_emb = P.to_device(W._normal((B, T, d), 1e-2, "bf16", 83))
+    pad, sent = 1024, -12345.0
+
+    def guarded(n):
+        buf = torch.full((n + 2 * pad,), sent, device=dev())
+        return buf, buf[pad:pad + n]
+
+    sq_buf, sq = guarded(B)
+    sq.zero_()
+    ldo = d + 8                                              # padded output pitch
+    lin_buf, lin_out = guarded(p * ldo)
+    emb_buf, emb_out = guarded(V * ldo)
+    noise_buf, noise_out = guarded(4099)
+    noise_out.zero_()
+    dp.dp_ghost_norms([lin], B, T, sq)
+    dp.dp_embed_norms(ids, G_emb, V, sq)
+    dp.dp_clip_accumulate(lin.A, lin.G, sq, 1.0, lin_out.view(p, ldo)[:, :d], d=d, p=p)
+    dp.dp_clip_accumulate_embed(ids, G_emb, V, sq, 1.0, emb_out.view(V, ldo)[:, :d])
+    dp.dp_add_noise(noise_out, 1.0, 1.0, 1.0, 1, 2, 3)
+    torch.cuda.synchronize()
+    for buf in (sq_buf, lin_buf, emb_buf, noise_buf):
+        assert bool((buf[:pad] == sent).all()) and bool((buf[-pad:] == sent).all())
+    assert bool((lin_out.view(p, ldo)[:, d:] == sent).all())     # pitch padding untouched
+    assert bool((emb_out.view(V, ldo)[:, d:] == sent).all())
+    assert bool(torch.isfinite(lin_out.view(p, ldo)[:, :d]).all())
+
+
+@pytest.mark.parametrize("B,T,d,p", [(1, 1024, 64, 72), (1, 640, 136, 64), (2, 129, 64, 64)])
+def test_long_sequences_many_tile_pairs(B, T, d, p):
+    """T well beyond one 128-row tile: 8 x 8 tile pairs, ragged last tile, both norm modes."""
+    A, G = host_linear(B, T, d, p, "bf16", seed=T + d)
+    want = O.linear_sq_norms(A.widened(), G.widened())
+    for mode in (dp.DP_NORM_GHOST, dp.DP_NORM_DIRECT):
+        sq = torch.zeros(B, device=dev())
+        dp.dp_ghost_norms([dev_linear(A, G, mode)], B, T, sq)
+        torch.cuda.synchronize()
+        assert rel(sq.cpu().numpy(), want).max() < TIGHT_BF16, mode
+
+
+def test_embedding_at_the_longest_supported_sequence():
+    B, T, d, V = 1, 4096, 64, 50257
+    ids = W.zipf_ids(B, T, V, 1.1, 91)
+    G = W._normal((B, T, d), 1e-2, "bf16", 92)
+    sq = torch.zeros(B, device=dev())
+    fo = torch.zeros(B, T, dtype=torch.int32, device=dev())
+    dp.dp_embed_norms(torch.from_numpy(ids).to(dev()), P.to_device(G), V, sq, first_occ=fo)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(fo.cpu().numpy(), O.first_occurrence(ids))
+    assert rel(sq.cpu().numpy(), O.embed_sq_norms(ids, G.widened(), V)).max() < TIGHT_BF16
+    with pytest.raises(dp.DpGhostError) as e:                # one token more is refused, not mis-run
+        dp.dp_embed_norms(torch.zeros(1, 4097, dtype=torch.int32, device=dev()),
+                          torch.zeros(1, 4097, d, dtype=torch.bfloat16, device=dev()), V, sq)
+    assert e.value.status == 2
