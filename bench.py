@@ -389,6 +389,27 @@ def run_ours(args):
                           f"({t_ex:.1f} s) and noise on {n_noise} of {counts['n_params']} parameters "
                           f"({t_noise:.1f} s), scaled to one full step ({est_step:.1f} s)")}
 
+    # the same step replayed from a CUDA graph (captured once; the noise step advances on the
+    # device), and the peak device memory of the whole run
+    graph_info = None
+    if world == 1 and fused and not args.prefill:
+        sg = P.StepGraph(ds, seed=args.seed, first_step=args.warmup + args.steps)
+        for _ in range(3):
+            sg.replay()
+        q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        q0.record(stream)
+        for _ in range(args.steps):
+            sg.replay()
+        q1.record(stream)
+        torch.cuda.synchronize()
+        g_ms = q0.elapsed_time(q1) / args.steps
+        assert int(ds.dev_status.item()) == 0, "device status flagged a problem in the graph replays"
+        graph_info = {"ms_per_step": g_ms, "value": w.B / (g_ms * 1e-3), "unit": UNIT,
+                      "what": "pipeline.StepGraph: the whole step as one CUDA graph launch"}
+    memory = {"max_allocated_bytes": int(torch.cuda.max_memory_allocated(dev)),
+              "input_bytes": int(ds.input_bytes())}
+
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -402,6 +423,8 @@ def run_ours(args):
                       "norm_plus_clip": ms_norm + ms_clip,
                       "noise_fused_into_clip_accumulate": fused},
         "gpu_launches": int(launches),
+        "cuda_graph": graph_info,
+        "memory": memory,
         "clocks": clocks,
         "roofline": roofline,
         "roofline_other": others,

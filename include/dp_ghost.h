@@ -237,6 +237,23 @@ dp_status dp_clip_accumulate_embed_noise(const int32_t* ids, const void* G, int6
 dp_status dp_add_noise(float* out, int64_t n, float sigma, float C, float scale,
                        uint64_t seed, uint32_t tensor_id, uint32_t step, void* stream);
 
+/* The same on a SLICE of a tensor: out [dev, n floats, 16-byte aligned] holds elements
+ * first_element .. first_element+n-1 of the logical tensor and receives exactly the noise those
+ * elements get from dp_add_noise on the whole tensor (first_element a multiple of 4, so that a
+ * slice owns whole Philox counters; otherwise DP_ERR_ALIGNMENT).  For the data-parallel form in
+ * which each rank owns a slice of the summed gradient after a reduce-scatter: the noise is drawn
+ * once, on the owner, and equals the single-GPU stream. */
+dp_status dp_add_noise_slice(float* out, int64_t n, int64_t first_element, float sigma, float C,
+                             float scale, uint64_t seed, uint32_t tensor_id, uint32_t step,
+                             void* stream);
+
+/* Registers a device counter [dev, one uint32, must stay valid] whose current value is ADDED to
+ * the `step` argument of every noise-drawing launch enqueued afterwards (NULL: none, the
+ * default).  The kernels read it when they run, so a step captured once into a CUDA graph draws
+ * fresh noise at each replay if the graph also increments the counter.  Process-wide setting;
+ * not part of the paper (Eq. 3 only needs independent draws per step). */
+dp_status dp_noise_step_device(const uint32_t* dev_counter);
+
 /* Write-only form: out[j] = scale * sigma*C*z_j, the same stream as dp_add_noise on a zero
  * buffer.  It depends on no gradient, so it can run on a second stream while the norms are
  * computed; the clipped sums are then accumulated on top with beta = 1. */

@@ -46,7 +46,8 @@ EXPORTS = ["dp_vector_norms", "dp_vector_norms_ws_bytes", "dp_clip_accumulate_ve
            "dp_clip_accumulate", "dp_clip_accumulate_ws_bytes", "dp_clip_accumulate_grouped",
            "dp_clip_accumulate_grouped_ws_bytes", "dp_clip_accumulate_noise_grouped",
            "dp_clip_accumulate_embed_noise", "dp_clip_accumulate_embed",
-           "dp_clip_accumulate_embed_ws_bytes", "dp_add_noise", "dp_fill_noise", "dp_status_string",
+           "dp_clip_accumulate_embed_ws_bytes", "dp_add_noise", "dp_add_noise_slice", "dp_noise_step_device",
+           "dp_fill_noise", "dp_status_string",
            "dp_last_cuda_error", "dp_version", "dp_kernel_launches", "dp_debug_force_fma",
            "dp_debug_noise_error_scan", "dp_debug_max_active_pairs", "dp_debug_set_wait_limit"]
 
@@ -106,6 +107,8 @@ def load():
     L.dp_clip_accumulate_embed_ws_bytes.restype = sz
     L.dp_add_noise.argtypes = [vp, i64, f32, f32, f32, C.c_uint64, C.c_uint32, C.c_uint32, vp]
     L.dp_fill_noise.argtypes = [vp, i64, f32, f32, f32, C.c_uint64, C.c_uint32, C.c_uint32, vp]
+    L.dp_add_noise_slice.argtypes = [vp, i64, i64, f32, f32, f32, C.c_uint64, C.c_uint32, C.c_uint32, vp]
+    L.dp_noise_step_device.argtypes = [vp]
     L.dp_status_string.argtypes = [i32]
     L.dp_status_string.restype = C.c_char_p
     L.dp_last_cuda_error.restype = i32
@@ -433,6 +436,21 @@ def dp_add_noise(out: torch.Tensor, sigma: float, C_: float, scale: float, seed:
     st = L.dp_add_noise(_ptr(out), n, float(sigma), float(C_), float(scale), int(seed) & (2 ** 64 - 1),
                         int(tensor_id), int(step), _stream(stream))
     _check(st, "dp_add_noise")
+
+
+def dp_add_noise_slice(out: torch.Tensor, first_element: int, sigma: float, C_: float, scale: float,
+                       seed: int, tensor_id: int, step: int, n=None, stream=None):
+    """dp_add_noise on the slice of a tensor that starts at element `first_element` (a multiple of 4)."""
+    L = load()
+    n = out.numel() if n is None else n
+    st = L.dp_add_noise_slice(_ptr(out), n, int(first_element), float(sigma), float(C_), float(scale),
+                              int(seed) & (2 ** 64 - 1), int(tensor_id), int(step), _stream(stream))
+    _check(st, "dp_add_noise_slice")
+
+
+def dp_noise_step_device(counter) -> None:
+    """Register (tensor of one uint32/int32 on the device) or clear (None) the device step counter."""
+    _check(load().dp_noise_step_device(None if counter is None else _ptr(counter)), "dp_noise_step_device")
 
 
 def dp_fill_noise(out: torch.Tensor, sigma: float, C_: float, scale: float, seed: int,

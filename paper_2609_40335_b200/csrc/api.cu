@@ -16,6 +16,7 @@ int g_last_cuda_error = 0;
 int g_force_fma = 0;
 long long g_kernel_launches = 0;
 long long g_wait_limit = 1500000000LL;
+const uint32_t* g_step_dev = nullptr;
 
 int sm_count() {
   static int n = 0;
@@ -536,6 +537,21 @@ dp_status dp_add_noise(float* out, int64_t n, float sigma, float C, float scale,
   // a flat buffer is the (n, 1) tensor with pitch 1
   return launch_add_noise(out, n, 1, 1, false, sigma * C, scale, seed, tensor_id, step,
                           (cudaStream_t)stream);
+}
+
+dp_status dp_add_noise_slice(float* out, int64_t n, int64_t first_element, float sigma, float C,
+                             float scale, uint64_t seed, uint32_t tensor_id, uint32_t step,
+                             void* stream) {
+  if (!out || n < 0 || first_element < 0) return DP_ERR_INVALID_ARG;
+  if (!noise_args_ok(sigma, C, scale)) return DP_ERR_INVALID_ARG;
+  if (!aligned16(out) || (first_element & 3)) return DP_ERR_ALIGNMENT;   // whole Philox counters
+  return launch_add_noise(out, n, 1, 1, false, sigma * C, scale, seed, tensor_id, step,
+                          (cudaStream_t)stream, first_element >> 2);
+}
+
+dp_status dp_noise_step_device(const uint32_t* dev_counter) {
+  g_step_dev = dev_counter;
+  return DP_OK;
 }
 
 dp_status dp_fill_noise(float* out, int64_t n, float sigma, float C, float scale, uint64_t seed,

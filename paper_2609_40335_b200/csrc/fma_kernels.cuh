@@ -46,7 +46,7 @@ size_t embed_scatter_partial_bytes(long long n, int d);
 // fill: write scale*amp*z without reading out.
 dp_status launch_add_noise(float* out, long long rows, int cols, long long ld, bool fill, float amp,
                            float scale, uint64_t seed, uint32_t tensor_id, uint32_t step,
-                           cudaStream_t st);
+                           cudaStream_t st, long long first_quad = 0);
 
 dp_status launch_noise_error_scan(float t_max, double* out3, cudaStream_t st);
 

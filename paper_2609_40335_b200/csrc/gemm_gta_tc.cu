@@ -74,6 +74,7 @@ struct __align__(64) GtaParams {
   int total_items;
   const float* clip;         // [B] R_i (scale mode)
   uint32_t noise_k0, noise_k1, noise_step;   // Gaussian stream of the fused noise (per-layer id)
+  const uint32_t* step_dev;  // optional device counter added to noise_step
   float noise_scale;
   float* sq_partials;        // [B][n_per] (square-sum mode)
   int n_per;
@@ -344,7 +345,7 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
         const bool vec_ok = ((ld & 3) == 0) && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0);
         // fused Gaussian mechanism (Eq. 3): only on the final destination, never on a K-split plane
         const bool noisy = (L.noise_amp >= 0.f) && (L.nsplit == 1);
-        const NoiseKey nkey{P.noise_k0, P.noise_k1, L.tensor_id, P.noise_step};
+        const NoiseKey nkey{P.noise_k0, P.noise_k1, L.tensor_id, effective_step(P.noise_step, P.step_dev)};
 #pragma unroll 1
         for (int c = c_lo; c < c_hi; ++c) {
           uint32_t r[32];
@@ -554,6 +555,7 @@ dp_status launch_clip_accumulate_tc(const dp_linear_desc* layers, int n_layers, 
     if (noise) {
       P.noise_k0 = uint32_t(noise->seed); P.noise_k1 = uint32_t(noise->seed >> 32);
       P.noise_step = noise->step; P.noise_scale = noise->scale;
+      P.step_dev = g_step_dev;
     }
     P.n_layers = g1 - g0; P.B = B; P.T = T; P.tsteps = tsteps;
     P.total_items = items;

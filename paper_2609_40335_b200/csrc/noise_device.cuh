@@ -22,6 +22,13 @@ struct NoiseKey {
   uint32_t tensor_id, step;
 };
 
+// The step word of a launch: the host's value plus, when a device counter is registered
+// (dp_noise_step_device), the counter's current value -- so that a captured CUDA graph draws
+// fresh noise at every replay.
+__device__ __forceinline__ uint32_t effective_step(uint32_t step, const uint32_t* step_dev) {
+  return step_dev ? step + __ldg(step_dev) : step;
+}
+
 struct U4 { uint32_t x, y, z, w; };
 
 __device__ __forceinline__ U4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,

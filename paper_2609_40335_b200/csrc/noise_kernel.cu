@@ -16,13 +16,14 @@ namespace {
 template <bool kFill>
 __global__ void __launch_bounds__(256)
 add_noise_kernel(float* __restrict__ out, long long n, int cols, long long ld, float amp,
-                 float scale, NoiseKey key) {
+                 float scale, NoiseKey key, const uint32_t* __restrict__ step_dev, long long q0) {
+  key.step = effective_step(key.step, step_dev);
   const long long nq = (n + 3) >> 2;
   const bool flat = (ld == cols);
   for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < nq;
        q += (long long)gridDim.x * blockDim.x) {
     float z[4];
-    normals4((unsigned long long)q, key, z);
+    normals4((unsigned long long)(q0 + q), key, z);       // q0: first counter of a slice
     const long long j = q << 2;
     if (flat && j + 3 < n) {
       float4 v = kFill ? make_float4(0.f, 0.f, 0.f, 0.f) : *reinterpret_cast<float4*>(out + j);
@@ -81,7 +82,7 @@ dp_status launch_noise_error_scan(float t_max, double* out3 /*4 doubles*/, cudaS
 
 dp_status launch_add_noise(float* out, long long rows, int cols, long long ld, bool fill, float amp,
                            float scale, uint64_t seed, uint32_t tensor_id, uint32_t step,
-                           cudaStream_t st) {
+                           cudaStream_t st, long long first_quad) {
   const long long n = rows * cols;
   if (n == 0) return DP_OK;
   const long long nq = (n + 3) >> 2;
@@ -99,9 +100,9 @@ dp_status launch_add_noise(float* out, long long rows, int cols, long long ld, b
     carveout_set = true;
   }
   if (fill)
-    add_noise_kernel<true><<<grid, 256, 0, st>>>(out, n, cols, ld, amp, scale, key);
+    add_noise_kernel<true><<<grid, 256, 0, st>>>(out, n, cols, ld, amp, scale, key, g_step_dev, first_quad);
   else
-    add_noise_kernel<false><<<grid, 256, 0, st>>>(out, n, cols, ld, amp, scale, key);
+    add_noise_kernel<false><<<grid, 256, 0, st>>>(out, n, cols, ld, amp, scale, key, g_step_dev, first_quad);
   DP_LAUNCH_OK();
   return DP_OK;
 }

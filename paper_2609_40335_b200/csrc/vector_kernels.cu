@@ -156,7 +156,7 @@ vector_sum_kernel(const __grid_constant__ VecParams P, const float* __restrict__
 __global__ void __launch_bounds__(256)
 vector_combine_kernel(const __grid_constant__ VecParams P, const float* __restrict__ partial,
                       int nsplit, float beta, int with_noise, float amp, float scale, uint32_t k0,
-                      uint32_t k1, uint32_t step) {
+                      uint32_t k1, uint32_t step, const uint32_t* __restrict__ step_dev) {
   const int slab = blockIdx.x;
   const VecParam& q = P.prm[find_param(P, slab)];
   const int cc = (slab - q.slab_begin) * kVecCols + threadIdx.x;
@@ -165,7 +165,7 @@ vector_combine_kernel(const __grid_constant__ VecParams P, const float* __restri
   for (int s = 0; s < nsplit; ++s) v += partial[size_t(s) * P.total_cols + q.col_begin + cc];
   if (beta != 0.f) v += q.out[cc];
   if (with_noise) {
-    const NoiseKey key{k0, k1, q.tensor_id, step};
+    const NoiseKey key{k0, k1, q.tensor_id, effective_step(step, step_dev)};
     float z[4];
     normals4((unsigned long long)(cc >> 2), key, z);
     const int e = cc & 3;
@@ -246,7 +246,7 @@ dp_status launch_vector_sums(const dp_vector_desc* prm, int n, dp_dtype dt, int 
     else vector_sum_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(P, clip, rps, partial_ws);
     DP_LAUNCH_OK();
     vector_combine_kernel<<<slabs, 256, 0, st>>>(P, partial_ws, nsplit, beta, with_noise, amp, scale,
-                                                uint32_t(seed), uint32_t(seed >> 32), step);
+                                                uint32_t(seed), uint32_t(seed >> 32), step, g_step_dev);
     DP_LAUNCH_OK();
   }
   return DP_OK;

@@ -379,3 +379,36 @@ def dp_step(ds: DeviceStep, seed: int = 0, step: int = 0, noise: bool = True, fu
     clip_phase(ds, stream)
     if noise:
         noise_phase(ds, seed, step, stream=stream)
+
+
+class StepGraph:
+    """One whole step (norms -> clipped sums -> noise) captured once into a CUDA graph.
+
+    The noise `step` word cannot be baked into the captured launches, so the kernels read a device
+    counter (dp_noise_step_device) that the graph itself increments: replay k draws the stream of
+    step `first_step + k`, exactly what `dp_step(ds, seed, step=first_step + k)` draws.  The graph
+    holds the addresses of `ds`'s tensors: refill them in place between replays.
+    """
+
+    def __init__(self, ds: DeviceStep, seed: int = 0, first_step: int = 0):
+        self.ds = ds
+        dev = ds.sq.device
+        self.counter = torch.full((1,), int(first_step), dtype=torch.int32, device=dev)
+        # one eager step first: one-time kernel attribute setup must not happen during capture
+        side = torch.cuda.Stream(device=dev)
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            dp_step(ds, seed=seed, step=first_step)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize(dev)
+        self.graph = torch.cuda.CUDAGraph()
+        dp.dp_noise_step_device(self.counter)
+        try:
+            with torch.cuda.graph(self.graph):
+                dp_step(ds, seed=seed, step=0)
+                self.counter.add_(1)
+        finally:
+            dp.dp_noise_step_device(None)        # eager calls made later take their step as given
+
+    def replay(self) -> None:
+        self.graph.replay()

@@ -738,3 +738,52 @@ def test_embedding_at_the_longest_supported_sequence():
         dp.dp_embed_norms(torch.zeros(1, 4097, dtype=torch.int32, device=dev()),
                           torch.zeros(1, 4097, d, dtype=torch.bfloat16, device=dev()), V, sq)
     assert e.value.status == 2
+
+
+# ------------------------------------------------- slice noise, device step counter, step graph
+def test_noise_on_slices_equals_the_whole_tensor_stream():
+    seed, tid, step, n = 0x1234567890ABCDEF, 3, 9, 10007
+    base = torch.randn(n, device=dev())
+    whole = base.clone()
+    dp.dp_add_noise(whole, 0.7, 1.3, 1.0, seed, tid, step)
+    sliced = torch.empty_like(base)
+    for lo, hi in [(0, 4096), (4096, 4100), (4100, 10007)]:
+        part = base[lo:hi].clone()                         # its own 16-byte aligned buffer
+        dp.dp_add_noise_slice(part, lo, 0.7, 1.3, 1.0, seed, tid, step)
+        sliced[lo:hi] = part
+        z = NO.standard_normals(hi - lo, seed, tid, step, start=lo)
+        want = base[lo:hi].cpu().numpy().astype(np.float64) + 0.7 * 1.3 * z
+        assert np.abs(part.cpu().numpy() - want).max() < 2e-6
+    assert torch.equal(whole, sliced)                      # bit for bit the single-call result
+    with pytest.raises(dp.DpGhostError):                   # a slice must start on a counter boundary
+        dp.dp_add_noise_slice(base[:8].clone(), 2, 0.7, 1.3, 1.0, seed, tid, step)
+
+
+def test_device_step_counter_is_added_to_the_step_word():
+    seed, tid, n = 77, 1, 4099
+    counter = torch.full((1,), 5, dtype=torch.int32, device=dev())
+    x = torch.empty(n, device=dev())
+    dp.dp_noise_step_device(counter)
+    try:
+        dp.dp_fill_noise(x, 1.0, 1.0, 1.0, seed, tid, 2)
+        torch.cuda.synchronize()
+    finally:
+        dp.dp_noise_step_device(None)
+    assert np.abs(x.cpu().numpy() - NO.standard_normals(n, seed, tid, 7)).max() < 1e-6
+    dp.dp_fill_noise(x, 1.0, 1.0, 1.0, seed, tid, 2)       # cleared: the step is taken as given
+    assert np.abs(x.cpu().numpy() - NO.standard_normals(n, seed, tid, 2)).max() < 1e-6
+
+
+def test_step_graph_replays_equal_eager_steps():
+    w = W.named_workload("cfg4", B=3, n_blocks=1, V=4099)
+    a, b = P.upload(w), P.upload(w)
+    g = P.StepGraph(a, seed=13, first_step=4)
+    for k in range(3):                                     # replay k draws the noise of step 4 + k
+        g.replay()
+        P.dp_step(b, seed=13, step=4 + k)
+        torch.cuda.synchronize()
+        check_status(a.dev_status)
+        for name in a.outs:
+            assert torch.equal(a.outs[name], b.outs[name]), (k, name)
+        assert torch.equal(a.sq, b.sq)
+    assert int(g.counter.item()) == 7

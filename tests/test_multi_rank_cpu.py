@@ -32,8 +32,18 @@ def _worker(rank, world, port, ret):
     def add_noise(t, tid):
         t.copy_(torch.from_numpy(NO.add_noise(t.numpy(), 0.5, C, 1.0, 3, tid, 11)))
 
+    outs2 = {k: v.clone() for k, v in outs.items()}
     parallel.reduce_then_noise(outs, add_noise)
     ret[rank] = {k: v.numpy().copy() for k, v in outs.items()}
+
+    # reduce-scatter form: each rank noises only the slice it owns, the slices are gathered back
+    def add_noise_slice(t, first, tid):
+        z = NO.standard_normals(t.numel(), 3, tid, 11, start=first)
+        t.copy_(torch.from_numpy(1.0 * (t.numpy() + 0.5 * C * z)))
+
+    owned = parallel.reduce_scatter_then_noise(outs2, add_noise_slice)
+    ret[f"rs{rank}"] = {k: v.numpy().copy() for k, v in outs2.items()}
+    ret[f"own{rank}"] = {k: (lo, hi) for k, (lo, hi, _) in owned.items()}
     ret[f"clip{rank}"] = (lo, hi, res["clip"])
     dist.destroy_process_group()
 
@@ -45,6 +55,8 @@ def test_two_ranks_reproduce_the_single_process_step():
 
     assert [parallel.shard_range(5, r, 2) for r in range(2)] == [(0, 3), (3, 5)]
     assert [parallel.shard_range(7, r, 3) for r in range(3)] == [(0, 3), (3, 5), (5, 7)]
+    assert [parallel.slice_bounds(10, r, 3) for r in range(3)] == [(4, 0, 4), (4, 4, 8), (4, 8, 10)]
+    assert parallel.slice_bounds(3, 1, 2) == (4, 3, 3)                     # empty trailing slice
     ctx = mp.get_context("spawn")
     ret = ctx.Manager().dict()
     port = 29500 + os.getpid() % 2000
@@ -63,6 +75,12 @@ def test_two_ranks_reproduce_the_single_process_step():
         want = NO.add_noise(full["sums"][k], 0.5, C, 1.0, 3, tid, 11)
         np.testing.assert_allclose(ret[0][k], want, rtol=1e-12, atol=1e-12)
         np.testing.assert_array_equal(ret[0][k], ret[1][k])       # replicas stay identical
+        # the reduce-scatter form gives the same noised sums on both ranks
+        np.testing.assert_allclose(ret["rs0"][k], want, rtol=1e-12, atol=1e-12)
+        np.testing.assert_array_equal(ret["rs0"][k], ret["rs1"][k])
+        n = want.size
+        (lo0, hi0), (lo1, hi1) = ret["own0"][k], ret["own1"][k]
+        assert lo0 == 0 and hi0 == lo1 and hi1 == n and lo1 % 4 == 0      # slices tile the tensor
     for r in range(2):
         lo, hi, clip = ret[f"clip{r}"]
         np.testing.assert_allclose(clip, full["clip"][lo:hi], rtol=1e-12)
