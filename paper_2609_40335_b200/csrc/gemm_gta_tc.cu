@@ -39,24 +39,39 @@ namespace dpg {
 
 namespace {
 
-constexpr int kBM = 128, kBN = 256, kBK = 64;
-constexpr int kBoxBytes = 64 * 128;                 // 64 token rows x 128 bytes
+#ifndef DPG_GTA_BK
+#define DPG_GTA_BK 64
+#endif
+constexpr int kBM = 128, kBN = 256, kBK = DPG_GTA_BK;
+constexpr int kBoxBytes = kBK * 128;                // kBK token rows x 128 bytes
 constexpr int kGBytes = (kBM / 64) * kBoxBytes;     // 16 KiB: this CTA's 128 rows of the G tile
 
 // Tile geometry.  Single CTA: 128 x 256 output tile, the CTA loads all 256 columns of the A
 // tile (48 KiB per stage, 4 stages).  CTA pair (cta_group::2): 256 x 256 output tile per pair;
-// each CTA loads its own 128 G rows and HALF of the A tile's columns (32 KiB per stage, 6
-// stages), the pair's MMA reads both halves -- a third less operand traffic per flop.
+// each CTA loads its own 128 G rows and HALF of the A tile's columns (32 KiB per stage, 7
+// stages: all the shared memory there is -- the ring is latency-bound, 7 stages measured 973
+// TFLOP/s where 6 gave 895; 32- and 128-row K steps were both slower), the pair's MMA reads
+// both halves -- a third less operand traffic per flop.
+#ifndef DPG_GTA_PAIR_STAGES
+#define DPG_GTA_PAIR_STAGES 7
+#endif
 template <bool kPair>
 struct Geo {
   static constexpr int kAColsPerCta = kPair ? kBN / 2 : kBN;
   static constexpr int kABytes = (kAColsPerCta / 64) * kBoxBytes;
   static constexpr int kStageBytes = kGBytes + kABytes;
-  static constexpr int kStages = kPair ? 6 : 4;
+  static constexpr int kStages = kPair ? DPG_GTA_PAIR_STAGES : 4;
   static constexpr int kTileM = kPair ? 2 * kBM : kBM;       // output rows per work item
-  static constexpr size_t kSmemBytes = size_t(kStages) * kStageBytes + 1024 + 256;
+  static constexpr size_t kSmemBytes = size_t(kStages) * kStageBytes + 1024 + 512;
 };
-constexpr int kScalerWarps = 4;
+#ifndef DPG_GTA_SCALERS
+#define DPG_GTA_SCALERS 4
+#endif
+constexpr int kScalerWarps = DPG_GTA_SCALERS;
+// A scaler warp steps kScalerWarps K steps at a time and tells "this stage has landed" from the
+// parity of the stage's barrier alone, which is only unambiguous while it is less than one trip
+// round the ring ahead of the loads.
+static_assert(kScalerWarps <= 4 && kScalerWarps <= DPG_GTA_PAIR_STAGES, "scaler warps may not lap the stage ring");
 constexpr int kEpiWarp0 = 2 + kScalerWarps;          // first epilogue warp
 #ifndef DPG_GTA_EPI_WARPS
 #define DPG_GTA_EPI_WARPS 16
@@ -530,9 +545,9 @@ dp_status launch_clip_accumulate_tc(const dp_linear_desc* layers, int n_layers, 
     int items = 0;
     for (int g = g0; g < g1; ++g) {
       const dp_linear_desc& D = layers[g];
-      s = make_tmap_bf16_3d(&P.tmG[g - g0], D.G, D.ldg, D.p, T, B, 64, 64);
+      s = make_tmap_bf16_3d(&P.tmG[g - g0], D.G, D.ldg, D.p, T, B, 64, kBK);
       if (s != DP_OK) return s;
-      s = make_tmap_bf16_3d(&P.tmA[g - g0], D.A, D.lda, D.d, T, B, 64, 64);
+      s = make_tmap_bf16_3d(&P.tmA[g - g0], D.A, D.lda, D.d, T, B, 64, kBK);
       if (s != DP_OK) return s;
       GtaLayer& L = P.layer[g - g0];
       L.out = outs[g]; L.ldo = ldos[g]; L.beta = beta;
@@ -614,9 +629,9 @@ dp_status launch_direct_norm_tc(const dp_linear_desc* layers, const GhostPlan& p
     for (size_t g = g0; g < g1; ++g) {
       const int li = plan.direct_layers[g];
       const dp_linear_desc& D = layers[li];
-      s = make_tmap_bf16_3d(&P.tmG[g - g0], D.G, D.ldg, D.p, T, B, 64, 64);
+      s = make_tmap_bf16_3d(&P.tmG[g - g0], D.G, D.ldg, D.p, T, B, 64, kBK);
       if (s != DP_OK) return s;
-      s = make_tmap_bf16_3d(&P.tmA[g - g0], D.A, D.lda, D.d, T, B, 64, 64);
+      s = make_tmap_bf16_3d(&P.tmA[g - g0], D.A, D.lda, D.d, T, B, 64, kBK);
       if (s != DP_OK) return s;
       GtaLayer& L = P.layer[g - g0];
       L.M = D.p; L.N = D.d;
