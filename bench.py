@@ -240,6 +240,17 @@ def run_ours(args):
             P.noise_phase(ds, seed=args.seed, step=k)
         if ev: ev[3].record(stream)
 
+    # default at N = 1: the whole step captured once as a CUDA graph and replayed (the noise step
+    # advances on the device); --eager issues the same calls one by one instead
+    use_graph = (world == 1) and fused and not args.prefill and not args.eager
+    sg = None
+    if use_graph:
+        sg = P.StepGraph(ds, seed=args.seed, first_step=0)
+        eager_step = step
+
+        def step(k, ev=None):          # noqa: F811  (replaces the eager step for every later use)
+            sg.replay()
+
     for k in range(args.warmup):
         step(k)
     torch.cuda.synchronize()
@@ -265,6 +276,8 @@ def run_ours(args):
     if world > 1:
         dist.barrier()
     launches = dp.dp_kernel_launches() - launches0
+    if use_graph:
+        launches = sg.kernels_per_replay * args.steps      # replays do not pass through the library
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
     ms_total = e0.elapsed_time(e1)
     if world > 1:
@@ -274,9 +287,28 @@ def run_ours(args):
     assert int(ds.dev_status.item()) == 0, "device status flagged a problem in the timed region"
     ms_step = ms_total / args.steps
     value = world * w.B / (ms_step * 1e-3)
-    ms_norm = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
-    ms_clip = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
-    ms_noise = statistics.mean(e[2].elapsed_time(e[3]) for e in evs)
+    graph_detail = None
+    if use_graph:
+        # per-phase and GEMM durations: external CUDA events inside the graph, read after each of
+        # K more replays (the events of the timed region's last replay are read first)
+        sgt = P.StepGraph(ds, seed=args.seed, first_step=args.warmup + args.steps, timing=True)
+        det = []
+        for _ in range(args.steps):
+            sgt.replay()
+            torch.cuda.synchronize()
+            det.append(sgt.phase_ms())
+        ms_norm = statistics.mean(d["norms"] for d in det)
+        ms_clip = statistics.mean(d["clip_accumulate"] for d in det)
+        ms_noise = 0.0
+        graph_detail = {"how": "phases and the GEMM are timed by external CUDA events inside a second "
+                               "capture of the same step (the event nodes cost ~40 us per step, so "
+                               "the timed region replays a capture without them); averages over %d "
+                               "replays, each read after a synchronize" % args.steps,
+                        "step_ms_with_event_nodes": statistics.mean(d["step"] for d in det)}
+    else:
+        ms_norm = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
+        ms_clip = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
+        ms_noise = statistics.mean(e[2].elapsed_time(e[3]) for e in evs)
 
     # dominant kernel: the tensor-core G^T A GEMM of the clipped sums.  Its duration is taken
     # live inside the timed region: CUDA events bracket the grouped call in every timed step (the
@@ -284,7 +316,9 @@ def run_ours(args):
     # accumulates onto pre-filled noise and is not bracketed.
     lin_layers = ds.linears + ([ds.lm] if ds.lm else [])
     g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    if fused and args.prefill:
+    if use_graph:
+        gemm_ms_avg = statistics.mean(d["gemm"] for d in det)
+    elif fused and args.prefill:
         gemm_ms_avg = ms_clip
     else:
         gemm_ms_avg = statistics.mean(e[4].elapsed_time(e[5]) for e in evs)
@@ -389,24 +423,23 @@ def run_ours(args):
                           f"({t_ex:.1f} s) and noise on {n_noise} of {counts['n_params']} parameters "
                           f"({t_noise:.1f} s), scaled to one full step ({est_step:.1f} s)")}
 
-    # the same step replayed from a CUDA graph (captured once; the noise step advances on the
-    # device), and the peak device memory of the whole run
+    # the same step issued call by call (no graph), for comparison
     graph_info = None
-    if world == 1 and fused and not args.prefill:
-        sg = P.StepGraph(ds, seed=args.seed, first_step=args.warmup + args.steps)
-        for _ in range(3):
-            sg.replay()
+    if use_graph:
+        for k in range(3):
+            eager_step(k)
         q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         q0.record(stream)
-        for _ in range(args.steps):
-            sg.replay()
+        for k in range(args.steps):
+            eager_step(k)
         q1.record(stream)
         torch.cuda.synchronize()
-        g_ms = q0.elapsed_time(q1) / args.steps
-        assert int(ds.dev_status.item()) == 0, "device status flagged a problem in the graph replays"
-        graph_info = {"ms_per_step": g_ms, "value": w.B / (g_ms * 1e-3), "unit": UNIT,
-                      "what": "pipeline.StepGraph: the whole step as one CUDA graph launch"}
+        e_ms = q0.elapsed_time(q1) / args.steps
+        assert int(ds.dev_status.item()) == 0, "device status flagged a problem in the eager steps"
+        graph_info = {"timed_region": "replays of pipeline.StepGraph (one CUDA graph launch per step)",
+                      "kernels_per_replay": int(sg.kernels_per_replay),
+                      "eager_ms_per_step": e_ms, "eager_value": w.B / (e_ms * 1e-3), **graph_detail}
     memory = {"max_allocated_bytes": int(torch.cuda.max_memory_allocated(dev)),
               "input_bytes": int(ds.input_bytes())}
 
@@ -444,6 +477,8 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--eager", action="store_true",
+                    help="issue the step call by call instead of replaying a captured CUDA graph")
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--B", type=int, default=0, help="override the workload's batch size (cfg5 sweep)")
     ap.add_argument("--T", type=int, default=0, help="override the workload's sequence length")

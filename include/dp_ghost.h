@@ -202,6 +202,22 @@ dp_status dp_clip_accumulate_embed(const int32_t* ids, const void* G, int64_t ld
                                    void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
 size_t dp_clip_accumulate_embed_ws_bytes(int32_t B, int32_t T, int32_t d, int32_t V);
 
+/* The same in two calls, so that the sort -- which needs only the ids -- can run early, e.g. on
+ * a second stream while the norms are computed.  dp_embed_sort writes perm [dev, B*T int32] and
+ * seg [dev, V+1 int32] as described above (ws of dp_embed_sort_ws_bytes);
+ * dp_clip_accumulate_embed_sorted is dp_clip_accumulate_embed with that sort given (perm, seg
+ * are inputs; ws of dp_clip_accumulate_embed_ws_bytes).  Out-of-range ids are flagged by the
+ * sort (DP_DEV_BAD_ID) and skipped by both. */
+dp_status dp_embed_sort(const int32_t* ids, int32_t B, int32_t T, int32_t V, int32_t* perm,
+                        int32_t* seg, void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+size_t dp_embed_sort_ws_bytes(int32_t B, int32_t T, int32_t V);
+dp_status dp_clip_accumulate_embed_sorted(const int32_t* ids, const void* G, int64_t ldg, dp_dtype dt,
+                                          int32_t B, int32_t T, int32_t d, int32_t V,
+                                          const float* sq, float C, float* clip,
+                                          float* out, int64_t ldo, float beta,
+                                          const int32_t* perm, const int32_t* seg,
+                                          void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
+
 /* ---- clipped sums with the Gaussian mechanism fused in (Eq. 2, Eq. 3, Eq. 7 in one pass) ----
  * Same as dp_clip_accumulate_grouped, then outs[k] = scale * (outs[k] + sigma*C*z) with the
  * stream (seed, tensor_ids[k], step) of dp_add_noise, element j = row*d + col.  The noise is

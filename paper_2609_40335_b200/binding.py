@@ -46,7 +46,8 @@ EXPORTS = ["dp_vector_norms", "dp_vector_norms_ws_bytes", "dp_clip_accumulate_ve
            "dp_clip_accumulate", "dp_clip_accumulate_ws_bytes", "dp_clip_accumulate_grouped",
            "dp_clip_accumulate_grouped_ws_bytes", "dp_clip_accumulate_noise_grouped",
            "dp_clip_accumulate_embed_noise", "dp_clip_accumulate_embed",
-           "dp_clip_accumulate_embed_ws_bytes", "dp_add_noise", "dp_add_noise_slice", "dp_noise_step_device",
+           "dp_clip_accumulate_embed_ws_bytes", "dp_embed_sort", "dp_embed_sort_ws_bytes",
+           "dp_clip_accumulate_embed_sorted", "dp_add_noise", "dp_add_noise_slice", "dp_noise_step_device",
            "dp_fill_noise", "dp_status_string",
            "dp_last_cuda_error", "dp_version", "dp_kernel_launches", "dp_debug_force_fma",
            "dp_debug_noise_error_scan", "dp_debug_max_active_pairs", "dp_debug_set_wait_limit"]
@@ -105,6 +106,11 @@ def load():
                                            f32, vp, vp, vp, sz, vp, vp]
     L.dp_clip_accumulate_embed_ws_bytes.argtypes = [i32, i32, i32, i32]
     L.dp_clip_accumulate_embed_ws_bytes.restype = sz
+    L.dp_embed_sort.argtypes = [vp, i32, i32, i32, vp, vp, vp, sz, vp, vp]
+    L.dp_embed_sort_ws_bytes.argtypes = [i32, i32, i32]
+    L.dp_embed_sort_ws_bytes.restype = sz
+    L.dp_clip_accumulate_embed_sorted.argtypes = [vp, vp, i64, i32, i32, i32, i32, i32, vp, f32, vp, vp,
+                                                  i64, f32, vp, vp, vp, sz, vp, vp]
     L.dp_add_noise.argtypes = [vp, i64, f32, f32, f32, C.c_uint64, C.c_uint32, C.c_uint32, vp]
     L.dp_fill_noise.argtypes = [vp, i64, f32, f32, f32, C.c_uint64, C.c_uint32, C.c_uint32, vp]
     L.dp_add_noise_slice.argtypes = [vp, i64, i64, f32, f32, f32, C.c_uint64, C.c_uint32, C.c_uint32, vp]
@@ -426,6 +432,31 @@ def dp_clip_accumulate_embed(ids, G, V: int, sq, C_: float, out, beta: float = 0
                                     _ptr(perm), _ptr(seg), _ptr(ws), ws.numel() * ws.element_size(),
                                     _ptr(dev_status), _stream(stream))
     _check(st, "dp_clip_accumulate_embed")
+
+
+def dp_embed_sort(ids, V: int, perm, seg, ws=None, dev_status=None, stream=None):
+    """Stable counting sort of the B*T token ids: perm (B*T int32), seg (V+1 int32)."""
+    L = load()
+    B, T = ids.shape
+    ws = _ws(int(L.dp_embed_sort_ws_bytes(B, T, V)), ws, ids.device)
+    st = L.dp_embed_sort(_ptr(ids), B, T, V, _ptr(perm), _ptr(seg), _ptr(ws),
+                         ws.numel() * ws.element_size(), _ptr(dev_status), _stream(stream))
+    _check(st, "dp_embed_sort")
+
+
+def dp_clip_accumulate_embed_sorted(ids, G, V: int, sq, C_: float, out, perm, seg, beta: float = 0.0,
+                                    d=None, clip=None, ws=None, dev_status=None, stream=None):
+    """dp_clip_accumulate_embed with the sort (dp_embed_sort) already done."""
+    L = load()
+    B, T = ids.shape
+    d = d if d is not None else G.shape[-1]
+    ws = _ws(int(L.dp_clip_accumulate_embed_ws_bytes(B, T, d, V)), ws, out.device)
+    st = L.dp_clip_accumulate_embed_sorted(_ptr(ids), _ptr(G), _rows_ld(G), _dt(G), B, T, d, V,
+                                           _ptr(sq), float(C_), _ptr(clip), _ptr(out), out.stride(0),
+                                           float(beta), _ptr(perm), _ptr(seg), _ptr(ws),
+                                           ws.numel() * ws.element_size(), _ptr(dev_status),
+                                           _stream(stream))
+    _check(st, "dp_clip_accumulate_embed_sorted")
 
 
 def dp_add_noise(out: torch.Tensor, sigma: float, C_: float, scale: float, seed: int,

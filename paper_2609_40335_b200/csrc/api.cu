@@ -460,8 +460,11 @@ static dp_status clip_accumulate_embed_impl(const int32_t* ids, const void* G, i
                                             const float* sq, float C, float* clip, float* out,
                                             int64_t ldo, float beta, const EmbedNoise* noise,
                                             int32_t* perm, int32_t* seg, void* ws, size_t ws_bytes,
-                                            int32_t* dev_status, void* stream) {
+                                            int32_t* dev_status, void* stream,
+                                            const int32_t* perm_in = nullptr,
+                                            const int32_t* seg_in = nullptr) {
   if (!ids || !G || !sq || !out || B <= 0 || T <= 0 || d <= 0 || V <= 0) return DP_ERR_INVALID_ARG;
+  if ((perm_in == nullptr) != (seg_in == nullptr)) return DP_ERR_INVALID_ARG;
   if (ldg < d || ldo < d) return DP_ERR_INVALID_ARG;
   if (dt != DP_F32 && dt != DP_BF16) return DP_ERR_INVALID_ARG;
   if (!(beta == 0.f || beta == 1.f) || !finite_pos(C)) return DP_ERR_INVALID_ARG;
@@ -483,8 +486,13 @@ static dp_status clip_accumulate_embed_impl(const int32_t* ids, const void* G, i
   if (s != DP_OK) return s;
   if (clip) DP_CUDA_OK(cudaMemcpyAsync(clip, clip_ws, size_t(B) * sizeof(float),
                                        cudaMemcpyDeviceToDevice, st));
-  s = launch_embed_sort(ids, n, V, sw, dev_status, st);
-  if (s != DP_OK) return s;
+  if (perm_in) {                         // sorted earlier by dp_embed_sort
+    sw.perm = const_cast<int*>(perm_in);
+    sw.seg = const_cast<int*>(seg_in);
+  } else {
+    s = launch_embed_sort(ids, n, V, sw, dev_status, st);
+    if (s != DP_OK) return s;
+  }
   if (perm) DP_CUDA_OK(cudaMemcpyAsync(perm, sw.perm, size_t(n) * sizeof(int),
                                        cudaMemcpyDeviceToDevice, st));
   if (seg) DP_CUDA_OK(cudaMemcpyAsync(seg, sw.seg, size_t(V + 1) * sizeof(int),
@@ -513,6 +521,38 @@ dp_status dp_clip_accumulate_embed(const int32_t* ids, const void* G, int64_t ld
                                    int32_t* dev_status, void* stream) {
   return clip_accumulate_embed_impl(ids, G, ldg, dt, B, T, d, V, sq, C, clip, out, ldo, beta, nullptr,
                                     perm, seg, ws, ws_bytes, dev_status, stream);
+}
+
+size_t dp_embed_sort_ws_bytes(int32_t B, int32_t T, int32_t V) {
+  if (B <= 0 || T <= 0 || V <= 0) return 0;
+  const size_t chunks = (size_t(B) * T + kSortChunk - 1) / kSortChunk;
+  return align_up(chunks * V * sizeof(int), 256) + align_up(size_t(ceil_div(V, 1024)) * sizeof(int), 256);
+}
+
+dp_status dp_embed_sort(const int32_t* ids, int32_t B, int32_t T, int32_t V, int32_t* perm,
+                        int32_t* seg, void* ws, size_t ws_bytes, int32_t* dev_status, void* stream) {
+  if (!ids || !perm || !seg || B <= 0 || T <= 0 || V <= 0) return DP_ERR_INVALID_ARG;
+  if ((long long)B * T > 0x7fffffffLL) return DP_ERR_UNSUPPORTED;
+  if (!ws || ws_bytes < dp_embed_sort_ws_bytes(B, T, V)) return DP_ERR_WORKSPACE;
+  const int n = B * T;
+  EmbedSortWs sw;
+  sw.chunks = (n + kSortChunk - 1) / kSortChunk;
+  sw.counts = static_cast<int*>(ws);
+  sw.block_sums = reinterpret_cast<int*>(static_cast<char*>(ws) +
+                                         align_up(size_t(sw.chunks) * V * sizeof(int), 256));
+  sw.seg = seg;
+  sw.perm = perm;
+  return launch_embed_sort(ids, n, V, sw, dev_status, (cudaStream_t)stream);
+}
+
+dp_status dp_clip_accumulate_embed_sorted(const int32_t* ids, const void* G, int64_t ldg, dp_dtype dt,
+                                          int32_t B, int32_t T, int32_t d, int32_t V, const float* sq,
+                                          float C, float* clip, float* out, int64_t ldo, float beta,
+                                          const int32_t* perm, const int32_t* seg, void* ws,
+                                          size_t ws_bytes, int32_t* dev_status, void* stream) {
+  if (!perm || !seg) return DP_ERR_INVALID_ARG;
+  return clip_accumulate_embed_impl(ids, G, ldg, dt, B, T, d, V, sq, C, clip, out, ldo, beta, nullptr,
+                                    nullptr, nullptr, ws, ws_bytes, dev_status, stream, perm, seg);
 }
 
 dp_status dp_clip_accumulate_embed_noise(const int32_t* ids, const void* G, int64_t ldg, dp_dtype dt,

@@ -52,7 +52,8 @@ class DeviceStep:
     outs: Dict[str, torch.Tensor] = field(default_factory=dict)
     vectors: List[dp.Vector] = field(default_factory=list)      # biases / LayerNorm parameters
     ws: Optional[torch.Tensor] = None
-    side_stream: Optional[torch.cuda.Stream] = None     # noise fills that overlap the norm phase
+    side_stream: Optional[torch.cuda.Stream] = None     # work that overlaps the big norm kernel
+    side: Optional[dict] = None       # side-stream buffers: own workspace, norm accumulator, sorts
 
     def input_bytes(self) -> int:
         """Bytes of input one step reads (a tensor shared by several layers counts every time)."""
@@ -337,40 +338,95 @@ def clip_after_prefill(ds: DeviceStep, seed: int, step: int, filled: torch.cuda.
         if gemm_events:
             gemm_events[1].record(torch.cuda.current_stream())
     torch.cuda.current_stream().wait_event(filled)
-    # beta = 1: rows are added onto the noise (untied) or onto head sum + noise (tied)
-    dp.dp_clip_accumulate_embed(ds.ids, ds.G_emb, ds.V, ds.sq, ds.C, ds.outs["wte"], beta=1.0,
-                                d=ds.d_model, **kw)
+    # beta = 1: rows are added onto the noise (untied) or onto head sum + noise (tied); the token
+    # sorts were made beside the norm phase
+    sb = ds.side
+    dp.dp_clip_accumulate_embed_sorted(ds.ids, ds.G_emb, ds.V, ds.sq, ds.C, ds.outs["wte"], sb["perm"],
+                                       sb["seg"], beta=1.0, d=ds.d_model, **kw)
     if ds.positions:
-        dp.dp_clip_accumulate_embed(ds.pos_ids, ds.G_emb, WPE_ROWS, ds.sq, ds.C, ds.outs["wpe"],
-                                    beta=1.0, d=ds.d_model, **kw)
+        dp.dp_clip_accumulate_embed_sorted(ds.pos_ids, ds.G_emb, WPE_ROWS, ds.sq, ds.C, ds.outs["wpe"],
+                                           sb["pos_perm"], sb["pos_seg"], beta=1.0, d=ds.d_model, **kw)
     _clip_vectors(ds, 0.0, noise=(seed, step, scale))
 
 
+def _side_buffers(ds: DeviceStep) -> dict:
+    """Buffers of the side stream (allocated once): it runs beside the main stream, so it needs its
+    own workspace and its own norm accumulator; the token sorts it makes are kept for the scatter."""
+    if ds.side is None:
+        dev = ds.sq.device
+        L = dp.load()
+        rows = max(ds.V, WPE_ROWS if ds.positions else 0)
+        need = max(int(L.dp_embed_norms_ws_bytes(ds.B, ds.T, ds.d_model)),
+                   int(L.dp_embed_sort_ws_bytes(ds.B, ds.T, rows)), 256)
+        ds.side = dict(
+            ws=torch.empty(need, dtype=torch.uint8, device=dev),
+            sq=torch.zeros(ds.B, dtype=torch.float32, device=dev),
+            perm=torch.empty(ds.B * ds.T, dtype=torch.int32, device=dev),
+            seg=torch.empty(ds.V + 1, dtype=torch.int32, device=dev),
+            pos_perm=torch.empty(ds.B * ds.T, dtype=torch.int32, device=dev) if ds.positions else None,
+            pos_seg=torch.empty(WPE_ROWS + 1, dtype=torch.int32, device=dev) if ds.positions else None)
+    return ds.side
+
+
 def overlapped_norms(ds: DeviceStep, seed: int, step: int) -> torch.cuda.Event:
-    """Norm phase with the embedding tables' noise fill beside it.  The fill is enqueued right
-    AFTER the big norm kernel: measured on B200, a fill that is already resident keeps the norm
-    kernel's CTAs out until it ends, while a fill that arrives second shares the SMs."""
+    """Norm phase with everything that does not need the big norm kernel running BESIDE it on a
+    side stream: the embedding norms (small kernels), the token sorts of the scatter (they need
+    only the ids) and the embedding tables' noise fill (ALU-bound, depends on no gradient).  The
+    side work is enqueued right AFTER the big kernel: measured on B200, work that is already
+    resident keeps the norm kernel's CTAs out until it ends, while work that arrives second shares
+    the SMs.  Returns the event after which the tables hold their noise and the sorts exist."""
+    main = torch.cuda.current_stream()
+    if ds.side_stream is None:
+        ds.side_stream = torch.cuda.Stream(device=ds.sq.device)
+    side, sb = ds.side_stream, _side_buffers(ds)
     start = torch.cuda.Event()
-    start.record(torch.cuda.current_stream())
-    box = {}
-
-    def launch_fill():
-        box["ev"] = prefill_embedding_noise(ds, seed, step, after=start)
-
-    norms_phase(ds, after_first_launch=launch_fill)
-    return box["ev"]
+    start.record(main)
+    ds.sq.zero_()
+    every = ds.linears + ([ds.lm] if ds.lm else [])
+    if every:
+        dp.dp_ghost_norms(every, ds.B, ds.T, ds.sq, ws=ds.ws, dev_status=ds.dev_status)
+    # ---- side stream
+    side.wait_event(start)                       # previous step's readers of these buffers are done
+    with torch.cuda.stream(side):
+        sb["sq"].zero_()
+    kw = dict(ws=sb["ws"], dev_status=ds.dev_status, stream=side)
+    dp.dp_embed_norms(ds.ids, ds.G_emb, ds.V, sb["sq"], **kw)
+    if ds.positions:
+        dp.dp_embed_norms(ds.pos_ids, ds.G_emb, ds.T, sb["sq"], **kw)
+    normed = torch.cuda.Event()
+    normed.record(side)
+    dp.dp_embed_sort(ds.ids, ds.V, sb["perm"], sb["seg"], **kw)
+    if ds.positions:
+        dp.dp_embed_sort(ds.pos_ids, WPE_ROWS, sb["pos_perm"], sb["pos_seg"], **kw)
+    filled = prefill_embedding_noise(ds, seed, step, after=start)
+    # ---- main stream again
+    if ds.vectors:
+        dp.dp_vector_norms(ds.vectors, ds.B, ds.T, ds.sq, ws=ds.ws)
+    if ds.tied:
+        dp.dp_tied_cross_term(ds.ids, ds.G_emb, ds.lm.A, ds.lm.G, ds.V, sq=ds.sq, cross=ds.cross,
+                              d=ds.d_model, ws=ds.ws, dev_status=ds.dev_status)
+    main.wait_event(normed)
+    ds.sq.add_(sb["sq"])                         # one fixed order of additions: deterministic
+    dp.dp_clip_factors(ds.sq, ds.C, clip=ds.clip, norms=ds.norms)
+    return filled
 
 
 def dp_step(ds: DeviceStep, seed: int = 0, step: int = 0, noise: bool = True, fused: bool = True,
-            overlap: bool = True, stream=None) -> None:
+            overlap: bool = True, stream=None, events=None) -> None:
     """norms -> clipped sums -> noise.
 
     fused=True draws the linear-layer noise inside the clipped-sum GEMM; with overlap=True the
     embedding tables' noise is filled on a side stream while the norms run (scale 1 only).
     """
     if noise and fused and overlap and stream is None:
+        # events (optional, default path only): five CUDA events recorded at step start, after the
+        # norm phase, around the grouped GEMM call and at step end
+        cur = torch.cuda.current_stream()
+        if events: events[0].record(cur)
         filled = overlapped_norms(ds, seed, step)
-        clip_after_prefill(ds, seed, step, filled)
+        if events: events[1].record(cur)
+        clip_after_prefill(ds, seed, step, filled, gemm_events=(events[2], events[3]) if events else None)
+        if events: events[4].record(cur)
         return
     norms_phase(ds, stream)
     if noise and fused:
@@ -390,8 +446,12 @@ class StepGraph:
     holds the addresses of `ds`'s tensors: refill them in place between replays.
     """
 
-    def __init__(self, ds: DeviceStep, seed: int = 0, first_step: int = 0):
+    def __init__(self, ds: DeviceStep, seed: int = 0, first_step: int = 0, timing: bool = False):
         self.ds = ds
+        # timing=True: external events inside the graph (step start, norms done, GEMM start, GEMM
+        # end, step end), readable after a replay has completed
+        self.events = ([torch.cuda.Event(enable_timing=True, external=True) for _ in range(5)]
+                       if timing else None)
         dev = ds.sq.device
         self.counter = torch.full((1,), int(first_step), dtype=torch.int32, device=dev)
         # one eager step first: one-time kernel attribute setup must not happen during capture
@@ -404,11 +464,19 @@ class StepGraph:
         self.graph = torch.cuda.CUDAGraph()
         dp.dp_noise_step_device(self.counter)
         try:
+            n0 = dp.dp_kernel_launches()
             with torch.cuda.graph(self.graph):
-                dp_step(ds, seed=seed, step=0)
+                dp_step(ds, seed=seed, step=0, events=self.events)
                 self.counter.add_(1)
+            self.kernels_per_replay = dp.dp_kernel_launches() - n0    # this library's kernels
         finally:
             dp.dp_noise_step_device(None)        # eager calls made later take their step as given
 
     def replay(self) -> None:
         self.graph.replay()
+
+    def phase_ms(self) -> dict:
+        """Durations inside the LAST completed replay (timing=True; synchronize first)."""
+        e = self.events
+        return {"norms": e[0].elapsed_time(e[1]), "clip_accumulate": e[1].elapsed_time(e[4]),
+                "gemm": e[2].elapsed_time(e[3]), "step": e[0].elapsed_time(e[4])}
