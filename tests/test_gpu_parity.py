@@ -787,3 +787,31 @@ def test_step_graph_replays_equal_eager_steps():
             assert torch.equal(a.outs[name], b.outs[name]), (k, name)
         assert torch.equal(a.sq, b.sq)
     assert int(g.counter.item()) == 7
+
+
+@pytest.mark.parametrize("B,T,d,V,beta", [(3, 128, 768, 50257, 0.0), (5, 700, 100, 300, 1.0), (2, 40, 132, 7, 1.0)])
+def test_sort_in_its_own_call_then_sorted_scatter(B, T, d, V, beta):
+    """dp_embed_sort + dp_clip_accumulate_embed_sorted == dp_clip_accumulate_embed, bit for bit."""
+    ids = W.zipf_ids(B, T, V, 1.1, 31)
+    G = W._normal((B, T, d), 1e-2, "bf16", 32)
+    sq_true = O.embed_sq_norms(ids, G.widened(), V)
+    Cc = float(np.median(np.sqrt(sq_true)))
+    sq = torch.from_numpy(sq_true.astype(np.float32)).to(dev())
+    ids_d, G_d = torch.from_numpy(ids).to(dev()), P.to_device(G)
+    out0 = torch.randn(V, d, device=dev())
+    one, two = out0.clone(), out0.clone()
+    st = torch.zeros(1, dtype=torch.int32, device=dev())
+    dp.dp_clip_accumulate_embed(ids_d, G_d, V, sq, Cc, one, beta=beta, dev_status=st)
+    perm = torch.full((B * T,), -1, dtype=torch.int32, device=dev())
+    seg = torch.full((V + 1,), -1, dtype=torch.int32, device=dev())
+    dp.dp_embed_sort(ids_d, V, perm, seg, dev_status=st)
+    dp.dp_clip_accumulate_embed_sorted(ids_d, G_d, V, sq, Cc, two, perm, seg, beta=beta, dev_status=st)
+    torch.cuda.synchronize()
+    check_status(st)
+    want_perm, want_seg = O.stable_token_sort(ids, V)
+    np.testing.assert_array_equal(perm.cpu().numpy(), want_perm)
+    np.testing.assert_array_equal(seg.cpu().numpy(), want_seg)
+    assert torch.equal(one, two)
+    _, R = O.clip_factors(sq.cpu().numpy().astype(np.float64), Cc)
+    want = O.clipped_sum_embed(ids, G.widened(), R, V) + beta * out0.cpu().numpy().astype(np.float64)
+    assert frob_rel(two.cpu().numpy(), want) < 1e-5
