@@ -276,6 +276,22 @@ dp_status dp_noise_step_device(const uint32_t* dev_counter);
 dp_status dp_fill_noise(float* out, int64_t n, float sigma, float C, float scale,
                         uint64_t seed, uint32_t tensor_id, uint32_t step, void* stream);
 
+/* ---- privacy accounting on the host (no device work) ----
+ * The paper calibrates sigma with a Renyi-DP accountant from the target epsilon (3 in the main
+ * experiments), delta = N^-1.1, the sampling rate q = batch / N and the number of steps.  One step
+ * is the Poisson-subsampled Gaussian mechanism with sensitivity 1 (clipping to C, noise sigma*C);
+ * for integer orders alpha = 2..256 its Renyi divergence is a binomial sum, RDP adds over steps,
+ * and epsilon = min_alpha steps*rdp(alpha) + log(1/delta)/(alpha-1).
+ * dp_rdp_epsilon: epsilon [host, out] and the minimising order best_order [host, out or NULL]
+ * for 0 <= q <= 1, sigma > 0, steps >= 0, 0 < delta < 1 (else DP_ERR_INVALID_ARG).
+ * dp_sigma_for_epsilon: the smallest sigma, to `tolerance`, whose epsilon does not exceed
+ * target_epsilon (bisection; DP_ERR_UNSUPPORTED when the target is below what the conversion
+ * term alone leaves).  All pointers are host pointers. */
+dp_status dp_rdp_epsilon(double q, double sigma, int64_t steps, double delta, double* epsilon,
+                         int32_t* best_order);
+dp_status dp_sigma_for_epsilon(double q, int64_t steps, double target_epsilon, double delta,
+                               double tolerance, double* sigma);
+
 /* ---- helpers ---- */
 const char* dp_status_string(dp_status s);
 int32_t dp_last_cuda_error(void);      /* cudaError_t / CUresult of the last DP_ERR_CUDA */

@@ -48,7 +48,7 @@ EXPORTS = ["dp_vector_norms", "dp_vector_norms_ws_bytes", "dp_clip_accumulate_ve
            "dp_clip_accumulate_embed_noise", "dp_clip_accumulate_embed",
            "dp_clip_accumulate_embed_ws_bytes", "dp_embed_sort", "dp_embed_sort_ws_bytes",
            "dp_clip_accumulate_embed_sorted", "dp_add_noise", "dp_add_noise_slice", "dp_noise_step_device",
-           "dp_fill_noise", "dp_status_string",
+           "dp_fill_noise", "dp_rdp_epsilon", "dp_sigma_for_epsilon", "dp_status_string",
            "dp_last_cuda_error", "dp_version", "dp_kernel_launches", "dp_debug_force_fma",
            "dp_debug_noise_error_scan", "dp_debug_max_active_pairs", "dp_debug_set_wait_limit"]
 
@@ -115,6 +115,8 @@ def load():
     L.dp_fill_noise.argtypes = [vp, i64, f32, f32, f32, C.c_uint64, C.c_uint32, C.c_uint32, vp]
     L.dp_add_noise_slice.argtypes = [vp, i64, i64, f32, f32, f32, C.c_uint64, C.c_uint32, C.c_uint32, vp]
     L.dp_noise_step_device.argtypes = [vp]
+    L.dp_rdp_epsilon.argtypes = [C.c_double, C.c_double, i64, C.c_double, vp, vp]
+    L.dp_sigma_for_epsilon.argtypes = [C.c_double, i64, C.c_double, C.c_double, C.c_double, vp]
     L.dp_status_string.argtypes = [i32]
     L.dp_status_string.restype = C.c_char_p
     L.dp_last_cuda_error.restype = i32
@@ -492,6 +494,23 @@ def dp_fill_noise(out: torch.Tensor, sigma: float, C_: float, scale: float, seed
     st = L.dp_fill_noise(_ptr(out), n, float(sigma), float(C_), float(scale), int(seed) & (2 ** 64 - 1),
                          int(tensor_id), int(step), _stream(stream))
     _check(st, "dp_fill_noise")
+
+
+def dp_rdp_epsilon(q: float, sigma: float, steps: int, delta: float):
+    """(epsilon, best order) of `steps` DP-SGD steps with sampling rate q and noise multiplier sigma."""
+    eps, order = C.c_double(0.0), C.c_int32(0)
+    _check(load().dp_rdp_epsilon(float(q), float(sigma), int(steps), float(delta), C.byref(eps),
+                                 C.byref(order)), "dp_rdp_epsilon")
+    return eps.value, order.value
+
+
+def dp_sigma_for_epsilon(q: float, steps: int, target_epsilon: float, delta: float,
+                         tolerance: float = 1e-6) -> float:
+    """Smallest noise multiplier (to `tolerance`) that keeps epsilon within the target."""
+    sigma = C.c_double(0.0)
+    _check(load().dp_sigma_for_epsilon(float(q), int(steps), float(target_epsilon), float(delta),
+                                       float(tolerance), C.byref(sigma)), "dp_sigma_for_epsilon")
+    return sigma.value
 
 
 def dp_debug_force_fma(on: bool) -> bool:
