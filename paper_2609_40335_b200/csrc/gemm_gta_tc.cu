@@ -126,6 +126,7 @@ __device__ __forceinline__ Item decode_item(const GtaParams& P, int item) {
 template <bool kScale, bool kSqsum, bool kPair>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_gta_kernel(const __grid_constant__ GtaParams P) {
+  static_assert(kScale || !kPair, "CTA pairs need the scaler warps' cross-CTA stage hand-off");
   constexpr int kStages = Geo<kPair>::kStages;
   constexpr int kStageBytes = Geo<kPair>::kStageBytes;
   constexpr int kTileM = Geo<kPair>::kTileM;
@@ -451,11 +452,11 @@ __global__ void splitk_reduce_kernel(const float* __restrict__ partial, int nspl
   }
 }
 
-#ifdef DPG_GTA_NOSCALE
-constexpr bool kClipScale = false;   // experiment only: clip factors are ignored
-#else
+// The clipped sum always runs with kScale = true: on CTA pairs the scaler warps are also what
+// tells rank 0's MMA issuer that BOTH CTAs' halves of a stage have landed.  (kScale = false is
+// for the single-CTA DIRECT-norm kernel only; a pair kernel without the scalers' hand-off would
+// let the issuer run ahead of the partner's loads and re-arm a stage barrier in mid-phase.)
 constexpr bool kClipScale = true;
-#endif
 
 #ifdef DPG_GTA_SINGLE_CTA
 constexpr bool kUsePair = false;     // experiment only: clipped sums on the single-CTA tiles
