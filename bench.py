@@ -254,7 +254,7 @@ def run_ours(args):
     for k in range(args.warmup):
         step(k)
     torch.cuda.synchronize()
-    assert int(ds.dev_status.item()) == 0, "device status flagged a problem during warm-up"
+    assert int(ds.dev_status.item()) == 0, "device status %#x flagged a problem during warm-up" % int(ds.dev_status.item())
 
     sampler = ClockSampler(local)
     if rank == 0:

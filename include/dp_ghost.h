@@ -303,6 +303,10 @@ int64_t dp_kernel_launches(void);
  * instead of the tensor-core ones (used to cross-check the two on the device).  Returns
  * the previous value.  Off by default; not meant for production use. */
 int32_t dp_debug_force_fma(int32_t on);
+/* Test hook: when non-zero, sequences longer than 128 tokens keep the single-CTA 128 x 128 Gram
+ * kernel instead of the CTA-pair 256 x 256 one (used to cross-check the two on the device).
+ * Returns the previous value. */
+int32_t dp_debug_ghost_single(int32_t on);
 /* Diagnostics.  dp_debug_noise_error_scan: exhaustive float64 check of the fp32 Box-Muller
  * factors over all 2^24 inputs; out4 [dev, 4 doubles] = {max relative error of the radius for
  * r^2 <= t_max (t_max <= 0: the threshold in use), max absolute error of cos/sin, largest radius

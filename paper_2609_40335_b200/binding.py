@@ -50,7 +50,8 @@ EXPORTS = ["dp_vector_norms", "dp_vector_norms_ws_bytes", "dp_clip_accumulate_ve
            "dp_clip_accumulate_embed_sorted", "dp_add_noise", "dp_add_noise_slice", "dp_noise_step_device",
            "dp_fill_noise", "dp_rdp_epsilon", "dp_sigma_for_epsilon", "dp_status_string",
            "dp_last_cuda_error", "dp_version", "dp_kernel_launches", "dp_debug_force_fma",
-           "dp_debug_noise_error_scan", "dp_debug_max_active_pairs", "dp_debug_set_wait_limit"]
+           "dp_debug_noise_error_scan", "dp_debug_max_active_pairs", "dp_debug_set_wait_limit",
+           "dp_debug_ghost_single"]
 
 
 def lib_path() -> str:
@@ -126,6 +127,8 @@ def load():
     L.dp_debug_max_active_pairs.restype = i32
     L.dp_debug_set_wait_limit.argtypes = [i64]
     L.dp_debug_set_wait_limit.restype = i64
+    L.dp_debug_ghost_single.argtypes = [i32]
+    L.dp_debug_ghost_single.restype = i32
     L.dp_debug_force_fma.argtypes = [i32]
     L.dp_debug_force_fma.restype = i32
     for name in EXPORTS:
@@ -511,6 +514,10 @@ def dp_sigma_for_epsilon(q: float, steps: int, target_epsilon: float, delta: flo
     _check(load().dp_sigma_for_epsilon(float(q), int(steps), float(target_epsilon), float(delta),
                                        float(tolerance), C.byref(sigma)), "dp_sigma_for_epsilon")
     return sigma.value
+
+
+def dp_debug_ghost_single(on: bool) -> bool:
+    return bool(load().dp_debug_ghost_single(1 if on else 0))
 
 
 def dp_debug_force_fma(on: bool) -> bool:

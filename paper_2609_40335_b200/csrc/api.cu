@@ -17,6 +17,7 @@ int g_force_fma = 0;
 long long g_kernel_launches = 0;
 long long g_wait_limit = 1500000000LL;
 const uint32_t* g_step_dev = nullptr;
+int g_ghost_single = 0;
 
 int sm_count() {
   static int n = 0;
@@ -34,7 +35,10 @@ int sm_count() {
 // ---- planning of dp_ghost_norms ------------------------------------------------------------
 GhostPlan plan_ghost_norms(const dp_linear_desc* layers, int n_layers, int B, int T, int sms) {
   GhostPlan plan;
-  const int nt = ceil_div(T, 128);
+  plan.pair = T > 128 && !g_ghost_single;
+  const int nt = ceil_div(T, plan.pair ? 256 : 128);
+  const int slots = plan.pair ? 2 : 1;           // partial sums per work item
+  const int units = plan.pair ? sms / 2 : sms;   // persistent CTAs or CTA pairs
   plan.ntp = nt * (nt + 1) / 2;
   plan.layer.resize(n_layers);
   plan.direct.resize(n_layers);
@@ -64,7 +68,7 @@ GhostPlan plan_ghost_norms(const dp_linear_desc* layers, int n_layers, int B, in
       L.nsplit = ceil_div(large, L.chunk_steps);
       items += (long long)B * plan.ntp * L.nsplit;
     }
-    if (items >= 2LL * sms || budget <= 8 || plan.ghost_layers.empty()) break;
+    if (items >= 2LL * units || budget <= 8 || plan.ghost_layers.empty()) break;
     budget /= 2;
   }
   // longest items first: with a static round-robin split the last, partly filled wave then
@@ -81,7 +85,7 @@ GhostPlan plan_ghost_norms(const dp_linear_desc* layers, int n_layers, int B, in
     if (plan.mode_used[l] == DP_NORM_GHOST) {
       plan.layer[l].col_begin = col;
       plan.layer[l].item_begin = 0;
-      col += plan.ntp * plan.layer[l].nsplit;
+      col += plan.ntp * plan.layer[l].nsplit * slots;
     } else {
       plan.direct[l].tiles_m = ceil_div(layers[l].p, 128);
       plan.direct[l].tiles_n = ceil_div(layers[l].d, 256);
@@ -128,6 +132,12 @@ const char* dp_status_string(dp_status s) {
 int32_t dp_last_cuda_error(void) { return g_last_cuda_error; }
 const char* dp_version(void) { return "dp_ghost 0.1.0 (sm_100a)"; }
 int64_t dp_kernel_launches(void) { return g_kernel_launches; }
+
+int32_t dp_debug_ghost_single(int32_t on) {
+  const int prev = g_ghost_single;
+  g_ghost_single = on ? 1 : 0;
+  return prev;
+}
 int32_t dp_debug_max_active_pairs(void) { return gta_max_active_pairs(); }
 int64_t dp_debug_set_wait_limit(int64_t cycles) {
   const long long prev = g_wait_limit;
@@ -178,7 +188,8 @@ dp_status dp_ghost_norms(dp_linear_desc* layers, int32_t n_layers, dp_dtype dt, 
   float* partials = static_cast<float*>(ws);
   dp_status s = DP_OK;
   if (!plan.ghost_layers.empty()) {
-    s = launch_ghost_norm_tc(layers, plan, B, T, partials, dev_status, st);
+    s = plan.pair ? launch_ghost_norm_pair(layers, plan, B, T, partials, dev_status, st)
+                  : launch_ghost_norm_tc(layers, plan, B, T, partials, dev_status, st);
     if (s != DP_OK) return s;
   }
   if (!plan.direct_layers.empty()) {

@@ -14,6 +14,7 @@ extern int g_last_cuda_error;
 extern int g_force_fma;
 extern long long g_kernel_launches;
 extern const uint32_t* g_step_dev;   // device counter added to every noise step (NULL: none)
+extern int g_ghost_single;           // test knob: keep the single-CTA Gram kernel for T > 128
 extern long long g_wait_limit;       // cycles a device-side barrier wait may take (test knob)   // kernels enqueued by this library since load
 
 inline dp_status cuda_fail(cudaError_t e) {

@@ -68,10 +68,6 @@ struct Geo {
 #define DPG_GTA_SCALERS 4
 #endif
 constexpr int kScalerWarps = DPG_GTA_SCALERS;
-// A scaler warp steps kScalerWarps K steps at a time and tells "this stage has landed" from the
-// parity of the stage's barrier alone, which is only unambiguous while it is less than one trip
-// round the ring ahead of the loads.
-static_assert(kScalerWarps <= 4 && kScalerWarps <= DPG_GTA_PAIR_STAGES, "scaler warps may not lap the stage ring");
 constexpr int kEpiWarp0 = 2 + kScalerWarps;          // first epilogue warp
 #ifndef DPG_GTA_EPI_WARPS
 #define DPG_GTA_EPI_WARPS 16
@@ -269,7 +265,13 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
         const Item it = decode_item<kSqsum>(P, item);
         for (int ks = it.k0; ks < it.k1; ++ks, ++cnt) {
           if (int(cnt % kScalerWarps) != sw) continue;
-          const uint32_t stage = cnt % kStages, phase = (cnt / kStages) & 1u;
+          const uint32_t stage = cnt % kStages, fill = cnt / kStages, phase = fill & 1u;
+          // A warp hops between stages, so it has not seen the previous fill of this one, and the
+          // parity of `full` alone cannot tell "fill n landed" from "fill n-1 still in flight".
+          // Waiting first until the MMAs have retired fill n-1 (the same condition the producer
+          // waits for before it issues fill n, so no time is lost) leaves only "fill n pending"
+          // or "fill n landed".
+          if (fill > 0 && !ptx::mbar_wait(&empty[stage], phase ^ 1, abort_flag, P.wait_limit)) { ok = false; break; }
           if (!ptx::mbar_wait(&full[stage], phase, abort_flag, P.wait_limit)) { ok = false; break; }
           const int ex = ks / P.tsteps;
           const float r = __ldg(P.clip + ex);

@@ -27,7 +27,8 @@ struct DirectLayerPlan {
 };
 
 struct GhostPlan {
-  int ntp = 0;                          // 128 x 128 tile pairs (ti <= tj) of a T x T Gram matrix
+  bool pair = false;                    // T > 128: 256 x 256 tiles on CTA pairs (two partial sums per item)
+  int ntp = 0;                          // tile pairs (ti <= tj) of a T x T Gram matrix
   int n_per = 0;                        // partial sums per example over all layers
   std::vector<GhostLayerPlan> layer;    // indexed like the caller's layer array
   std::vector<DirectLayerPlan> direct;  // indexed like the caller's layer array
@@ -38,6 +39,9 @@ struct GhostPlan {
 
 // T*T > d*p selects DIRECT under AUTO (strict), otherwise GHOST.
 GhostPlan plan_ghost_norms(const dp_linear_desc* layers, int n_layers, int B, int T, int sms);
+
+dp_status launch_ghost_norm_pair(const dp_linear_desc* layers, const GhostPlan& plan, int B, int T,
+                                 float* partials, int* dev_status, cudaStream_t st);
 
 dp_status launch_ghost_norm_tc(const dp_linear_desc* layers, const GhostPlan& plan, int B, int T,
                                float* partials, int* dev_status, cudaStream_t st);

@@ -815,3 +815,26 @@ def test_sort_in_its_own_call_then_sorted_scatter(B, T, d, V, beta):
     _, R = O.clip_factors(sq.cpu().numpy().astype(np.float64), Cc)
     want = O.clipped_sum_embed(ids, G.widened(), R, V) + beta * out0.cpu().numpy().astype(np.float64)
     assert frob_rel(two.cpu().numpy(), want) < 1e-5
+
+
+@pytest.mark.parametrize("B,T,d,p,ldg", [(2, 200, 192, 320, None), (1, 384, 128, 64, None), (3, 512, 256, 1024, None),
+                                          (2, 300, 128, 5003, 5008), (2, 257, 72, 136, None)])
+def test_pair_and_single_cta_gram_kernels_agree(B, T, d, p, ldg):
+    """T > 128 runs on CTA pairs (256 x 256 Gram tiles); the single-CTA kernel (128 x 128 tiles)
+    computes the same sum in another order.  Both against the oracle, and against each other."""
+    A, G = host_linear(B, T, d, p, "bf16", seed=7 * T + p, ldg=ldg)
+    want = O.linear_sq_norms(A.widened(), G.widened())
+    got = {}
+    for single in (False, True):
+        prev = dp.dp_debug_ghost_single(single)
+        try:
+            sq = torch.zeros(B, device=dev())
+            st = torch.zeros(1, dtype=torch.int32, device=dev())
+            dp.dp_ghost_norms([dev_linear(A, G, dp.DP_NORM_GHOST)], B, T, sq, dev_status=st)
+            torch.cuda.synchronize()
+            check_status(st)
+        finally:
+            dp.dp_debug_ghost_single(prev)
+        got[single] = sq.cpu().numpy()
+        assert rel(got[single], want).max() < TIGHT_BF16, single
+    assert rel(got[False], got[True]).max() < 1e-5
