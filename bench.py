@@ -236,8 +236,14 @@ def run_ours(args):
         else:
             P.clip_phase(ds, gemm_events=ge)
             if ev: ev[2].record(stream)
-            reduce_sums()
-            P.noise_phase(ds, seed=args.seed, step=k)
+            if world > 1 and args.exchange == "reduce_scatter":
+                # each rank noises only the slice it owns (same stream as a single-GPU draw)
+                parallel.reduce_scatter_then_noise(
+                    ds.outs, lambda t, first, tid: dp.dp_add_noise_slice(
+                        t, first, ds.sigma, ds.C, 1.0, args.seed, tid, k))
+            else:
+                reduce_sums()
+                P.noise_phase(ds, seed=args.seed, step=k)
         if ev: ev[3].record(stream)
 
     # default at N = 1: the whole step captured once as a CUDA graph and replayed (the noise step
@@ -485,6 +491,8 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--exchange", default="all_reduce", choices=["all_reduce", "reduce_scatter"],
+                    help="N > 1: how the clipped sums are summed over ranks before the noise draw")
     ap.add_argument("--eager", action="store_true",
                     help="issue the step call by call instead of replaying a captured CUDA graph")
     ap.add_argument("--workload", default="cfg2")
