@@ -838,3 +838,44 @@ def test_pair_and_single_cta_gram_kernels_agree(B, T, d, p, ldg):
         got[single] = sq.cpu().numpy()
         assert rel(got[single], want).max() < TIGHT_BF16, single
     assert rel(got[False], got[True]).max() < 1e-5
+
+
+def test_pair_gram_kernel_wide_input_side_and_many_layers():
+    """CTA-pair Gram kernel: the WIDE operand is the layer input (its columns are chunked across
+    work items, each recomputing the narrow Gram), and more layers than one launch holds."""
+    B, T = 2, 300
+    # (a) d >> p: the split runs over A's columns
+    rng = np.random.default_rng(5)
+    A = W._normal((B, T, 5003), 1.0, "bf16", int(rng.integers(1 << 60)), ld=5008)
+    G = W._normal((B, T, 128), 1e-2, "bf16", int(rng.integers(1 << 60)))
+    sq = torch.zeros(B, device=dev())
+    st = torch.zeros(1, dtype=torch.int32, device=dev())
+    dp.dp_ghost_norms([dev_linear(A, G, dp.DP_NORM_GHOST)], B, T, sq, dev_status=st)
+    torch.cuda.synchronize()
+    check_status(st)
+    assert rel(sq.cpu().numpy(), O.linear_sq_norms(A.widened(), G.widened())).max() < TIGHT_BF16
+    # (b) 100 small layers: two launches of the pair kernel, one sum
+    layers, want = [], np.zeros(B)
+    for k in range(100):
+        Ak, Gk = host_linear(B, T, 64, 72, "bf16", seed=1000 + k)
+        layers.append(dev_linear(Ak, Gk, dp.DP_NORM_GHOST))
+        want += O.linear_sq_norms(Ak.widened(), Gk.widened())
+    sq = torch.zeros(B, device=dev())
+    dp.dp_ghost_norms(layers, B, T, sq, dev_status=st)
+    torch.cuda.synchronize()
+    check_status(st)
+    assert rel(sq.cpu().numpy(), want).max() < TIGHT_BF16
+
+
+def test_step_graph_with_positions_and_full_parameter_set():
+    """Graph replays of a step that has a position table and every bias / LayerNorm parameter."""
+    w = W.named_workload("cfg3", B=2, T=200, n_blocks=1, V=3001, full_model=True)
+    a, b = P.upload(w), P.upload(w)
+    g = P.StepGraph(a, seed=21, first_step=0)
+    for k in range(2):
+        g.replay()
+        P.dp_step(b, seed=21, step=k)
+        torch.cuda.synchronize()
+        check_status(a.dev_status)
+        for name in a.outs:
+            assert torch.equal(a.outs[name], b.outs[name]), (k, name)
