@@ -21,10 +21,11 @@ namespace dpg {
 namespace {
 
 constexpr int kVecCols = 256;        // columns per block (8 per lane)
-// 16-byte row loads in flight per lane: four G rows for a bias, two G and two X rows for a
-// LayerNorm gain, so that four 256-thread blocks (<= 64 registers per thread) fit on an SM
-constexpr int kVecBatchBias = 4;
-constexpr int kVecBatchGain = 2;
+// 16-byte row loads in flight per lane: eight G rows for a bias, four G and four X rows for a
+// LayerNorm gain (kept unconverted: 32 registers), so that four 256-thread blocks
+// (<= 64 registers per thread) fit on an SM
+constexpr int kVecBatchBias = 8;
+constexpr int kVecBatchGain = 4;
 
 struct VecParam {
   const void* G;
@@ -49,40 +50,93 @@ __device__ __forceinline__ int find_param(const VecParams& P, int slab) {
   return k;
 }
 
-// sum over the rows [r0, r1) (stride 8 from warp w) of weight(row) * G[row, cols] * X[row, cols]
+// Eight consecutive columns of one row, kept as loaded (a bf16 row chunk stays one 16-byte
+// register quad until it is consumed, so twice as many loads fit in flight per thread).
+template <typename T> struct Raw8;
+template <> struct Raw8<__nv_bfloat16> {
+  uint4 q;
+  __device__ __forceinline__ void load(const __nv_bfloat16* p, int nvalid, bool vec) {
+    if (vec && nvalid >= 8) {
+      q = *reinterpret_cast<const uint4*>(p);
+    } else {
+      uint32_t w[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+      for (int e = 0; e < 8; ++e)
+        if (e < nvalid) w[e >> 1] |= uint32_t(__bfloat16_as_ushort(p[e])) << (16 * (e & 1));
+      q = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  }
+  __device__ __forceinline__ void unpack(float (&v)[8]) const {
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      v[2 * e] = __uint_as_float(w[e] << 16);
+      v[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+    }
+  }
+};
+template <> struct Raw8<float> {
+  float v8[8];
+  __device__ __forceinline__ void load(const float* p, int nvalid, bool vec) { load8<float>(p, nvalid, vec, v8); }
+  __device__ __forceinline__ void unpack(float (&v)[8]) const {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[e] = v8[e];
+  }
+};
+
+// sum over the rows [r0, r1) (stride 8 from warp w) of weight(row) * G[row, cols] * X[row, cols].
+// All loads of a batch are issued before any is consumed; rows past r1 re-read row r1-1 with
+// weight 0, so the loads are unconditional.  The example of a row (for its clip factor) is
+// tracked by stepping, not by a division per row.
 template <typename T, bool kWeighted, bool kHasX>
 __device__ __forceinline__ void stream_rows_t(const VecParam& q, long long row_base, int r0, int r1,
                                               int c, int nvalid, int Tn, const float* clip,
                                               float (&acc)[8]) {
-  constexpr int kBatch = kHasX ? kVecBatchGain : kVecBatchBias;
+  // fp32 chunks are twice as large in registers: half the batch
+  constexpr int kBatch = (kHasX ? kVecBatchGain : kVecBatchBias) / (sizeof(T) == 2 ? 1 : 2);
   const int w = threadIdx.x >> 5;
+  if (r0 + w >= r1) return;
   const T* G = static_cast<const T*>(q.G) + row_base * q.ldg + c;
   const T* X = kHasX ? static_cast<const T*>(q.X) + row_base * q.ldx + c : nullptr;
   const bool gvec = ((reinterpret_cast<uintptr_t>(q.G) & 15) == 0) && ((q.ldg * sizeof(T)) % 16 == 0);
   const bool xvec = kHasX && ((reinterpret_cast<uintptr_t>(q.X) & 15) == 0) && ((q.ldx * sizeof(T)) % 16 == 0);
+  // example and token of the first row this warp takes
+  long long ex = kWeighted ? (row_base + r0 + w) / Tn : 0;
+  int t = kWeighted ? int((row_base + r0 + w) - ex * Tn) : 0;
   for (int rr = r0 + w; rr < r1; rr += 8 * kBatch) {
-    float g[kBatch][8], x[kHasX ? kBatch : 1][8], wt[kBatch];
+    Raw8<T> g[kBatch], x[kHasX ? kBatch : 1];
+    float wt[kBatch];
 #pragma unroll
     for (int b = 0; b < kBatch; ++b) {
       const int r = rr + 8 * b;
-      if (r < r1) {
-        load8<T>(G + size_t(r) * q.ldg, nvalid, gvec, g[b]);
-        if (kHasX) load8<T>(X + size_t(r) * q.ldx, nvalid, xvec, x[kHasX ? b : 0]);
-        wt[b] = kWeighted ? clip[(row_base + r) / Tn] : 1.f;
-      } else {
-        wt[b] = 0.f;
-#pragma unroll
-        for (int e = 0; e < 8; ++e) g[b][e] = 0.f;
-      }
+      const int rc = min(r, r1 - 1);
+      g[b].load(G + size_t(rc) * q.ldg, nvalid, gvec);
+      if (kHasX) x[kHasX ? b : 0].load(X + size_t(rc) * q.ldx, nvalid, xvec);
     }
 #pragma unroll
     for (int b = 0; b < kBatch; ++b) {
-      if (rr + 8 * b < r1) {
+      float f = 1.f;
+      if (kWeighted) {
+        long long eb = ex;
+        int tb = t + 8 * b;
+        while (tb >= Tn) { tb -= Tn; ++eb; }
+        f = (rr + 8 * b < r1) ? __ldg(clip + eb) : 0.f;      // eb < B whenever the row exists
+      }
+      wt[b] = (rr + 8 * b < r1) ? f : 0.f;
+    }
+    if (kWeighted) {
+      t += 8 * kBatch;
+      while (t >= Tn) { t -= Tn; ++ex; }
+    }
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const float v = kHasX ? g[b][e] * x[kHasX ? b : 0][e] : g[b][e];
-          acc[e] = kWeighted ? fmaf(wt[b], v, acc[e]) : acc[e] + v;
-        }
+    for (int b = 0; b < kBatch; ++b) {
+      float gv[8], xv[8];
+      g[b].unpack(gv);
+      if (kHasX) x[kHasX ? b : 0].unpack(xv);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const float v = kHasX ? gv[e] * xv[e] : gv[e];
+        acc[e] = fmaf(wt[b], v, acc[e]);
       }
     }
   }

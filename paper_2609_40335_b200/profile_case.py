@@ -1,6 +1,6 @@
 """Small single-kernel cases for profilers (each runs one entry point a few times on cuda:0).
 
-    python -m paper_2609_40335_b200.profile_case gemm|ghost|noise|embed|cross [reps]
+    python -m paper_2609_40335_b200.profile_case gemm|ghost|ghost512|noise|embed|embed_small|cross|vectors [reps]
 
 Sizes are chosen so that inputs exceed the 126 MB L2 but stay well under a few GB, which keeps
 a multi-pass `ncu` capture short.
@@ -134,12 +134,28 @@ def case_cross(reps):
         dp.dp_tied_cross_term(ids, G_emb, A_lm, G_lm, V, sq=sq, d=d)
 
 
+def case_vectors(reps):
+    """Bias and LayerNorm parameters of 6 GPT-2 blocks at B=32, T=128 (norms, then clipped sums)."""
+    B, T = 32, 128
+    vec = []
+    for _ in range(6):
+        for p_, with_x in [(768, True), (768, False), (2304, False), (768, False), (768, True), (768, False),
+                           (3072, False), (768, False)]:
+            G = _randn_bf16(B, T, p_, std=1e-2)
+            vec.append(dp.Vector(G, _randn_bf16(B, T, p_) if with_x else None, p=p_))
+    sq = torch.zeros(B, device="cuda")
+    outs = [torch.empty(v.p, device="cuda") for v in vec]
+    for _ in range(reps):
+        dp.dp_vector_norms(vec, B, T, sq)
+        dp.dp_clip_accumulate_vectors(vec, B, T, sq, 1.0, outs)
+
+
 def main():
     which = sys.argv[1] if len(sys.argv) > 1 else "gemm"
     reps = int(sys.argv[2]) if len(sys.argv) > 2 else 3
     torch.manual_seed(0)
     {"gemm": case_gemm, "gemm1": case_gemm_unclipped, "ghost512": case_ghost_long, "overlap": case_overlap, "ghost": case_ghost, "noise": case_noise, "embed": case_embed, "embed_small": case_embed_small,
-     "cross": case_cross}[which](reps)
+     "cross": case_cross, "vectors": case_vectors}[which](reps)
     torch.cuda.synchronize()
     print("done", which, reps)
 
