@@ -879,3 +879,90 @@ def test_step_graph_with_positions_and_full_parameter_set():
         check_status(a.dev_status)
         for name in a.outs:
             assert torch.equal(a.outs[name], b.outs[name]), (k, name)
+
+
+# ------------------------------- full-size configurations in the launch configuration of the bench
+def _full_size_graph_check(w, examples, layers, lm_rows, table_rows, seed=7, first_step=3):
+    """One replay of the captured step graph (what bench.py times) at full size; the oracle checks
+    sampled outputs: norms (and cross terms) of `examples`, clip factors of all, the noised clipped
+    sums of `layers`, of rows `lm_rows` of the head and rows `table_rows` of the token table."""
+    ds = P.upload(w)
+    g = P.StepGraph(ds, seed=seed, first_step=first_step)
+    g.replay()
+    torch.cuda.synchronize()
+    check_status(ds.dev_status)
+    step = first_step                                        # replay k draws step first_step + k
+    tid = P.tensor_ids(ds)
+    sq_gpu = ds.sq.cpu().numpy().astype(np.float64)
+    for i in examples:
+        sl = slice(i, i + 1)
+        lin = [(l.A.widened_rows(sl), l.G.widened_rows(sl)) for l in w.linears]
+        ref = O.dp_step(lin, w.ids[sl], w.G_emb.widened_rows(sl), w.V, w.C,
+                        lm=(w.lm.A.widened_rows(sl), w.lm.G.widened_rows(sl)), tied=w.tied,
+                        positions=w.positions, want_sums=False)
+        assert abs(sq_gpu[i] - ref["sq"][0]) / ref["sq"][0] < TIGHT_BF16, i
+        if w.tied:
+            scale = np.sqrt(ref["sq_in"][0] * ref["sq_out"][0])
+            assert abs(ds.cross.cpu().numpy()[i] - ref["cross"][0]) / scale < TIGHT_BF16, i
+    _, R = O.clip_factors(sq_gpu, w.C)                       # Eq. 7 from the (checked) norms
+    assert rel(ds.clip.cpu().numpy(), R).max() < 1e-5
+    amp = w.sigma * w.C
+
+    def noise(name, n, start=0):
+        return amp * NO.standard_normals(n, seed, tid[name], step, start=start)
+
+    for k in layers:
+        l = w.linears[k]
+        want = O.clipped_sum_linear(l.A.widened(), l.G.widened(), R)
+        want = want + noise(f"linear{k}", want.size).reshape(want.shape)
+        assert frob_rel(ds.outs[f"linear{k}"].cpu().numpy(), want) < 5e-3, k
+    # sampled rows of the head (its own matrix, or the shared table when tied)
+    d = w.d_model
+    head = "wte" if w.tied else "lm_head"
+    rows = np.array(lm_rows)
+    Gs = W.bf16_bits_to_f32(w.lm.G.data[:, :, rows]).astype(np.float64)
+    want = O.clipped_sum_linear(w.lm.A.widened(), Gs, R)
+    emb = O.clipped_sum_embed(w.ids, w.G_emb.widened(), R, w.V)
+    if w.tied:
+        want = want + emb[rows]                              # one table receives both (Eq. 8)
+    for j, r_ in enumerate(rows):
+        want[j] += noise(head, d, start=int(r_) * d)
+    assert frob_rel(ds.outs[head].cpu().numpy()[rows], want) < 5e-3
+    if not w.tied:
+        trow = np.array(table_rows)
+        want_t = emb[trow]
+        for j, r_ in enumerate(trow):
+            want_t[j] += noise("wte", d, start=int(r_) * d)
+        assert frob_rel(ds.outs["wte"].cpu().numpy()[trow], want_t) < 5e-3
+    if w.positions:
+        pos_ids = np.tile(np.arange(w.T), (w.B, 1))
+        want_p = O.clipped_sum_embed(pos_ids, w.G_emb.widened(), R, w.T)
+        want_p = want_p + noise("wpe", want_p.size).reshape(want_p.shape)
+        assert frob_rel(ds.outs["wpe"].cpu().numpy()[: w.T], want_p) < 5e-3
+
+
+HEAD_ROWS = [0, 1, 255, 256, 25000, 50175, 50176, 50256]
+
+
+def test_cfg2_full_size_graph_replay_sampled():
+    w = W.named_workload("cfg2")
+    hot = [int(np.bincount(w.ids.reshape(-1)).argmax()), int(w.ids[0, 0]), 0, 50256]
+    _full_size_graph_check(w, examples=(0, 31), layers=(0, 23), lm_rows=HEAD_ROWS, table_rows=hot)
+
+
+def test_cfg4_full_size_tied_graph_replay_sampled():
+    w = W.named_workload("cfg4")
+    hot = [int(np.bincount(w.ids.reshape(-1)).argmax())]
+    _full_size_graph_check(w, examples=(5,), layers=(2, 47), lm_rows=HEAD_ROWS + hot, table_rows=[])
+
+
+def test_cfg3_full_size_graph_replay_sampled():
+    w = W.named_workload("cfg3")                             # B = 64, T = 256: the CTA-pair Gram kernel
+    hot = [int(np.bincount(w.ids.reshape(-1)).argmax()), 50256]
+    _full_size_graph_check(w, examples=(63,), layers=(1,), lm_rows=HEAD_ROWS[:4], table_rows=hot)
+
+
+def test_cfg5_cell_full_size_graph_replay_sampled():
+    w = W.named_workload("cfg5", B=16, T=128)                # GPT-2-medium shape, 97 layers
+    hot = [int(np.bincount(w.ids.reshape(-1)).argmax())]
+    _full_size_graph_check(w, examples=(7,), layers=(3, 95), lm_rows=HEAD_ROWS[:4], table_rows=hot)
