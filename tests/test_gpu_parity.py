@@ -966,3 +966,47 @@ def test_cfg5_cell_full_size_graph_replay_sampled():
     w = W.named_workload("cfg5", B=16, T=128)                # GPT-2-medium shape, 97 layers
     hot = [int(np.bincount(w.ids.reshape(-1)).argmax())]
     _full_size_graph_check(w, examples=(7,), layers=(3, 95), lm_rows=HEAD_ROWS[:4], table_rows=hot)
+
+
+@pytest.mark.parametrize("B,T", [(64, 512), (256, 128), (256, 512)])
+def test_cfg5_large_cells_against_library_gemms_on_the_device(B, T):
+    """GPT-2-medium cells too large for the CPU oracle (inputs drawn on the device): sampled
+    quantities are recomputed with plain library matrix products in float64 / fp32 on the GPU --
+    the definition ||G_i^T A_i||_F^2 for sampled (example, layer) pairs, and sum_i R_i G_i^T A_i for a
+    sampled layer -- and the whole step must be bitwise reproducible."""
+    ds = P.synthesize_on_device("cfg5", B, T, 1024, 24, seed=3)
+    P.dp_step(ds, seed=5, step=1)
+    torch.cuda.synchronize()
+    check_status(ds.dev_status)
+    sq1 = ds.sq.clone()
+    out1 = ds.outs["linear2"].clone()
+    every = ds.linears + [ds.lm]
+    # (a) per-example norm: all layers of one example, by definition, in float64 on the device
+    i = B // 3
+    want = 0.0
+    for l in every:
+        A = l.A[i, :, : l.d].double()
+        G = l.G[i, :, : l.p].double()
+        if l.p > 8192:                                       # the head: through the Gram identity's
+            want += float(((A @ A.T) * (G @ G.T)).sum())     # T x T form (the p x d matrix is 0.4 GB)
+        else:
+            want += float((G.T @ A).pow(2).sum())
+    ids = ds.ids[i].long()
+    Ge = ds.G_emb[i, :, : ds.d_model].double()
+    want += float(((ids[:, None] == ids[None, :]).double() * (Ge @ Ge.T)).sum())
+    assert abs(float(sq1[i]) - want) / want < TIGHT_BF16
+    # (b) clipped sum of one layer against a library GEMM with the rows scaled by R_i (fp32)
+    R = torch.clamp(ds.C / ds.sq.sqrt(), max=1.0)
+    l = ds.linears[2]
+    Gs = (l.G[..., : l.p].float() * R[:, None, None]).reshape(-1, l.p)
+    ref = Gs.T @ l.A[..., : l.d].float().reshape(-1, l.d)
+    amp = ds.sigma * ds.C
+    z = torch.zeros_like(ref)
+    dp.dp_add_noise(z, ds.sigma, ds.C, 1.0, 5, P.tensor_ids(ds)["linear2"], 1)
+    torch.cuda.synchronize()
+    assert float((out1 - (ref + z)).norm() / (ref + z).norm()) < 5e-3
+    assert amp > 0
+    # (c) the step is deterministic
+    P.dp_step(ds, seed=5, step=1)
+    torch.cuda.synchronize()
+    assert torch.equal(ds.sq, sq1) and torch.equal(ds.outs["linear2"], out1)
