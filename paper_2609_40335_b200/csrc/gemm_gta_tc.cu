@@ -119,6 +119,23 @@ __device__ __forceinline__ Item decode_item(const GtaParams& P, int item) {
   return it;
 }
 
+// In-register transpose of a 32 x 32 tile held one row per lane: afterwards v[j] of lane l is
+// what v[l] of lane j was (five butterfly stages of 16 exchanges).
+__device__ __forceinline__ void warp_transpose32(float (&v)[32], int lane) {
+#pragma unroll
+  for (int d = 16; d >= 1; d >>= 1) {
+    const bool up = (lane & d) != 0;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      if ((j & d) == 0) {
+        const float send = up ? v[j] : v[j + d];
+        const float recv = __shfl_xor_sync(0xffffffffu, send, d);
+        if (up) v[j] = recv; else v[j + d] = recv;
+      }
+    }
+  }
+}
+
 template <bool kScale, bool kSqsum, bool kPair>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_gta_kernel(const __grid_constant__ GtaParams P) {
@@ -370,47 +387,53 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
           ptx::tmem_ld_32x32b_x32(t0 + c * 32, r);
           ptx::tmem_ld_wait();
           const int col0 = it.tn * kBN + c * 32;
-          if (row < L.M && col0 < L.N) {
-            float* o = dst + size_t(row) * ld + col0;
-            const bool full32 = col0 + 32 <= L.N;
+          const int row_base = row - lane;                   // first row of this warp's 32
+          if (row_base < L.M && col0 < L.N) {                // the same for the whole warp
             float v[32];
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-            if (beta != 0.f) {
-              if (vec_ok && full32) {
+            if (row < L.M) {
+              const bool full32 = col0 + 32 <= L.N;
+              if (beta != 0.f) {
+                const float* o = dst + size_t(row) * ld + col0;
+                if (vec_ok && full32) {
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                  const float4 old = *reinterpret_cast<const float4*>(o + 4 * j);
-                  v[4 * j] += old.x; v[4 * j + 1] += old.y; v[4 * j + 2] += old.z; v[4 * j + 3] += old.w;
-                }
-              } else {
+                  for (int j = 0; j < 8; ++j) {
+                    const float4 old = *reinterpret_cast<const float4*>(o + 4 * j);
+                    v[4 * j] += old.x; v[4 * j + 1] += old.y; v[4 * j + 2] += old.z; v[4 * j + 3] += old.w;
+                  }
+                } else {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) if (col0 + j < L.N) v[j] += o[j];
-              }
-            }
-            if (noisy) {
-              const unsigned long long j0 = (unsigned long long)row * L.N + col0;   // stream index
-              // N is a multiple of 4 here (the host fuses only such layers), so the Philox
-              // counters of this thread's 32 columns never straddle a row
-#pragma unroll
-              for (int qd = 0; qd < 8; ++qd) {
-                if (col0 + 4 * qd < L.N) {
-                  float z[4];
-                  normals4((j0 >> 2) + qd, nkey, z);
-#pragma unroll
-                  for (int e = 0; e < 4; ++e)
-                    v[4 * qd + e] = noised(v[4 * qd + e], z[e], L.noise_amp, P.noise_scale);
+                  for (int j = 0; j < 32; ++j) if (col0 + j < L.N) v[j] += o[j];
                 }
               }
+              if (noisy) {
+                const unsigned long long j0 = (unsigned long long)row * L.N + col0;   // stream index
+                // N is a multiple of 4 here (the host fuses only such layers), so the Philox
+                // counters of this thread's 32 columns never straddle a row
+#pragma unroll
+                for (int qd = 0; qd < 8; ++qd) {
+                  if (col0 + 4 * qd < L.N) {
+                    float z[4];
+                    normals4((j0 >> 2) + qd, nkey, z);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                      v[4 * qd + e] = noised(v[4 * qd + e], z[e], L.noise_amp, P.noise_scale);
+                  }
+                }
+              }
             }
-            if (vec_ok && full32) {
+            // Stores by whole rows: with one row per lane a warp store would touch 32 different
+            // 128-byte lines, 16 bytes each -- measured, those write requests took a fifth of the
+            // kernel's throughput away from the operand loads.  After the transpose lane l holds
+            // column col0 + l of the 32 rows and every store is one 128-byte line.
+            warp_transpose32(v, lane);
+            const int col = col0 + lane;
+            if (col < L.N) {
+              float* o = dst + size_t(row_base) * ld + col;
 #pragma unroll
-              for (int j = 0; j < 8; ++j)
-                *reinterpret_cast<float4*>(o + 4 * j) =
-                    make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j) if (col0 + j < L.N) o[j] = v[j];
+              for (int j = 0; j < 32; ++j)
+                if (row_base + j < L.M) __stcs(o + size_t(j) * ld, v[j]);   // written once: evict first
             }
           }
         }
