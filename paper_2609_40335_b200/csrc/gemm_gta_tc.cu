@@ -119,11 +119,14 @@ __device__ __forceinline__ Item decode_item(const GtaParams& P, int item) {
   return it;
 }
 
-// In-register transpose of a 32 x 32 tile held one row per lane: afterwards v[j] of lane l is
-// what v[l] of lane j was (five butterfly stages of 16 exchanges).
-__device__ __forceinline__ void warp_transpose32(float (&v)[32], int lane) {
+// Partial in-register transpose of a 32 x 32 tile held one row per lane (v[c] = column c): the
+// upper three lane bits are exchanged with the upper three register bits (three butterfly stages
+// of 16 exchanges).  Afterwards lane l holds, in v[4i .. 4i+3], columns 4(l>>2) .. +3 of row
+// 4i + (l&3): four consecutive columns per register quad, and the 32 lanes of quad i cover rows
+// 4i .. 4i+3 completely -- one float4 store per quad writes four whole 128-byte lines.
+__device__ __forceinline__ void warp_transpose_quads(float (&v)[32], int lane) {
 #pragma unroll
-  for (int d = 16; d >= 1; d >>= 1) {
+  for (int d = 16; d >= 4; d >>= 1) {
     const bool up = (lane & d) != 0;
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
@@ -423,17 +426,29 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
                 }
               }
             }
-            // Stores by whole rows: with one row per lane a warp store would touch 32 different
+            // Stores by whole lines: with one row per lane a warp store would touch 32 different
             // 128-byte lines, 16 bytes each -- measured, those write requests took a fifth of the
-            // kernel's throughput away from the operand loads.  After the transpose lane l holds
-            // column col0 + l of the 32 rows and every store is one 128-byte line.
-            warp_transpose32(v, lane);
-            const int col = col0 + lane;
-            if (col < L.N) {
-              float* o = dst + size_t(row_base) * ld + col;
+            // kernel's throughput away from the operand loads.  After the partial transpose every
+            // float4 store of the warp writes four complete rows of this 32-column chunk.
+            warp_transpose_quads(v, lane);
+            const int colq = col0 + 4 * (lane >> 2);         // this lane's four columns
+            const int rsub = lane & 3;
+            if (vec_ok && col0 + 32 <= L.N) {
 #pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (row_base + j < L.M) __stcs(o + size_t(j) * ld, v[j]);   // written once: evict first
+              for (int i = 0; i < 8; ++i) {
+                const int rr = row_base + 4 * i + rsub;
+                if (rr < L.M)
+                  __stcs(reinterpret_cast<float4*>(dst + size_t(rr) * ld + colq),
+                         make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]));
+              }
+            } else {
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const int rr = row_base + 4 * i + rsub;
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                  if (rr < L.M && colq + e < L.N) dst[size_t(rr) * ld + colq + e] = v[4 * i + e];
+              }
             }
           }
         }
