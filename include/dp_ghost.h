@@ -163,6 +163,14 @@ size_t dp_tied_cross_term_ws_bytes(int32_t B, int32_t T, int32_t d, int32_t V);
  * norms [dev, B or NULL] receives sqrt(sq[i]).  C > 0 and finite. */
 dp_status dp_clip_factors(const float* sq, int32_t B, float C, float* clip, float* norms,
                           void* stream);
+/* The same after joining a second accumulator: sq[i] += sq_extra[i] (one addition, fixed order),
+ * then clip and norms from the sum.  For norm calls that ran on two streams into two
+ * accumulators.  clip, norms [dev, B or NULL]. */
+dp_status dp_clip_factors_sum(float* sq, const float* sq_extra, int32_t B, float C, float* clip,
+                              float* norms, void* stream);
+/* In every dp_clip_accumulate* call below, sq may be NULL: `clip` [dev, B] then is an INPUT that
+ * already holds the factors R_i (from dp_clip_factors / dp_clip_factors_sum), and the call does
+ * not recompute them -- one kernel less per call when a step makes several. */
 
 /* ---- clipped sum of a linear layer: out = beta*out + sum_i R_i G_i^T A_i  (Eq. 3) ----
  * One GEMM with M = p, N = d, K = B*T whose K rows are scaled by R_i = min(1, C/sqrt(sq[i]))

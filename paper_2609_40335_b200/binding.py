@@ -42,7 +42,7 @@ class _VectorDesc(C.Structure):
 EXPORTS = ["dp_vector_norms", "dp_vector_norms_ws_bytes", "dp_clip_accumulate_vectors",
            "dp_clip_accumulate_vectors_ws_bytes", "dp_ghost_norms", "dp_ghost_norms_ws_bytes", "dp_embed_norms", "dp_embed_norms_ws_bytes",
            "dp_embed_norms_static",
-           "dp_tied_cross_term", "dp_tied_cross_term_ws_bytes", "dp_clip_factors",
+           "dp_tied_cross_term", "dp_tied_cross_term_ws_bytes", "dp_clip_factors", "dp_clip_factors_sum",
            "dp_clip_accumulate", "dp_clip_accumulate_ws_bytes", "dp_clip_accumulate_grouped",
            "dp_clip_accumulate_grouped_ws_bytes", "dp_clip_accumulate_noise_grouped",
            "dp_clip_accumulate_embed_noise", "dp_clip_accumulate_embed",
@@ -88,6 +88,7 @@ def load():
     L.dp_tied_cross_term_ws_bytes.argtypes = [i32, i32, i32, i32]
     L.dp_tied_cross_term_ws_bytes.restype = sz
     L.dp_clip_factors.argtypes = [vp, i32, f32, vp, vp, vp]
+    L.dp_clip_factors_sum.argtypes = [vp, vp, i32, f32, vp, vp, vp]
     L.dp_clip_accumulate.argtypes = [vp, i64, vp, i64, i32, i32, i32, i32, i32, vp, f32, vp, vp, i64,
                                      f32, vp, sz, vp, vp]
     L.dp_clip_accumulate_ws_bytes.argtypes = [i32, i32, i32, i32, i32]
@@ -339,6 +340,14 @@ def dp_clip_factors(sq: torch.Tensor, C_: float, clip=None, norms=None, stream=N
     L = load()
     _check(L.dp_clip_factors(_ptr(sq), sq.numel(), float(C_), _ptr(clip), _ptr(norms), _stream(stream)),
            "dp_clip_factors")
+
+
+def dp_clip_factors_sum(sq: torch.Tensor, sq_extra: torch.Tensor, C_: float, clip=None, norms=None,
+                        stream=None):
+    """sq += sq_extra, then clip factors and norms from the sum (one kernel)."""
+    L = load()
+    _check(L.dp_clip_factors_sum(_ptr(sq), _ptr(sq_extra), sq.numel(), float(C_), _ptr(clip),
+                                 _ptr(norms), _stream(stream)), "dp_clip_factors_sum")
 
 
 def dp_clip_accumulate_ws_bytes(dt: int, B: int, T: int, d: int, p: int) -> int:

@@ -112,6 +112,19 @@ static dp_status check_linear(const dp_linear_desc& L, dp_dtype dt, bool tc) {
 
 using namespace dpg;
 
+// Clip factors of a clip-accumulate call.  With sq given they are computed (Eq. 7) into the
+// workspace and copied to `clip` if the caller wants them; with sq == NULL the caller has them
+// already (dp_clip_factors / dp_clip_factors_sum) and `clip` is the input.
+static dp_status resolve_clip(const float* sq, int B, float C, float* clip, float** clip_ws,
+                              cudaStream_t st) {
+  if (!sq) { *clip_ws = clip; return DP_OK; }
+  const dp_status s = launch_clip_factors(sq, B, C, *clip_ws, nullptr, st);
+  if (s != DP_OK) return s;
+  if (clip) DP_CUDA_OK(cudaMemcpyAsync(clip, *clip_ws, size_t(B) * sizeof(float),
+                                       cudaMemcpyDeviceToDevice, st));
+  return DP_OK;
+}
+
 extern "C" {
 
 const char* dp_status_string(dp_status s) {
@@ -313,7 +326,7 @@ dp_status dp_clip_accumulate_vectors(const dp_vector_desc* prm, int32_t n, dp_dt
                                      uint32_t step, void* ws, size_t ws_bytes, void* stream) {
   const dp_status c = check_vectors(prm, n, B, T);
   if (c != DP_OK) return c;
-  if (!sq || !outs || (dt != DP_F32 && dt != DP_BF16)) return DP_ERR_INVALID_ARG;
+  if ((!sq && !clip) || !outs || (dt != DP_F32 && dt != DP_BF16)) return DP_ERR_INVALID_ARG;
   if (!(beta == 0.f || beta == 1.f) || !finite_pos(C)) return DP_ERR_INVALID_ARG;
   for (int k = 0; k < n; ++k) if (!outs[k]) return DP_ERR_INVALID_ARG;
   if (with_noise && (!tensor_ids || !std::isfinite(sigma) || sigma < 0.f || !std::isfinite(scale)))
@@ -321,10 +334,8 @@ dp_status dp_clip_accumulate_vectors(const dp_vector_desc* prm, int32_t n, dp_dt
   if (!ws || ws_bytes < dp_clip_accumulate_vectors_ws_bytes(prm, n, B, T)) return DP_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   float* clip_ws = static_cast<float*>(ws);
-  dp_status s = launch_clip_factors(sq, B, C, clip_ws, nullptr, st);
+  dp_status s = resolve_clip(sq, B, C, clip, &clip_ws, st);
   if (s != DP_OK) return s;
-  if (clip) DP_CUDA_OK(cudaMemcpyAsync(clip, clip_ws, size_t(B) * sizeof(float),
-                                       cudaMemcpyDeviceToDevice, st));
   float* partial = reinterpret_cast<float*>(static_cast<char*>(ws) +
                                             align_up(size_t(B) * sizeof(float), 256));
   return launch_vector_sums(prm, n, dt, B, T, clip_ws, outs, beta, with_noise ? 1 : 0, sigma * C,
@@ -332,6 +343,12 @@ dp_status dp_clip_accumulate_vectors(const dp_vector_desc* prm, int32_t n, dp_dt
 }
 
 // --------------------------------------------------------------------------- clip factors
+dp_status dp_clip_factors_sum(float* sq, const float* sq_extra, int32_t B, float C, float* clip,
+                              float* norms, void* stream) {
+  if (!sq || !sq_extra || B <= 0 || !finite_pos(C)) return DP_ERR_INVALID_ARG;
+  return launch_clip_factors(sq, B, C, clip, norms, (cudaStream_t)stream, sq_extra, sq);
+}
+
 dp_status dp_clip_factors(const float* sq, int32_t B, float C, float* clip, float* norms,
                           void* stream) {
   if (!sq || B <= 0 || (!clip && !norms) || !finite_pos(C)) return DP_ERR_INVALID_ARG;
@@ -352,7 +369,7 @@ static dp_status clip_accumulate_impl(const dp_linear_desc* layers, int32_t n_la
                                       float* const* outs, const int64_t* ldos, float beta,
                                       const GtaNoise* noise, void* ws, size_t ws_bytes,
                                       int32_t* dev_status, void* stream) {
-  if (!layers || n_layers <= 0 || !outs || !ldos || !sq || B <= 0 || T <= 0) return DP_ERR_INVALID_ARG;
+  if (!layers || n_layers <= 0 || !outs || !ldos || (!sq && !clip) || B <= 0 || T <= 0) return DP_ERR_INVALID_ARG;
   if (dt != DP_F32 && dt != DP_BF16) return DP_ERR_INVALID_ARG;
   if (!(beta == 0.f || beta == 1.f) || !finite_pos(C)) return DP_ERR_INVALID_ARG;
   const bool tc = (dt == DP_BF16) && !g_force_fma;
@@ -367,10 +384,8 @@ static dp_status clip_accumulate_impl(const dp_linear_desc* layers, int32_t n_la
     return DP_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
   float* clip_ws = static_cast<float*>(ws);
-  dp_status s = launch_clip_factors(sq, B, C, clip_ws, nullptr, st);
+  dp_status s = resolve_clip(sq, B, C, clip, &clip_ws, st);
   if (s != DP_OK) return s;
-  if (clip) DP_CUDA_OK(cudaMemcpyAsync(clip, clip_ws, size_t(B) * sizeof(float),
-                                       cudaMemcpyDeviceToDevice, st));
   if (!tc) {
     for (int l = 0; l < n_layers; ++l) {
       s = launch_clip_accumulate_fma(layers[l].A, layers[l].lda, layers[l].G, layers[l].ldg, dt, B, T,
@@ -474,7 +489,7 @@ static dp_status clip_accumulate_embed_impl(const int32_t* ids, const void* G, i
                                             int32_t* dev_status, void* stream,
                                             const int32_t* perm_in = nullptr,
                                             const int32_t* seg_in = nullptr) {
-  if (!ids || !G || !sq || !out || B <= 0 || T <= 0 || d <= 0 || V <= 0) return DP_ERR_INVALID_ARG;
+  if (!ids || !G || (!sq && !clip) || !out || B <= 0 || T <= 0 || d <= 0 || V <= 0) return DP_ERR_INVALID_ARG;
   if ((perm_in == nullptr) != (seg_in == nullptr)) return DP_ERR_INVALID_ARG;
   if (ldg < d || ldo < d) return DP_ERR_INVALID_ARG;
   if (dt != DP_F32 && dt != DP_BF16) return DP_ERR_INVALID_ARG;
@@ -493,10 +508,8 @@ static dp_status clip_accumulate_embed_impl(const int32_t* ids, const void* G, i
   sw.block_sums = reinterpret_cast<int*>(w + o_blk);
   sw.chunks = chunks;
   const int n = B * T;
-  dp_status s = launch_clip_factors(sq, B, C, clip_ws, nullptr, st);
+  dp_status s = resolve_clip(sq, B, C, clip, &clip_ws, st);
   if (s != DP_OK) return s;
-  if (clip) DP_CUDA_OK(cudaMemcpyAsync(clip, clip_ws, size_t(B) * sizeof(float),
-                                       cudaMemcpyDeviceToDevice, st));
   if (perm_in) {                         // sorted earlier by dp_embed_sort
     sw.perm = const_cast<int*>(perm_in);
     sw.seg = const_cast<int*>(seg_in);

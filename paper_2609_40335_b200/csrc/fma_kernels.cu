@@ -142,10 +142,15 @@ __global__ void cross_term_fma_kernel(const int* __restrict__ ids, const T* __re
 }
 
 __global__ void clip_factors_kernel(const float* __restrict__ sq, int B, float C,
-                                    float* __restrict__ clip, float* __restrict__ norms) {
+                                    float* __restrict__ clip, float* __restrict__ norms,
+                                    const float* __restrict__ extra, float* __restrict__ sq_out) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= B) return;
-  const float s = sq[i];
+  float s = sq[i];
+  if (extra) {                 // a second accumulator of squared norms joins first (fixed order)
+    s += extra[i];
+    sq_out[i] = s;
+  }
   if (clip) clip[i] = clip_from_sq(s, C);
   if (norms) norms[i] = __fsqrt_rn(s);
 }
@@ -203,8 +208,8 @@ dp_status launch_cross_term_fma(const int* ids, const void* Ge, int64_t ldge, co
 }
 
 dp_status launch_clip_factors(const float* sq, int B, float C, float* clip, float* norms,
-                              cudaStream_t st) {
-  clip_factors_kernel<<<ceil_div(B, 128), 128, 0, st>>>(sq, B, C, clip, norms);
+                              cudaStream_t st, const float* extra, float* sq_out) {
+  clip_factors_kernel<<<ceil_div(B, 128), 128, 0, st>>>(sq, B, C, clip, norms, extra, sq_out);
   DP_LAUNCH_OK();
   return DP_OK;
 }

@@ -17,7 +17,8 @@ dp_status launch_cross_term_fma(const int* ids, const void* Ge, int64_t ldge, co
                                 int T, int d, int V, float* partials, int* dev_status,
                                 cudaStream_t st);
 dp_status launch_clip_factors(const float* sq, int B, float C, float* clip, float* norms,
-                              cudaStream_t st);
+                              cudaStream_t st, const float* extra = nullptr,
+                              float* sq_out = nullptr);
 
 // embedding
 constexpr int kEmbedMaxT = 4096;

@@ -187,7 +187,7 @@ def norms_phase(ds: DeviceStep, stream=None, after_first_launch=None) -> None:
     dp.dp_clip_factors(ds.sq, ds.C, clip=ds.clip, norms=ds.norms, stream=stream)
 
 
-def _clip_vectors(ds: DeviceStep, beta: float, noise=None, stream=None) -> None:
+def _clip_vectors(ds: DeviceStep, beta: float, noise=None, stream=None, factors: bool = False) -> None:
     """Clipped sums of the bias / LayerNorm parameters (noise = (seed, step, scale) fuses Eq. 3)."""
     if not ds.vectors:
         return
@@ -197,8 +197,10 @@ def _clip_vectors(ds: DeviceStep, beta: float, noise=None, stream=None) -> None:
         seed, step, scale = noise
         tid = tensor_ids(ds)
         args = (ds.sigma, scale, seed, [tid[n] for n in names], step)
-    dp.dp_clip_accumulate_vectors(ds.vectors, ds.B, ds.T, ds.sq, ds.C, [ds.outs[n] for n in names],
-                                  beta=beta, noise=args, ws=ds.ws, stream=stream)
+    # factors=True: ds.clip already holds the clip factors of this step
+    dp.dp_clip_accumulate_vectors(ds.vectors, ds.B, ds.T, None if factors else ds.sq, ds.C,
+                                  [ds.outs[n] for n in names], beta=beta, noise=args, ws=ds.ws,
+                                  stream=stream, clip=ds.clip if factors else None)
 
 
 def clip_phase(ds: DeviceStep, stream=None, gemm_events=None) -> None:
@@ -332,21 +334,23 @@ def clip_after_prefill(ds: DeviceStep, seed: int, step: int, filled: torch.cuda.
     if layers:
         if gemm_events:
             gemm_events[0].record(torch.cuda.current_stream())
-        dp.dp_clip_accumulate_noise_grouped(layers, ds.B, ds.T, ds.sq, ds.C, [ds.outs[n] for n in names],
+        # sq=None: ds.clip already holds the factors (overlapped_norms computed them)
+        dp.dp_clip_accumulate_noise_grouped(layers, ds.B, ds.T, None, ds.C, [ds.outs[n] for n in names],
                                             ds.sigma, scale, seed, [tid[n] for n in names], step,
-                                            beta=0.0, **kw)
+                                            beta=0.0, clip=ds.clip, **kw)
         if gemm_events:
             gemm_events[1].record(torch.cuda.current_stream())
     torch.cuda.current_stream().wait_event(filled)
     # beta = 1: rows are added onto the noise (untied) or onto head sum + noise (tied); the token
     # sorts were made beside the norm phase
     sb = ds.side
-    dp.dp_clip_accumulate_embed_sorted(ds.ids, ds.G_emb, ds.V, ds.sq, ds.C, ds.outs["wte"], sb["perm"],
-                                       sb["seg"], beta=1.0, d=ds.d_model, **kw)
+    dp.dp_clip_accumulate_embed_sorted(ds.ids, ds.G_emb, ds.V, None, ds.C, ds.outs["wte"], sb["perm"],
+                                       sb["seg"], beta=1.0, d=ds.d_model, clip=ds.clip, **kw)
     if ds.positions:
-        dp.dp_clip_accumulate_embed_sorted(ds.pos_ids, ds.G_emb, WPE_ROWS, ds.sq, ds.C, ds.outs["wpe"],
-                                           sb["pos_perm"], sb["pos_seg"], beta=1.0, d=ds.d_model, **kw)
-    _clip_vectors(ds, 0.0, noise=(seed, step, scale))
+        dp.dp_clip_accumulate_embed_sorted(ds.pos_ids, ds.G_emb, WPE_ROWS, None, ds.C, ds.outs["wpe"],
+                                           sb["pos_perm"], sb["pos_seg"], beta=1.0, d=ds.d_model,
+                                           clip=ds.clip, **kw)
+    _clip_vectors(ds, 0.0, noise=(seed, step, scale), factors=True)
 
 
 def _side_buffers(ds: DeviceStep) -> dict:
@@ -406,8 +410,8 @@ def overlapped_norms(ds: DeviceStep, seed: int, step: int) -> torch.cuda.Event:
         dp.dp_tied_cross_term(ds.ids, ds.G_emb, ds.lm.A, ds.lm.G, ds.V, sq=ds.sq, cross=ds.cross,
                               d=ds.d_model, ws=ds.ws, dev_status=ds.dev_status)
     main.wait_event(normed)
-    ds.sq.add_(sb["sq"])                         # one fixed order of additions: deterministic
-    dp.dp_clip_factors(ds.sq, ds.C, clip=ds.clip, norms=ds.norms)
+    # join the two accumulators (one fixed order of additions: deterministic) and take Eq. 7
+    dp.dp_clip_factors_sum(ds.sq, sb["sq"], ds.C, clip=ds.clip, norms=ds.norms)
     return filled
 
 

@@ -1010,3 +1010,41 @@ def test_cfg5_large_cells_against_library_gemms_on_the_device(B, T):
     P.dp_step(ds, seed=5, step=1)
     torch.cuda.synchronize()
     assert torch.equal(ds.sq, sq1) and torch.equal(ds.outs["linear2"], out1)
+
+
+def test_precomputed_clip_factors_and_fused_accumulator_join():
+    """sq = None makes `clip` an input of the clip-accumulate calls; dp_clip_factors_sum joins two
+    norm accumulators and takes Eq. 7 in one kernel.  Both must equal the plain calls bit for bit."""
+    B, T, d, p, V = 5, 100, 136, 264, 777
+    A, G = host_linear(B, T, d, p, "bf16", seed=3, ldg=W.round_up(p, 8))
+    lin = dev_linear(A, G)
+    rng = np.random.default_rng(4)
+    sq_a = torch.from_numpy(rng.uniform(0.1, 3.0, B).astype(np.float32)).to(dev())
+    sq_b = torch.from_numpy(rng.uniform(0.1, 3.0, B).astype(np.float32)).to(dev())
+    # (a) the fused join
+    want_sq = sq_a + sq_b
+    clip_ref, norms_ref = torch.empty(B, device=dev()), torch.empty(B, device=dev())
+    dp.dp_clip_factors(want_sq, 1.0, clip=clip_ref, norms=norms_ref)
+    sq, clip, norms = sq_a.clone(), torch.empty(B, device=dev()), torch.empty(B, device=dev())
+    dp.dp_clip_factors_sum(sq, sq_b, 1.0, clip=clip, norms=norms)
+    torch.cuda.synchronize()
+    assert torch.equal(sq, want_sq) and torch.equal(clip, clip_ref) and torch.equal(norms, norms_ref)
+    _, R = O.clip_factors(want_sq.cpu().numpy().astype(np.float64), 1.0)
+    assert rel(clip.cpu().numpy(), R).max() < 1e-6
+    # (b) factors given instead of squared norms: linear layer, embedding, vector parameter
+    one, two = torch.empty(p, d, device=dev()), torch.empty(p, d, device=dev())
+    dp.dp_clip_accumulate_grouped([lin], B, T, want_sq, 1.0, [one])
+    dp.dp_clip_accumulate_grouped([lin], B, T, None, 1.0, [two], clip=clip)
+    ids = torch.from_numpy(W.zipf_ids(B, T, V, 1.1, 5)).to(dev())
+    Ge = P.to_device(W._normal((B, T, d), 1e-2, "bf16", 6))
+    e1, e2 = torch.empty(V, d, device=dev()), torch.empty(V, d, device=dev())
+    dp.dp_clip_accumulate_embed(ids, Ge, V, want_sq, 1.0, e1)
+    dp.dp_clip_accumulate_embed(ids, Ge, V, None, 1.0, e2, clip=clip)
+    vec = [dp.Vector(lin.G, None, p=p)]
+    v1, v2 = torch.empty(p, device=dev()), torch.empty(p, device=dev())
+    dp.dp_clip_accumulate_vectors(vec, B, T, want_sq, 1.0, [v1])
+    dp.dp_clip_accumulate_vectors(vec, B, T, None, 1.0, [v2], clip=clip)
+    torch.cuda.synchronize()
+    assert torch.equal(one, two) and torch.equal(e1, e2) and torch.equal(v1, v2)
+    with pytest.raises(dp.DpGhostError):                 # neither squared norms nor factors
+        dp.dp_clip_accumulate_grouped([lin], B, T, None, 1.0, [two])
