@@ -318,10 +318,8 @@ int32_t dp_debug_ghost_single(int32_t on);
 /* Diagnostics.  dp_debug_noise_error_scan: exhaustive float64 check of the fp32 Box-Muller
  * factors over all 2^24 inputs; out4 [dev, 4 doubles] = {max relative error of the radius for
  * r^2 <= t_max (t_max <= 0: the threshold in use), max absolute error of cos/sin, largest radius
- * seen, the compiled r^2 threshold}.  dp_debug_max_active_pairs: CTA pairs of the clipped-sum
- * kernel the device can hold. */
+ * seen, the compiled r^2 threshold}. */
 dp_status dp_debug_noise_error_scan(float t_max, double* out4, void* stream);
-int32_t dp_debug_max_active_pairs(void);
 /* Test knob for the failure path: device-side barrier waits give up after `cycles` (0: at the
  * first miss; negative: back to the default of about a second).  A kernel whose wait gives up
  * ORs DP_DEV_TIMEOUT into dev_status, lets its copies and MMAs in flight finish, frees its

@@ -50,7 +50,7 @@ EXPORTS = ["dp_vector_norms", "dp_vector_norms_ws_bytes", "dp_clip_accumulate_ve
            "dp_clip_accumulate_embed_sorted", "dp_add_noise", "dp_add_noise_slice", "dp_noise_step_device",
            "dp_fill_noise", "dp_rdp_epsilon", "dp_sigma_for_epsilon", "dp_status_string",
            "dp_last_cuda_error", "dp_version", "dp_kernel_launches", "dp_debug_force_fma",
-           "dp_debug_noise_error_scan", "dp_debug_max_active_pairs", "dp_debug_set_wait_limit",
+           "dp_debug_noise_error_scan", "dp_debug_set_wait_limit",
            "dp_debug_ghost_single"]
 
 
@@ -125,7 +125,6 @@ def load():
     L.dp_version.restype = C.c_char_p
     L.dp_kernel_launches.restype = C.c_int64
     L.dp_debug_noise_error_scan.argtypes = [f32, vp, vp]
-    L.dp_debug_max_active_pairs.restype = i32
     L.dp_debug_set_wait_limit.argtypes = [i64]
     L.dp_debug_set_wait_limit.restype = i64
     L.dp_debug_ghost_single.argtypes = [i32]

@@ -2,6 +2,9 @@
 #include <algorithm>
 #include <cmath>
 #include <cstring>
+#include <mutex>
+#include <set>
+#include <utility>
 
 #include "cross_term.cuh"
 #include "dp_common.cuh"
@@ -19,17 +22,30 @@ long long g_wait_limit = 1500000000LL;
 const uint32_t* g_step_dev = nullptr;
 int g_ghost_single = 0;
 
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_device_mutex;
+}
+
 int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0, v = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess &&
-        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
-      n = v;
+  static int n[kMaxDevices] = {};
+  int dev = 0, v = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 148;
+  if (n[dev] == 0) {
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+      n[dev] = v;
     else
       return 148;          // B200; not cached so a later call can still query the device
   }
-  return n;
+  return n[dev];
+}
+
+bool first_use_on_this_device(const void* key) {
+  static std::set<std::pair<const void*, int>> seen;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return true;     // set up again rather than never
+  std::lock_guard<std::mutex> lock(g_device_mutex);
+  return seen.insert(std::make_pair(key, dev)).second;
 }
 
 // ---- planning of dp_ghost_norms ------------------------------------------------------------
@@ -151,7 +167,6 @@ int32_t dp_debug_ghost_single(int32_t on) {
   g_ghost_single = on ? 1 : 0;
   return prev;
 }
-int32_t dp_debug_max_active_pairs(void) { return gta_max_active_pairs(); }
 int64_t dp_debug_set_wait_limit(int64_t cycles) {
   const long long prev = g_wait_limit;
   g_wait_limit = cycles < 0 ? 1500000000LL : cycles;

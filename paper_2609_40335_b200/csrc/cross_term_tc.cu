@@ -29,7 +29,7 @@ constexpr int kStageBytes = 2 * kTileBytes;          // G_emb row tile + A_lm ro
 constexpr int kStages = 6;
 constexpr int kThreads = 192;
 constexpr int kTmemCols = 256;                       // 2 accumulators x 128 columns
-constexpr size_t kSmemBytes = size_t(kStages) * kStageBytes + 1024 + 256;
+constexpr size_t kSmemBytes = size_t(kStages) * kStageBytes + 1024 + 512;
 
 struct __align__(64) CrossParams {
   CUtensorMap tmE;           // G_emb (B, T, d)
@@ -55,15 +55,17 @@ cross_term_tc_kernel(const __grid_constant__ CrossParams P) {
   uint64_t* acc_full = bars + 2 * kStages;
   uint64_t* acc_empty = acc_full + 2;
   uint64_t* mma_done = acc_empty + 2;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mma_done + 1);
+  uint64_t* red_bar = mma_done + 1;                           // [4] epilogue warps -> warp 0
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(red_bar + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  float* epi_red = reinterpret_cast<float*>(tmem_slot + 2);   // [2][4]
+  float* epi_red = reinterpret_cast<float*>(tmem_slot + 2);   // [4][4]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
     for (int b = 0; b < 2; ++b) { ptx::mbar_init(&acc_full[b], 1); ptx::mbar_init(&acc_empty[b], 4); }
     ptx::mbar_init(mma_done, 1);
+    for (int b = 0; b < 4; ++b) ptx::mbar_init(&red_bar[b], 4);
     *abort_flag = 0;
     ptx::fence_mbar_init();
   }
@@ -165,12 +167,18 @@ cross_term_tc_kernel(const __grid_constant__ CrossParams P) {
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&acc_empty[buf]);
+      // the four warps' sums meet through an mbarrier with a bounded wait (no blocking named
+      // barrier: a warp that gave up never arrives); four slots, since the other warps can run at
+      // most two items ahead of a waiting warp 0
       acc = warp_sum(acc);
-      if (lane == 0) epi_red[buf * 4 + ew] = acc;
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (ew == 0 && lane == 0)
-        P.partials[item] = (epi_red[buf * 4 + 0] + epi_red[buf * 4 + 1]) +
-                           (epi_red[buf * 4 + 2] + epi_red[buf * 4 + 3]);
+      const uint32_t slot = n_item & 3, red_phase = (n_item >> 2) & 1;
+      if (lane == 0) { epi_red[slot * 4 + ew] = acc; ptx::mbar_arrive(&red_bar[slot]); }
+      if (ew == 0) {
+        if (!ptx::mbar_wait_relaxed(&red_bar[slot], red_phase, abort_flag, P.wait_limit)) { ok = false; break; }
+        if (lane == 0)
+          P.partials[item] = (epi_red[slot * 4 + 0] + epi_red[slot * 4 + 1]) +
+                             (epi_red[slot * 4 + 2] + epi_red[slot * 4 + 3]);
+      }
     }
     if (!ok && lane == 0) {
       *abort_flag = 1;
@@ -196,12 +204,9 @@ int cross_term_tc_partials_per_example(int T) {
 dp_status launch_cross_term_tc(const int* ids, const void* Ge, int64_t ldge, const void* Al,
                                int64_t ldal, const void* Gl, int64_t ldgl, int B, int T, int d, int V,
                                float* partials, int* dev_status, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
+  if (first_use_on_this_device(reinterpret_cast<const void*>(&cross_term_tc_kernel)))
     DP_CUDA_OK(cudaFuncSetAttribute(cross_term_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)kSmemBytes));
-    attr_set = true;
-  }
   CrossParams P;
   memset(&P, 0, sizeof(P));
   dp_status s = make_tmap_bf16_3d(&P.tmE, Ge, ldge, d, T, B, kKStep, kTile);

@@ -39,8 +39,13 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
-// number of SMs of the current device (cached per process)
+// number of SMs of the current device (cached per device)
 int sm_count();
+
+// One-time set-up that CUDA keeps PER DEVICE (function attributes such as the dynamic
+// shared-memory limit): true the first time `key` is seen with the current device, false
+// afterwards.  A process that drives several GPUs gets the set-up on each of them.
+bool first_use_on_this_device(const void* key);
 
 template <typename T> __device__ __forceinline__ float to_f32(T v);
 template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
@@ -104,9 +109,14 @@ __device__ __forceinline__ void load8<float>(const float* p, int nvalid, bool ve
   }
 }
 
-// clip coefficient of Eq. 7 from a squared norm, IEEE sqrt and divide
+// Clip coefficient of Eq. 7 from a squared norm, IEEE sqrt and divide.  A zero norm gives 1
+// (nothing to clip).  The tied norm in + out + 2 cross can round to a tiny negative number when
+// the true norm is ~0: that is clamped to zero.  A squared norm that is not finite (NaN or inf
+// from corrupted inputs) gives 0 -- the example is dropped from the sum rather than added
+// unclipped, so a bad norm can never break the sensitivity bound of Eq. 2.
 __device__ __forceinline__ float clip_from_sq(float sq, float C) {
-  const float nrm = __fsqrt_rn(sq);
+  if (!(fabsf(sq) <= 3.402823466e38f)) return 0.f;       // NaN or +-inf
+  const float nrm = __fsqrt_rn(fmaxf(sq, 0.f));
   return nrm > 0.f ? fminf(1.f, __fdiv_rn(C, nrm)) : 1.f;
 }
 

@@ -465,15 +465,13 @@ dp_status launch_embed_norms(const int* ids, const void* G, int64_t ldg, dp_dtyp
                              cudaStream_t st) {
   const int slabs = ceil_div(d, kEmbedColsPerBlock);
   const size_t smem = size_t(3) * ((T + 3) & ~3) * sizeof(int);
-  static bool attr = false;
-  if (!attr) {
+  if (first_use_on_this_device(reinterpret_cast<const void*>(&launch_embed_norms))) {
     DP_CUDA_OK(cudaFuncSetAttribute(embed_norm_kernel<float>,
                                     cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     3 * kEmbedMaxT * (int)sizeof(int)));
     DP_CUDA_OK(cudaFuncSetAttribute(embed_norm_kernel<__nv_bfloat16>,
                                     cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     3 * kEmbedMaxT * (int)sizeof(int)));
-    attr = true;
   }
   if (dt == DP_F32)
     embed_norm_kernel<float><<<B * slabs, kEmbedNormThreads, smem, st>>>(ids, (const float*)G, ldg, T, d, V, slabs,

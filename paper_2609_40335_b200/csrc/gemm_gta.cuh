@@ -42,8 +42,6 @@ dp_status launch_clip_accumulate_tc(const dp_linear_desc* layers, int n_layers, 
                                     float beta, const GtaNoise* noise, float* partial_ws,
                                     int* dev_status, cudaStream_t st);
 
-int gta_max_active_pairs();
-
 dp_status launch_direct_norm_tc(const dp_linear_desc* layers, const GhostPlan& plan, int B, int T,
                                 float* partials, int* dev_status, cudaStream_t st);
 

@@ -39,10 +39,7 @@ namespace dpg {
 
 namespace {
 
-#ifndef DPG_GTA_BK
-#define DPG_GTA_BK 64
-#endif
-constexpr int kBM = 128, kBN = 256, kBK = DPG_GTA_BK;
+constexpr int kBM = 128, kBN = 256, kBK = 64;
 constexpr int kBoxBytes = kBK * 128;                // kBK token rows x 128 bytes
 constexpr int kGBytes = (kBM / 64) * kBoxBytes;     // 16 KiB: this CTA's 128 rows of the G tile
 
@@ -52,27 +49,20 @@ constexpr int kGBytes = (kBM / 64) * kBoxBytes;     // 16 KiB: this CTA's 128 ro
 // stages: all the shared memory there is -- the ring is latency-bound, 7 stages measured 973
 // TFLOP/s where 6 gave 895; 32- and 128-row K steps were both slower), the pair's MMA reads
 // both halves -- a third less operand traffic per flop.
-#ifndef DPG_GTA_PAIR_STAGES
-#define DPG_GTA_PAIR_STAGES 7
-#endif
 template <bool kPair>
 struct Geo {
   static constexpr int kAColsPerCta = kPair ? kBN / 2 : kBN;
   static constexpr int kABytes = (kAColsPerCta / 64) * kBoxBytes;
   static constexpr int kStageBytes = kGBytes + kABytes;
-  static constexpr int kStages = kPair ? DPG_GTA_PAIR_STAGES : 4;
+  static constexpr int kStages = kPair ? 7 : 4;
   static constexpr int kTileM = kPair ? 2 * kBM : kBM;       // output rows per work item
-  static constexpr size_t kSmemBytes = size_t(kStages) * kStageBytes + 1024 + 512;
+  static constexpr size_t kSmemBytes = size_t(kStages) * kStageBytes + 1024 + 1024;
 };
-#ifndef DPG_GTA_SCALERS
-#define DPG_GTA_SCALERS 4
-#endif
-constexpr int kScalerWarps = DPG_GTA_SCALERS;
-constexpr int kEpiWarp0 = 2 + kScalerWarps;          // first epilogue warp
-#ifndef DPG_GTA_EPI_WARPS
-#define DPG_GTA_EPI_WARPS 16
-#endif
-constexpr int kEpiWarps = DPG_GTA_EPI_WARPS;         // kEpiWarps/4 per TMEM lane quarter (column groups)
+constexpr int kProducerAWarp = 2;                    // warp 0 loads G, warp 2 loads A, warp 1 issues MMAs
+constexpr int kScalerWarp0 = 3;
+constexpr int kScalerWarps = 4;
+constexpr int kEpiWarp0 = kScalerWarp0 + kScalerWarps;   // first epilogue warp
+constexpr int kEpiWarps = 16;         // kEpiWarps/4 per TMEM lane quarter (column groups)
 constexpr int kThreads = (kEpiWarp0 + kEpiWarps) * 32;
 constexpr int kTmemCols = 512;                      // 2 accumulators x 256 columns
 
@@ -155,23 +145,28 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                               ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + size_t(kStages) * kStageBytes);
-  uint64_t* full = bars;                      // TMA landed
-  uint64_t* ready = bars + kStages;           // G tile scaled (scale mode)
+  uint64_t* full = bars;                      // both producers' TMA loads landed
+  uint64_t* ready = bars + kStages;           // G tile scaled in both CTAs (scale mode; rank 0's copy)
   uint64_t* empty = bars + 2 * kStages;       // MMAs retired
   uint64_t* acc_full = bars + 3 * kStages;    // [2]
   uint64_t* acc_empty = acc_full + 2;         // [2]
   uint64_t* mma_done = acc_empty + 2;         // only used when the MMA issuer gives up
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mma_done + 1);
+  uint64_t* red_bar = mma_done + 1;           // [4] epilogue warps -> epilogue warp 0 (square-sum mode)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(red_bar + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  float* epi_red = reinterpret_cast<float*>(tmem_slot + 2);   // [2][kEpiWarps]
+  float* epi_red = reinterpret_cast<float*>(tmem_slot + 2);   // [4][kEpiWarps]
+  uint32_t* sink = reinterpret_cast<uint32_t*>(epi_red + 4 * kEpiWarps);   // [kStages] written by st.async, never read
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  const uint32_t tiles_a = ptx::smem_u32(tiles);
+  const uint32_t full_a = ptx::smem_u32(full), ready_a = ptx::smem_u32(ready), empty_a = ptx::smem_u32(empty);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
-      ptx::mbar_init(&full[s], 1);
-      ptx::mbar_init(&ready[s], kPeers);                    // one scaler warp per CTA and stage
+      ptx::mbar_init(&full[s], 2);             // the G producer and the A producer
+      // pair: rank 0's scaler warp arrives (and announces 4 bytes), rank 1's sends those 4 bytes
+      ptx::mbar_init(&ready[s], 1);
       ptx::mbar_init(&empty[s], 1);
     }
     for (int b = 0; b < 2; ++b) {
@@ -179,6 +174,7 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
       ptx::mbar_init(&acc_empty[b], kEpiWarps * kPeers);    // epilogue warps of both CTAs
     }
     ptx::mbar_init(mma_done, 1);
+    for (int b = 0; b < 4; ++b) ptx::mbar_init(&red_bar[b], kEpiWarps);
     *abort_flag = 0;
     ptx::fence_mbar_init();
   }
@@ -192,29 +188,36 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == 0) {
-    // ------------------------------------------------------------- TMA producer
+  if (warp == 0 || warp == kProducerAWarp) {
+    // ------------------------------------------------------------- TMA producers
+    // Two threads in two warps: one loads this CTA's G rows, the other its A columns.  The time
+    // a producer needs per stage is part of every stage's round trip, so the work is halved and
+    // the loop is kept to a few instructions (32-bit shared addresses, running example / token
+    // counters instead of a division).
     if (lane == 0) {
+      const bool is_a = (warp != 0);
+      constexpr int kBoxes = kBM / 64;
+      constexpr int kBoxesA = Geo<kPair>::kAColsPerCta / 64;
+      const uint32_t my_bytes = is_a ? uint32_t(Geo<kPair>::kABytes) : uint32_t(kGBytes);
+      const int nbox = is_a ? kBoxesA : kBoxes;
       uint32_t stage = 0, phase = 0, issued = 0;
       bool ok = true;
       for (int item = first_item; item < P.total_items && ok; item += item_stride) {
         const Item it = decode_item<kSqsum>(P, item);
-        const CUtensorMap* tg = &P.tmG[it.layer];
-        const CUtensorMap* ta = &P.tmA[it.layer];
+        const uint64_t tm = reinterpret_cast<uint64_t>(is_a ? &P.tmA[it.layer] : &P.tmG[it.layer]);
+        // first column of this CTA's part of the tile: its G rows, or its share of the A columns
+        const int c0 = is_a ? it.tn * kBN + int(rank) * Geo<kPair>::kAColsPerCta
+                            : it.tm * kTileM + int(rank) * kBM;
+        int ex = it.k0 / P.tsteps, ts = it.k0 - ex * P.tsteps;
         for (int ks = it.k0; ks < it.k1; ++ks) {
-          if (!ptx::mbar_wait(&empty[stage], phase ^ 1, abort_flag, P.wait_limit)) { ok = false; break; }
-          const int ex = ks / P.tsteps, t0 = (ks - ex * P.tsteps) * kBK;
-          uint8_t* dst = tiles + size_t(stage) * kStageBytes;
-          ptx::mbar_arrive_expect_tx(&full[stage], kStageBytes);
-          const int m0 = it.tm * kTileM + int(rank) * kBM;                   // this CTA's G rows
-          const int n0 = it.tn * kBN + int(rank) * Geo<kPair>::kAColsPerCta;   // and A columns
-#pragma unroll
-          for (int j = 0; j < kBM / 64; ++j)
-            ptx::tma_load_3d(dst + j * kBoxBytes, tg, &full[stage], m0 + j * 64, t0, ex);
-#pragma unroll
-          for (int j = 0; j < Geo<kPair>::kAColsPerCta / 64; ++j)
-            ptx::tma_load_3d(dst + kGBytes + j * kBoxBytes, ta, &full[stage], n0 + j * 64, t0, ex);
+          if (!ptx::mbar_wait_a(empty_a + 8 * stage, phase ^ 1, abort_flag, P.wait_limit)) { ok = false; break; }
+          const uint32_t bar = full_a + 8 * stage;
+          const uint32_t dst = tiles_a + stage * kStageBytes + (is_a ? kGBytes : 0);
+          ptx::mbar_arrive_expect_tx_a(bar, my_bytes);
+          for (int j = 0; j < nbox; ++j)
+            ptx::tma_load_3d_a(dst + j * kBoxBytes, tm, bar, c0 + j * 64, ts * kBK, ex);
           ++issued;
+          if (++ts == P.tsteps) { ts = 0; ++ex; }
           if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
       }
@@ -229,8 +232,11 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
     if (lane == 0 && rank == 0) {
       constexpr uint32_t idesc = ptx::idesc_bf16_f32(kTileM, kBN, 1, 1);
       // MN-major, 128-byte swizzle: 64-column chunks are one box (8 KiB) apart, groups of
-      // 8 token rows are 1 KiB apart
+      // 8 token rows are 1 KiB apart.  Only the 14-bit start address in the low word changes.
       constexpr uint64_t dbase = ptx::smem_desc_base(kBoxBytes, 1024, ptx::SWIZZLE_128B);
+      constexpr uint32_t desc_hi = uint32_t(dbase >> 32);
+      const uint32_t desc_lo0 = uint32_t(dbase) | ((tiles_a >> 4) & 0x3FFF);
+      const uint32_t go_a = kScale ? ready_a : full_a;
       uint32_t stage = 0, phase = 0, n_item = 0;
       bool ok = true;
       for (int item = first_item; item < P.total_items && ok; item += item_stride, ++n_item) {
@@ -240,25 +246,23 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
                     : ptx::mbar_wait(&acc_empty[buf], acc_phase ^ 1, abort_flag, P.wait_limit))) { ok = false; break; }
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * kBN;
+        uint32_t accum = 0;
         for (int ks = it.k0; ks < it.k1; ++ks) {
-          uint64_t* go = kScale ? &ready[stage] : &full[stage];
-          if (!(kPair ? ptx::mbar_wait_cluster(go, phase, abort_flag, P.wait_limit)
-                      : ptx::mbar_wait(go, phase, abort_flag, P.wait_limit))) { ok = false; break; }
+          if (!(kPair ? ptx::mbar_wait_cluster_a(go_a + 8 * stage, phase, abort_flag, P.wait_limit)
+                      : ptx::mbar_wait_a(go_a + 8 * stage, phase, abort_flag, P.wait_limit))) { ok = false; break; }
           ptx::tc_fence_after();
-          const uint32_t sg = ptx::smem_u32(tiles + size_t(stage) * kStageBytes);
-          const uint32_t sa = sg + kGBytes;
+          const uint32_t lo_g = desc_lo0 + stage * (kStageBytes >> 4);
+          const uint32_t lo_a = lo_g + (kGBytes >> 4);
 #pragma unroll
           for (int kk = 0; kk < kBK / 16; ++kk) {
             // 16 token rows further = two 1 KiB row groups
-            const uint64_t da = ptx::smem_desc(dbase, sg + kk * 2048);
-            const uint64_t db = ptx::smem_desc(dbase, sa + kk * 2048);
-            const uint32_t accum = (ks > it.k0 || kk > 0) ? 1u : 0u;
-            if (kPair) ptx::mma_bf16_ss_pair(d_tmem, da, db, idesc, accum);
-            else ptx::mma_bf16_ss(d_tmem, da, db, idesc, accum);
+            if (kPair) ptx::mma_bf16_ss_pair_lh(d_tmem, lo_g + kk * 128, lo_a + kk * 128, desc_hi, idesc, accum);
+            else ptx::mma_bf16_ss_lh(d_tmem, lo_g + kk * 128, lo_a + kk * 128, desc_hi, idesc, accum);
+            accum = 1;
           }
           // stage reusable in both CTAs once these MMAs retire
-          if (kPair) ptx::mma_commit_pair(&empty[stage], 3);
-          else ptx::mma_commit(&empty[stage]);
+          if (kPair) ptx::mma_commit_pair_a(empty_a + 8 * stage, 3);
+          else ptx::mma_commit_a(empty_a + 8 * stage);
           if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
         if (ok) {
@@ -278,23 +282,35 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
       // Each scaler warp owns every kScalerWarps-th K step, so kScalerWarps stages are scaled
       // concurrently: the per-stage latency (shared-memory round trip, proxy fence, barrier
       // hand-off) is overlapped instead of serialised.
-      const int sw = warp - 2;
+      //
+      // Hand-off to the MMA issuer (rank 0).  Rank 0's warp arrives on its own `ready` barrier
+      // and announces 4 more bytes; rank 1's warp delivers those 4 bytes with an asynchronous
+      // store into rank 0's shared memory whose completion on the barrier is a release at
+      // cluster scope: the scaled tile it wrote (made visible to the tensor core's proxy by the
+      // fence before) is ordered before the MMAs that rank 0 issues after its acquire.
+      const int sw = warp - kScalerWarp0;
+      const uint32_t ready_remote = kPair ? ptx::mapa_u32(ready_a, 0) : 0u;
+      const uint32_t sink_remote = kPair ? ptx::mapa_u32(ptx::smem_u32(sink), 0) : 0u;
       uint32_t cnt = 0;
       bool ok = true;
       for (int item = first_item; item < P.total_items && ok; item += item_stride) {
         const Item it = decode_item<kSqsum>(P, item);
-        for (int ks = it.k0; ks < it.k1; ++ks, ++cnt) {
-          if (int(cnt % kScalerWarps) != sw) continue;
-          const uint32_t stage = cnt % kStages, fill = cnt / kStages, phase = fill & 1u;
+        // first K step of this item that belongs to this warp
+        int ks = it.k0 + int((uint32_t(sw) + kScalerWarps - cnt % kScalerWarps) % kScalerWarps);
+        uint32_t c = cnt + uint32_t(ks - it.k0);
+        float r_next = ks < it.k1 ? __ldg(P.clip + ks / P.tsteps) : 1.f;
+        for (; ks < it.k1; ks += kScalerWarps, c += kScalerWarps) {
+          const float r = r_next;
+          // the factor of this warp's next K step is fetched before the waits, off the stage's path
+          if (ks + kScalerWarps < it.k1) r_next = __ldg(P.clip + (ks + kScalerWarps) / P.tsteps);
+          const uint32_t stage = c % kStages, fill = c / kStages, phase = fill & 1u;
           // A warp hops between stages, so it has not seen the previous fill of this one, and the
           // parity of `full` alone cannot tell "fill n landed" from "fill n-1 still in flight".
-          // Waiting first until the MMAs have retired fill n-1 (the same condition the producer
-          // waits for before it issues fill n, so no time is lost) leaves only "fill n pending"
+          // Waiting first until the MMAs have retired fill n-1 (the same condition the producers
+          // wait for before they issue fill n, so no time is lost) leaves only "fill n pending"
           // or "fill n landed".
-          if (fill > 0 && !ptx::mbar_wait(&empty[stage], phase ^ 1, abort_flag, P.wait_limit)) { ok = false; break; }
-          if (!ptx::mbar_wait(&full[stage], phase, abort_flag, P.wait_limit)) { ok = false; break; }
-          const int ex = ks / P.tsteps;
-          const float r = __ldg(P.clip + ex);
+          if (fill > 0 && !ptx::mbar_wait_a(empty_a + 8 * stage, phase ^ 1, abort_flag, P.wait_limit)) { ok = false; break; }
+          if (!ptx::mbar_wait_a(full_a + 8 * stage, phase, abort_flag, P.wait_limit)) { ok = false; break; }
           if (r != 1.0f) {
             // r = r_hi + r_lo with both parts in bf16 (16 mantissa bits in total); g*r is formed
             // as fma(g, r_hi, g*r_lo) on packed bf16 pairs: one rounding of the exact g*r_hi plus
@@ -302,29 +318,32 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
             const __nv_bfloat16 rh = __float2bfloat16_rn(r);
             const __nv_bfloat16 rl = __float2bfloat16_rn(r - __bfloat162float(rh));
             const __nv_bfloat162 rh2 = __halves2bfloat162(rh, rh), rl2 = __halves2bfloat162(rl, rl);
-            uint4* g = reinterpret_cast<uint4*>(tiles + size_t(stage) * kStageBytes);
-            constexpr int kChunks = kGBytes / 16 / 32;          // 16-byte chunks per lane
+            // kChunks 16-byte chunks per lane, eight at a time
+            constexpr int kChunks = kGBytes / 16 / 32;
+            uint4* g = reinterpret_cast<uint4*>(tiles + size_t(stage) * kStageBytes) + lane;
 #pragma unroll 1
             for (int c0 = 0; c0 < kChunks; c0 += 8) {
               uint4 v[8];
 #pragma unroll
-              for (int c = 0; c < 8; ++c) v[c] = g[(c0 + c) * 32 + lane];
+              for (int q = 0; q < 8; ++q) v[q] = g[(c0 + q) * 32];
 #pragma unroll
-              for (int c = 0; c < 8; ++c) {
-                __nv_bfloat162* w = reinterpret_cast<__nv_bfloat162*>(&v[c]);
+              for (int q = 0; q < 8; ++q) {
+                __nv_bfloat162* w = reinterpret_cast<__nv_bfloat162*>(&v[q]);
 #pragma unroll
                 for (int e = 0; e < 4; ++e) w[e] = __hfma2(w[e], rh2, __hmul2(w[e], rl2));
-                g[(c0 + c) * 32 + lane] = v[c];
+                g[(c0 + q) * 32] = v[q];
               }
             }
             ptx::fence_proxy_async_smem();
           }
           __syncwarp();
           if (lane == 0) {
-            if (kPair) ptx::mbar_arrive_cluster(&ready[stage], 0);   // the MMA issuer lives in rank 0
-            else ptx::mbar_arrive(&ready[stage]);
+            if (!kPair) ptx::mbar_arrive(&ready[stage]);
+            else if (rank == 0) ptx::mbar_arrive_expect_tx_a(ready_a + 8 * stage, 4);
+            else ptx::st_async_signal_a(ready_remote + 8 * stage, sink_remote + 4 * stage);
           }
         }
+        cnt += uint32_t(it.k1 - it.k0);
       }
       if (!ok && lane == 0) {
         *abort_flag = 1;
@@ -364,14 +383,20 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
           if (kPair) ptx::mbar_arrive_cluster(&acc_empty[buf], 0);
           else ptx::mbar_arrive(&acc_empty[buf]);
         }
+        // the warps' sums meet through an mbarrier with a bounded wait (no blocking named
+        // barrier: a warp that gave up never arrives); four slots, since the other warps can run
+        // at most two items ahead of a waiting warp 0 (they need its acc_empty arrivals)
         acc = warp_sum(acc);
-        if (lane == 0) epi_red[buf * kEpiWarps + ew] = acc;
-        asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
-        if (ew == 0 && lane == 0) {
-          float s = 0.f;
+        const uint32_t slot = n_item & 3, red_phase = (n_item >> 2) & 1;
+        if (lane == 0) { epi_red[slot * kEpiWarps + ew] = acc; ptx::mbar_arrive(&red_bar[slot]); }
+        if (ew == 0) {
+          if (!ptx::mbar_wait_relaxed(&red_bar[slot], red_phase, abort_flag, P.wait_limit)) { ok = false; break; }
+          if (lane == 0) {
+            float s = 0.f;
 #pragma unroll
-          for (int e = 0; e < kEpiWarps; ++e) s += epi_red[buf * kEpiWarps + e];
-          P.sq_partials[size_t(it.example) * P.n_per + L.col_begin + it.tm * L.tiles_n + it.tn] = s;
+            for (int e = 0; e < kEpiWarps; ++e) s += epi_red[slot * kEpiWarps + e];
+            P.sq_partials[size_t(it.example) * P.n_per + L.col_begin + it.tm * L.tiles_n + it.tn] = s;
+          }
         }
       } else {
         // destination: the layer's output (no K split) or this split's partial plane
@@ -498,21 +523,14 @@ __global__ void splitk_reduce_kernel(const float* __restrict__ partial, int nspl
 // let the issuer run ahead of the partner's loads and re-arm a stage barrier in mid-phase.)
 constexpr bool kClipScale = true;
 
-#ifdef DPG_GTA_SINGLE_CTA
-constexpr bool kUsePair = false;     // experiment only: clipped sums on the single-CTA tiles
-#else
 constexpr bool kUsePair = true;
-#endif
 
 template <bool kScale, bool kSqsum, bool kPair>
 dp_status set_attr_once() {
-  static bool done = false;
-  if (!done) {
+  if (first_use_on_this_device(reinterpret_cast<const void*>(&gemm_gta_kernel<kScale, kSqsum, kPair>)))
     DP_CUDA_OK(cudaFuncSetAttribute(gemm_gta_kernel<kScale, kSqsum, kPair>,
                                     cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)Geo<kPair>::kSmemBytes));
-    done = true;
-  }
   return DP_OK;
 }
 
@@ -524,18 +542,13 @@ dp_status launch_gta(const GtaParams& P, int units, cudaStream_t st) {
   cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = Geo<kPair>::kSmemBytes;
   cfg.stream = st;
-  cudaLaunchAttribute attr[2];
+  cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = kPair ? 2 : 1;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-#ifdef DPG_GTA_POLICY_LB
-  attr[1].id = cudaLaunchAttributeClusterSchedulingPolicyPreference;
-  attr[1].val.clusterSchedulingPolicyPreference = cudaClusterSchedulingPolicyLoadBalancing;
-  cfg.numAttrs = 2;
-#endif
   DP_CUDA_OK(cudaLaunchKernelEx(&cfg, gemm_gta_kernel<kScale, kSqsum, kPair>, P));
   ++g_kernel_launches;
   return DP_OK;
@@ -640,22 +653,6 @@ dp_status launch_clip_accumulate_tc(const dp_linear_desc* layers, int n_layers, 
   return DP_OK;
 }
 
-// Diagnostic: how many CTA pairs of the clipped-sum kernel the device can hold at once.
-int gta_max_active_pairs() {
-  if (set_attr_once<kClipScale, false, true>() != DP_OK) return -1;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(2 * 74, 1, 1);
-  cfg.blockDim = dim3(kThreads, 1, 1);
-  cfg.dynamicSmemBytes = Geo<true>::kSmemBytes;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr; cfg.numAttrs = 1;
-  int n = -1;
-  if (cudaOccupancyMaxActiveClusters(&n, gemm_gta_kernel<kClipScale, false, true>, &cfg) != cudaSuccess)
-    return -2;
-  return n;
-}
 
 dp_status launch_direct_norm_tc(const dp_linear_desc* layers, const GhostPlan& plan, int B, int T,
                                 float* partials, int* dev_status, cudaStream_t st) {

@@ -39,7 +39,7 @@ constexpr int kKStep = 64;                        // bf16 columns per stage row 
 constexpr int kTileBytes = kRows * kKStep * 2;    // 16 KiB
 constexpr int kStageBytes = 2 * kTileBytes;       // rows of block I, rows of block J
 constexpr int kStages = 7;
-constexpr size_t kSmemBytes = size_t(kStages) * kStageBytes + 1024 /*alignment slack*/ + 512;
+constexpr size_t kSmemBytes = size_t(kStages) * kStageBytes + 1024 /*alignment slack*/ + 1024;
 constexpr int kEpiWarp0 = 4, kEpiWarps = 16;
 constexpr int kThreads = (kEpiWarp0 + kEpiWarps) * 32;
 constexpr int kTmemCols = 512;
@@ -106,9 +106,11 @@ ghost_norm_pair_kernel(const __grid_constant__ PairParams P) {
   uint64_t* sa_empty = sa_full + 2;            // S_A copied to registers in both CTAs (rank 0's copy)
   uint64_t* sg_empty = sa_full + 3;            // S_G consumed in both CTAs (rank 0's copy)
   uint64_t* mma_done = sa_full + 4;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mma_done + 1);
+  uint64_t* red_bar = mma_done + 1;            // [4] this CTA's epilogue warps -> its epilogue warp 0
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(red_bar + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  float* epi_red = reinterpret_cast<float*>(tmem_slot + 2);   // [2][kEpiWarps]
+  float* epi_red = reinterpret_cast<float*>(tmem_slot + 2);   // [4][kEpiWarps]
+  uint32_t* sink = reinterpret_cast<uint32_t*>(epi_red + 4 * kEpiWarps);   // [kStages] written by st.async, never read
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -116,7 +118,7 @@ ghost_norm_pair_kernel(const __grid_constant__ PairParams P) {
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       ptx::mbar_init(&full[s], 1);
-      ptx::mbar_init(&ready[s], 2);
+      ptx::mbar_init(&ready[s], 1);             // rank 0's relay arrives and announces 4 bytes, rank 1's sends them
       ptx::mbar_init(&empty[s], 1);
     }
     ptx::mbar_init(sa_full, 1);
@@ -124,6 +126,7 @@ ghost_norm_pair_kernel(const __grid_constant__ PairParams P) {
     ptx::mbar_init(sa_empty, kEpiWarps * 2);
     ptx::mbar_init(sg_empty, kEpiWarps * 2);
     ptx::mbar_init(mma_done, 1);
+    for (int b = 0; b < 4; ++b) ptx::mbar_init(&red_bar[b], kEpiWarps);
     *abort_flag = 0;
     ptx::fence_mbar_init();
   }
@@ -207,7 +210,14 @@ ghost_norm_pair_kernel(const __grid_constant__ PairParams P) {
     }
   } else if (warp == 2) {
     // -------------------------------------------------------------------- relay
+    // Tells rank 0's MMA issuer that this CTA's half of a stage has landed.  Rank 0's relay
+    // arrives on its own `ready` barrier and announces 4 more bytes; rank 1's relay, which has
+    // acquired its `full` barrier (so the TMA data are visible to it), delivers those 4 bytes with
+    // an asynchronous store into rank 0's shared memory whose completion on the barrier is a
+    // release at cluster scope.
     if (lane == 0) {
+      const uint32_t ready_a = ptx::smem_u32(ready), sink_a = ptx::smem_u32(sink);
+      const uint32_t ready_remote = ptx::mapa_u32(ready_a, 0), sink_remote = ptx::mapa_u32(sink_a, 0);
       uint32_t stage = 0, phase = 0;
       bool ok = true;
       for (int item = first_item; item < P.total_items && ok; item += item_stride) {
@@ -215,7 +225,8 @@ ghost_norm_pair_kernel(const __grid_constant__ PairParams P) {
         const int nsteps = (it.a1 - it.a0) + (it.g1 - it.g0);
         for (int k = 0; k < nsteps; ++k) {
           if (!ptx::mbar_wait(&full[stage], phase, abort_flag, P.wait_limit)) { ok = false; break; }
-          ptx::mbar_arrive_cluster(&ready[stage], 0);
+          if (rank == 0) ptx::mbar_arrive_expect_tx_a(ready_a + 8 * stage, 4);
+          else ptx::st_async_signal_a(ready_remote + 8 * stage, sink_remote + 4 * stage);
           if (++stage == kStages) { stage = 0; phase ^= 1; }
         }
       }
@@ -264,14 +275,20 @@ ghost_norm_pair_kernel(const __grid_constant__ PairParams P) {
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive_cluster(sg_empty, 0);
+      // the warps' sums meet through an mbarrier with a bounded wait (no blocking named barrier:
+      // a warp that gave up never arrives); four slots, since the other warps can run at most one
+      // item ahead of a waiting warp 0 (they need its sa_empty arrival)
       acc = warp_sum(acc);
-      if (lane == 0) epi_red[ph * kEpiWarps + ew] = acc;
-      asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
-      if (ew == 0 && lane == 0) {
-        float s = 0.f;
+      const uint32_t slot = n_item & 3, red_phase = (n_item >> 2) & 1;
+      if (lane == 0) { epi_red[slot * kEpiWarps + ew] = acc; ptx::mbar_arrive(&red_bar[slot]); }
+      if (ew == 0) {
+        if (!ptx::mbar_wait_relaxed(&red_bar[slot], red_phase, abort_flag, P.wait_limit)) { ok = false; break; }
+        if (lane == 0) {
+          float s = 0.f;
 #pragma unroll
-        for (int e = 0; e < kEpiWarps; ++e) s += epi_red[ph * kEpiWarps + e];
-        P.partials[it.pidx + int(rank)] = (it.ti == it.tj) ? s : 2.f * s;
+          for (int e = 0; e < kEpiWarps; ++e) s += epi_red[slot * kEpiWarps + e];
+          P.partials[it.pidx + int(rank)] = (it.ti == it.tj) ? s : 2.f * s;
+        }
       }
     }
     if (!ok && lane == 0) {
@@ -293,12 +310,9 @@ ghost_norm_pair_kernel(const __grid_constant__ PairParams P) {
 
 dp_status launch_ghost_norm_pair(const dp_linear_desc* layers, const GhostPlan& plan, int B, int T,
                                  float* partials, int* dev_status, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
+  if (first_use_on_this_device(reinterpret_cast<const void*>(&ghost_norm_pair_kernel)))
     DP_CUDA_OK(cudaFuncSetAttribute(ghost_norm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)kSmemBytes));
-    attr_set = true;
-  }
   const int nt = ceil_div(T, kTile2);
   for (size_t g0 = 0; g0 < plan.ghost_layers.size(); g0 += kGhostMaxLayers) {
     const size_t g1 = std::min(plan.ghost_layers.size(), g0 + kGhostMaxLayers);

@@ -100,9 +100,10 @@ ghost_norm_tc_kernel(const __grid_constant__ GhostParams P) {
   uint64_t* acc_full = bars + 2 * kStages; // [2]        MMA -> epilogue
   uint64_t* acc_empty = acc_full + 2;      // [2]        epilogue -> MMA
   uint64_t* mma_done = acc_empty + 2;      // only used when the MMA issuer gives up
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mma_done + 1);
+  uint64_t* red_bar = mma_done + 1;        // [4]        epilogue warps -> epilogue warp 0
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(red_bar + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  float* epi_red = reinterpret_cast<float*>(tmem_slot + 2);   // [2][4]
+  float* epi_red = reinterpret_cast<float*>(tmem_slot + 2);   // [4][4]
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -111,6 +112,7 @@ ghost_norm_tc_kernel(const __grid_constant__ GhostParams P) {
     for (int s = 0; s < kStages; ++s) { ptx::mbar_init(&full[s], 1); ptx::mbar_init(&empty[s], 1); }
     for (int b = 0; b < 2; ++b) { ptx::mbar_init(&acc_full[b], 1); ptx::mbar_init(&acc_empty[b], 4); }
     ptx::mbar_init(mma_done, 1);
+    for (int b = 0; b < 4; ++b) ptx::mbar_init(&red_bar[b], 4);
     *abort_flag = 0;
     ptx::fence_mbar_init();
   }
@@ -220,13 +222,20 @@ ghost_norm_tc_kernel(const __grid_constant__ GhostParams P) {
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&acc_empty[buf]);   // accumulators may be overwritten
+      // The four warps' sums meet through an mbarrier, not a blocking named barrier: a warp that
+      // gave up above never arrives, and warp 0's wait for the others is bounded like every other.
+      // Four slots: the other warps can run at most two items ahead of a waiting warp 0 (they
+      // need its acc_empty arrivals), so a slot is never rewritten before it has been read.
       acc = warp_sum(acc);
-      if (lane == 0) epi_red[buf * 4 + ew] = acc;
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (ew == 0 && lane == 0) {
-        const float s = (epi_red[buf * 4 + 0] + epi_red[buf * 4 + 1]) +
-                        (epi_red[buf * 4 + 2] + epi_red[buf * 4 + 3]);
-        P.partials[it.pidx] = (it.ti == it.tj) ? s : 2.f * s;
+      const uint32_t slot = n_item & 3, red_phase = (n_item >> 2) & 1;
+      if (lane == 0) { epi_red[slot * 4 + ew] = acc; ptx::mbar_arrive(&red_bar[slot]); }
+      if (ew == 0) {
+        if (!ptx::mbar_wait_relaxed(&red_bar[slot], red_phase, abort_flag, P.wait_limit)) { ok = false; break; }
+        if (lane == 0) {
+          const float s = (epi_red[slot * 4 + 0] + epi_red[slot * 4 + 1]) +
+                          (epi_red[slot * 4 + 2] + epi_red[slot * 4 + 3]);
+          P.partials[it.pidx] = (it.ti == it.tj) ? s : 2.f * s;
+        }
       }
     }
     if (!ok && lane == 0) {
@@ -273,15 +282,13 @@ dp_status launch_reduce_partials(const float* partials, int n_per, int B, float*
 // plan.partials layout inside `partials` (the caller reduces them afterwards).
 dp_status launch_ghost_norm_tc(const dp_linear_desc* layers, const GhostPlan& plan, int B, int T,
                                float* partials, int* dev_status, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
+  if (first_use_on_this_device(reinterpret_cast<const void*>(&launch_ghost_norm_tc))) {
     DP_CUDA_OK(cudaFuncSetAttribute(ghost_norm_tc_kernel<true>,
                                     cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)GhostGeo<true>::kSmemBytes));
     DP_CUDA_OK(cudaFuncSetAttribute(ghost_norm_tc_kernel<false>,
                                     cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)GhostGeo<false>::kSmemBytes));
-    attr_set = true;
   }
   const int nt = ceil_div(T, kTile);
   // layers are processed in groups that fit one parameter block

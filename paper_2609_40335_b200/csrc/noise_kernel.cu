@@ -20,12 +20,15 @@ add_noise_kernel(float* __restrict__ out, long long n, int cols, long long ld, f
   key.step = effective_step(key.step, step_dev);
   const long long nq = (n + 3) >> 2;
   const bool flat = (ld == cols);
+  // 16-byte accesses only on a 16-byte aligned base (the fused entry points accept any fp32
+  // tensor; an unaligned one takes the scalar branch)
+  const bool vec = flat && ((reinterpret_cast<uintptr_t>(out) & 15u) == 0);
   for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < nq;
        q += (long long)gridDim.x * blockDim.x) {
     float z[4];
     normals4((unsigned long long)(q0 + q), key, z);       // q0: first counter of a slice
     const long long j = q << 2;
-    if (flat && j + 3 < n) {
+    if (vec && j + 3 < n) {
       float4 v = kFill ? make_float4(0.f, 0.f, 0.f, 0.f) : *reinterpret_cast<float4*>(out + j);
       v.x = noised(v.x, z[0], amp, scale);
       v.y = noised(v.y, z[1], amp, scale);
@@ -91,13 +94,11 @@ dp_status launch_add_noise(float* out, long long rows, int cols, long long ld, b
   // per SM leave half of every SM's thread slots free for it.
   const int grid = (int)std::min<long long>(want, (long long)sm_count() * (fill ? 4 : 16));
   const NoiseKey key{uint32_t(seed), uint32_t(seed >> 32), tensor_id, step};
-  static bool carveout_set = false;
-  if (fill && !carveout_set) {
+  if (fill && first_use_on_this_device(reinterpret_cast<const void*>(&launch_add_noise))) {
     // same shared-memory carve-out as the TMA kernels, so that both can be resident on one SM
     DP_CUDA_OK(cudaFuncSetAttribute(add_noise_kernel<true>,
                                     cudaFuncAttributePreferredSharedMemoryCarveout,
                                     cudaSharedmemCarveoutMaxShared));
-    carveout_set = true;
   }
   if (fill)
     add_noise_kernel<true><<<grid, 256, 0, st>>>(out, n, cols, ld, amp, scale, key, g_step_dev, first_quad);

@@ -91,6 +91,47 @@ __device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity
   return true;
 }
 
+// ---- the same primitives on 32-bit shared-memory addresses --------------------------------
+// The single-thread roles (TMA producer, MMA issuer) sit on the latency chain of every pipeline
+// stage, so their per-stage instruction count matters: they keep shared addresses as 32-bit
+// values computed once, instead of converting generic pointers at every use.
+__device__ __forceinline__ bool mbar_try_wait_a(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred P;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, P;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_a(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                            long long limit = kDefaultWaitLimit) {
+  if (mbar_try_wait_a(bar, parity)) return true;
+  if (limit <= 0) return false;
+  const long long t0 = clock64();
+  uint32_t spins = 0;
+  while (!mbar_try_wait_a(bar, parity)) {
+    if ((++spins & 1023u) == 0) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > limit) return false;
+    }
+  }
+  return true;
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx_a(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_a(uint32_t smem_dst, uint64_t tmap, uint32_t bar,
+                                              int32_t c0, int32_t c1, int32_t c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(smem_dst), "l"(tmap), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+
 // After a producer gave up: wait (bounded, ~0.1 s per stage) until the copies it had already
 // issued have landed, so that the CTA does not exit with TMA writes to its shared memory in
 // flight.  `issued` counts all stages armed so far on the ring of `n_stages` full-barriers.
@@ -218,26 +259,59 @@ __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-// arrive on the barrier at the same shared-memory offset in CTA `cta` of this cluster
+// Arrive on the barrier at the same shared-memory offset in CTA `cta` of this cluster.  The
+// arrive is a release at CLUSTER scope: what this thread (and, through a preceding __syncwarp or
+// fence, its warp) did before it is ordered before whatever the waiting CTA does after its
+// acquire.  Used where the arrive is off the critical path (an epilogue warp freeing an
+// accumulator once per tile): its fence is slow.
 __device__ __forceinline__ void mbar_arrive_cluster(uint64_t* bar, uint32_t cta) {
   uint32_t remote;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(bar)), "r"(cta));
-  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
+// A cheaper cluster-scope release for a hand-off that is on the critical path of every pipeline
+// stage (measured on B200: the fence inside mbarrier.arrive.release.cluster costs about a
+// thousand cycles per arrive): signal the barrier of CTA `cta` through an asynchronous 4-byte
+// store into that CTA's shared memory (a word nobody reads).  The store's complete-tx on the
+// barrier is a release at cluster scope and the issuing thread does not wait for it.  The barrier
+// must expect those 4 bytes (the local arriver announces them with arrive.expect_tx).
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t cta) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(addr), "r"(cta));
+  return remote;
+}
+// st_async_signal on cluster addresses that were mapped once (mapa_u32)
+__device__ __forceinline__ void st_async_signal_a(uint32_t remote_bar, uint32_t remote_sink) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
+               ::"r"(remote_sink), "r"(1u), "r"(remote_bar) : "memory");
+}
+// Poll without ordering (cheap inside a spin loop) ...
+__device__ __forceinline__ bool mbar_try_wait_relaxed_cluster(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred P;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.relaxed.cluster.shared::cta.b64 P, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, P;\n\t}"
       : "=r"(ok)
       : "r"(smem_u32(bar)), "r"(parity)
       : "memory");
   return ok != 0;
 }
-// bounded wait on a barrier that the other CTA of the pair also arrives on.  Default
-// (.acquire/.release at CTA scope) forms are used on both sides: measured on B200, the
-// explicit .cluster-scope forms halved the kernel's throughput.
+// ... and the acquire at cluster scope that pairs with mbar_arrive_cluster
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred P;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 P, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, P;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait on a barrier that the other CTA of the pair also arrives on: spin on the relaxed
+// poll, then take ONE cluster-scope acquire of the completed phase (it succeeds at once), so the
+// ordering is paid once per hand-off and not once per poll.
 __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity,
                                                   volatile int* abort_flag,
                                                   long long limit = kDefaultWaitLimit) {
@@ -245,13 +319,44 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity
   if (limit <= 0) return false;
   const long long t0 = clock64();
   uint32_t spins = 0;
-  while (!mbar_try_wait_cluster(bar, parity)) {
+  while (!mbar_try_wait_relaxed_cluster(bar, parity)) {
     if ((++spins & 1023u) == 0) {
       if (*abort_flag) return false;
       if (clock64() - t0 > limit) return false;
     }
   }
-  return true;
+  return mbar_try_wait_cluster(bar, parity);
+}
+__device__ __forceinline__ bool mbar_wait_cluster_a(uint32_t bar, uint32_t parity,
+                                                    volatile int* abort_flag,
+                                                    long long limit = kDefaultWaitLimit) {
+  uint32_t ok;
+  auto poll = [&](bool acquire) {
+    if (acquire)
+      asm volatile(
+          "{\n\t.reg .pred P;\n\t"
+          "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 P, [%1], %2;\n\t"
+          "selp.u32 %0, 1, 0, P;\n\t}"
+          : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    else
+      asm volatile(
+          "{\n\t.reg .pred P;\n\t"
+          "mbarrier.try_wait.parity.relaxed.cluster.shared::cta.b64 P, [%1], %2;\n\t"
+          "selp.u32 %0, 1, 0, P;\n\t}"
+          : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+  };
+  if (poll(true)) return true;
+  if (limit <= 0) return false;
+  const long long t0 = clock64();
+  uint32_t spins = 0;
+  while (!poll(false)) {
+    if ((++spins & 1023u) == 0) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > limit) return false;
+    }
+  }
+  return poll(true);
 }
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t* smem_result, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
@@ -275,6 +380,42 @@ __device__ __forceinline__ void mma_bf16_ss_pair(uint32_t d_tmem, uint64_t a_des
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// The same MMAs with each 64-bit shared-memory descriptor given as (low word, high word): only
+// the low word (the 14-bit start address) changes from stage to stage.
+__device__ __forceinline__ void mma_bf16_ss_pair_lh(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo,
+                                                    uint32_t desc_hi, uint32_t idesc,
+                                                    uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %3};\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void mma_bf16_ss_lh(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo,
+                                               uint32_t desc_hi, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %3};\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void mma_commit_a(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void mma_commit_pair_a(uint32_t bar, uint16_t cta_mask) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 "
+      "[%0], %1;" ::"r"(bar), "h"(cta_mask)
+      : "memory");
+}
+
 // arrive (once the pair's MMAs so far have completed) on the barrier at this offset in every
 // CTA named by cta_mask
 __device__ __forceinline__ void mma_commit_pair(uint64_t* bar, uint16_t cta_mask) {
