@@ -1,13 +1,16 @@
 #!/usr/bin/env python
 """Benchmark of the DP-SGD ghost-clipping hot path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload cfg2]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload cfg3]
+    python bench.py --case gemm --reps 3          # one entry point on a small case (for profilers)
 
 A step is one pass of the whole path over one synthetic batch: per-example norms of every
 block linear layer, the LM head and the embedding (plus the tied cross term / position table
 where the workload has them), clip factors, the clipped sum of every parameter tensor and its
-Gaussian noise.  Prints ONE JSON line (rank 0).  `--impl reference` times the float64 CPU
-oracle instead (a reported baseline, not a target).
+Gaussian noise.  Prints ONE JSON line (rank 0).  The default workload is the GPT-2-small shape
+(cfg3); at one GPU the line also carries a `sweep` over the other configurations, the
+ghost-vs-direct timing per layer shape (`norm_modes`) and the tied path's extra cost.
+`--impl reference` times the float64 CPU oracle instead (a reported baseline, not a target).
 """
 from __future__ import annotations
 
@@ -19,17 +22,21 @@ import subprocess
 import sys
 import threading
 import time
+import types
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one grouped GEMM launch, from the ncu capture
-# summarised in profiles/gemm_gta_kernel_pair.md (scaled to the full launch as described there)
-GEMM_TRAFFIC_BYTES = {"cfg2": int(0.96 * (1.022e9 + 0.324e9))}
-
 METRIC = "dp_sgd_examples_per_sec"
 UNIT = "examples/s"
+
+# DRAM bytes of the clipped-sum GEMM (dram__bytes_read.sum + dram__bytes_write.sum, one ncu capture
+# of a three-wave launch of the same kernel) divided by that launch's algorithmic bytes (inputs
+# read once + fp32 outputs written once).  `roofline.traffic` of a workload is this ratio times
+# the algorithmic bytes of its own grouped launch: the kernel reads every operand tile from DRAM
+# once whatever the layer list, so traffic grows in proportion to the bytes.
+GEMM_DRAM_OVER_ALGORITHMIC = 0.97
 
 
 def measured_peaks():
@@ -46,7 +53,7 @@ def measured_peaks():
 
 # ------------------------------------------------------------------------------- clocks
 class ClockSampler:
-    """Samples SM clock, power and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clock, power and throttle reasons with nvidia-smi while timed regions run."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
@@ -71,14 +78,13 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.lines.append((time.time(), line.strip()))
 
-    def stop(self, t0: float, t1: float):
+    def window(self, t0: float, t1: float):
+        """Summary of the samples taken between two wall-clock times."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
-        self.proc.terminate()
         sm, mx, reasons, power = [], [], set(), []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ts, line in self.lines:
+        for ts, line in list(self.lines):
             if ts < t0 - 0.05 or ts > t1 + 0.15:
                 continue
             f = [x.strip() for x in line.split(",")]
@@ -94,6 +100,28 @@ class ClockSampler:
                 "power_w_max": max(power) if power else None,
                 "samples": len(sm), "reasons": sorted(reasons)}
 
+    def stop(self):
+        if self.proc is not None:
+            time.sleep(0.15)
+            self.proc.terminate()
+
+
+def choose_tensor_peak(peaks, region_s, clocks):
+    """Which measured bf16 peak a tensor-bound kernel of this run is compared with: the sustained
+    (power-capped) figure only when the timed region itself was sustained -- at least a second
+    long AND the sampler saw the power cap -- otherwise the burst figure."""
+    capped = bool(clocks) and "sw_power_cap" in (clocks.get("reasons") or [])
+    if region_s >= 1.0 and capped:
+        return peaks["bf16_tflops_sustained"], "sustained", (
+            "timed region %.2f s with sw_power_cap active (median SM clock %s MHz): sustained peak"
+            % (region_s, clocks.get("sm_mhz")))
+    why = []
+    if region_s < 1.0:
+        why.append("timed region only %.3f s" % region_s)
+    if not capped:
+        why.append("power cap not reached (median SM clock %s MHz)" % (clocks or {}).get("sm_mhz"))
+    return peaks["bf16_tflops"], "burst", "; ".join(why) + ": burst peak"
+
 
 # --------------------------------------------------------------------- algorithmic work
 def work_counts(w):
@@ -105,13 +133,22 @@ def work_counts(w):
     gram_flops = sum(B * T * (T + 1) * (d + p) for d, p in lin)
     acc_flops = sum(2 * B * T * d * p for d, p in lin)
     acc_bytes = sum(es * B * T * (d + p) + 4 * d * p for d, p in lin)
-    n_params = sum(d * p for d, p in lin if True) + w.V * w.d_model * (0 if (w.tied and w.lm) else 1)
+    n_params = sum(d * p for d, p in lin) + w.V * w.d_model * (0 if (w.tied and w.lm) else 1)
     if w.positions:
         n_params += 1024 * w.d_model
     embed_bytes = es * B * T * w.d_model + 4 * B * T
     return dict(norm_bytes=norm_bytes, gram_flops=gram_flops, acc_flops=acc_flops,
                 acc_bytes=acc_bytes, noise_bytes=8 * n_params, n_params=n_params,
                 embed_bytes=embed_bytes)
+
+
+def shape_of(ds, name):
+    """The fields work_counts needs, from a device step."""
+    return types.SimpleNamespace(
+        name=name, dtype="bf16" if ds.G_emb.dtype.itemsize == 2 else "f32", B=ds.B, T=ds.T, V=ds.V,
+        d_model=ds.d_model, tied=ds.tied, positions=ds.positions,
+        linears=[types.SimpleNamespace(d=l.d, p=l.p) for l in ds.linears],
+        lm=types.SimpleNamespace(d=ds.lm.d, p=ds.lm.p) if ds.lm else None)
 
 
 def make_workload(name, seed=0, B=None, T=None, full_model=False):
@@ -193,7 +230,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": per * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic", "config": {"workload": w.name, "B": w.B, "T": w.T},
+            "data": "synthetic", "config": {"workload": w.name, "B_per_gpu": w.B, "T": w.T},
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
                              "sample": sample},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -201,13 +238,204 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# ----------------------------------------------------------------- device-side measurements
+def _ev():
+    import torch
+    return torch.cuda.Event(enable_timing=True)
+
+
+def time_graph(fn, reps, rounds=3):
+    """Best-of-`rounds` device time of one call of fn, from a CUDA graph holding `reps` calls
+    (the host's per-call work -- tensor-map encodes, argument checks -- stays out of the figure)."""
+    import torch
+    fn()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for _ in range(reps):
+            fn()
+    g.replay()
+    torch.cuda.synchronize()
+    best = float("inf")
+    a, b = _ev(), _ev()
+    for _ in range(rounds):
+        a.record()
+        g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        best = min(best, a.elapsed_time(b) / reps)
+    return best
+
+
+def graph_phase_times(P, ds, seed, first_step, replays, batches=5):
+    """Per-phase and GEMM durations inside back-to-back replays of the captured step: a second
+    capture of the same step with external event nodes is replayed in `batches` runs of
+    replays/batches replays each (no synchronize inside a run, so the clock and power state are
+    those of the timed region) and the events of each run's LAST replay are read."""
+    import torch
+    sgt = P.StepGraph(ds, seed=seed, first_step=first_step, timing=True)
+    per = max(1, replays // batches)
+    det = []
+    for _ in range(batches):
+        for _ in range(per):
+            sgt.replay()
+        torch.cuda.synchronize()
+        det.append(sgt.phase_ms())
+    med = lambda k: statistics.median(d[k] for d in det)
+    return {"norms": med("norms"), "clip_accumulate": med("clip_accumulate"), "gemm": med("gemm"),
+            "step_with_event_nodes": med("step"), "samples": len(det), "replays_per_sample": per}
+
+
+def ghost_norm_alone(dp, ds, peaks, peak_tf, counts):
+    """The linear-layer norm call alone (five calls in one graph, each with its reduce)."""
+    import torch
+    lin_layers = ds.linears + ([ds.lm] if ds.lm else [])
+    ms = time_graph(lambda: dp.dp_ghost_norms(lin_layers, ds.B, ds.T, ds.sq, ws=ds.ws,
+                                              dev_status=ds.dev_status), reps=5)
+    t_hbm = counts["norm_bytes"] / (peaks["hbm_gbs"] * 1e9)
+    t_tc = counts["gram_flops"] / (peak_tf * 1e12)
+    return {"kernel": "ghost_norm_pair_kernel" if ds.T > 128 else "ghost_norm_tc_kernel",
+            "bound": "hbm" if t_hbm >= t_tc else "tensor", "ms": ms,
+            "achieved_GBs": counts["norm_bytes"] / (ms * 1e-3) / 1e9,
+            "achieved_TFLOPs": counts["gram_flops"] / (ms * 1e-3) / 1e12,
+            "peak_GBs": peaks["hbm_gbs"], "peak_TFLOPs": peak_tf,
+            "frac": max(t_hbm, t_tc) * 1e3 / ms,
+            "note": "frac = max(algorithmic bytes / HBM peak, symmetric-Gram flops / tensor peak) / measured"}
+
+
+def measure_cell(P, dp, name, B, T, d_model, n_blocks, tied, positions, sigma, peaks, sampler, seed,
+                 warmup=3, replays=10):
+    """One configuration with inputs drawn on the device: replays of the captured step graph."""
+    import torch
+    dev = torch.cuda.current_device()
+    torch.cuda.synchronize()
+    torch.cuda.empty_cache()
+    torch.cuda.reset_peak_memory_stats(dev)
+    ds = P.synthesize_on_device(name, B, T, d_model, n_blocks, tied=tied, positions=positions,
+                                sigma=sigma, seed=seed)
+    counts = work_counts(shape_of(ds, name))
+    sg = P.StepGraph(ds, seed=seed, first_step=0)
+    for _ in range(warmup):
+        sg.replay()
+    torch.cuda.synchronize()
+    a, b = _ev(), _ev()
+    t0 = time.time()
+    a.record()
+    for _ in range(replays):
+        sg.replay()
+    b.record()
+    torch.cuda.synchronize()
+    t1 = time.time()
+    assert int(ds.dev_status.item()) == 0, "device status flagged a problem in %s B=%d T=%d" % (name, B, T)
+    ms = a.elapsed_time(b) / replays
+    clocks = sampler.window(t0, t1) if sampler else None
+    peak_tf, which, why = choose_tensor_peak(peaks, (t1 - t0), clocks)
+    ph = graph_phase_times(P, ds, seed, warmup + replays, replays, batches=3)
+    gemm_tf = counts["acc_flops"] / (ph["gemm"] * 1e-3) / 1e12
+    ghost = ghost_norm_alone(dp, ds, peaks, peak_tf, counts)
+    cell = {"workload": name, "B": B, "T": T, "blocks": n_blocks, "d_model": d_model, "tied": tied,
+            "positions": positions, "replays": replays, "ms_per_step": ms,
+            "examples_per_s": B / (ms * 1e-3), "norms_ms": ph["norms"],
+            "clip_accumulate_ms": ph["clip_accumulate"], "norm_plus_clip_ms": ph["norms"] + ph["clip_accumulate"],
+            "gemm": {"ms": ph["gemm"], "achieved_TFLOPs": gemm_tf, "peak_TFLOPs": peak_tf,
+                     "peak": which, "frac": gemm_tf / peak_tf},
+            "ghost_norm": {k: ghost[k] for k in ("kernel", "bound", "ms", "achieved_GBs",
+                                                   "achieved_TFLOPs", "frac")},
+            "input_bytes": int(ds.input_bytes()),
+            "max_memory_allocated_bytes": int(torch.cuda.max_memory_allocated(dev)),
+            "clocks": clocks}
+    return cell, ds
+
+
+def cross_term_alone(dp, ds):
+    """The tied cross-term call alone (five calls in one graph), in microseconds."""
+    import torch
+    sq = torch.zeros_like(ds.sq)
+    ms = time_graph(lambda: dp.dp_tied_cross_term(ds.ids, ds.G_emb, ds.lm.A, ds.lm.G, ds.V, sq=sq,
+                                                  cross=ds.cross, d=ds.d_model, ws=ds.ws,
+                                                  dev_status=ds.dev_status), reps=5)
+    return ms * 1e3
+
+
+def norm_modes(dp, ds, peaks):
+    """GHOST against DIRECT per distinct layer shape of this workload (the per-layer switch):
+    device time of one dp_ghost_norms call on that one layer in each forced mode, and what the
+    AUTO rule (DIRECT iff T^2 > d p) picks."""
+    import torch
+    seen, rows = set(), []
+    for l in ds.linears + ([ds.lm] if ds.lm else []):
+        if (l.d, l.p) in seen:
+            continue
+        seen.add((l.d, l.p))
+        sq = torch.zeros_like(ds.sq)
+        row = {"d": l.d, "p": l.p, "T": ds.T, "B": ds.B}
+        for label, mode in (("ghost_ms", dp.DP_NORM_GHOST), ("direct_ms", dp.DP_NORM_DIRECT)):
+            one = dp.Linear(l.A, l.G, d=l.d, p=l.p, mode=mode)
+            ws = torch.empty(max(256, dp.dp_ghost_norms_ws_bytes([one], ds.B, ds.T)), dtype=torch.uint8,
+                             device=sq.device)
+            row[label] = time_graph(lambda: dp.dp_ghost_norms([one], ds.B, ds.T, sq, ws=ws,
+                                                               dev_status=ds.dev_status), reps=3)
+        auto = dp.Linear(l.A, l.G, d=l.d, p=l.p, mode=dp.DP_NORM_AUTO)
+        used = dp.dp_ghost_norms([auto], ds.B, ds.T, sq, dev_status=ds.dev_status)
+        row["auto_chose"] = "direct" if used[0] == dp.DP_NORM_DIRECT else "ghost"
+        row["direct_TFLOPs"] = 2.0 * ds.B * ds.T * l.d * l.p / (row["direct_ms"] * 1e-3) / 1e12
+        row["ghost_GBs"] = 2.0 * ds.B * ds.T * (l.d + l.p) / (row["ghost_ms"] * 1e-3) / 1e9
+        rows.append(row)
+    torch.cuda.synchronize()
+    return rows
+
+
+SWEEP_CELLS = [
+    # name, B, T, d_model, blocks, tied, positions, sigma
+    ("cfg2", 32, 128, 768, 6, False, False, 0.8),
+    ("cfg4", 32, 128, 768, 12, True, False, 0.8),
+    ("cfg5", 16, 128, 1024, 24, False, False, 1.0),
+    ("cfg5", 64, 128, 1024, 24, False, False, 1.0),
+    ("cfg5", 256, 128, 1024, 24, False, False, 1.0),
+    ("cfg5", 16, 512, 1024, 24, False, False, 1.0),
+    ("cfg5", 64, 512, 1024, 24, False, False, 1.0),
+    ("cfg5", 256, 512, 1024, 24, False, False, 1.0),
+]
+
+
+def run_sweep(P, dp, peaks, sampler, seed):
+    """The other configurations, a few graph replays each, inputs drawn on the device.  Under cfg4
+    (tied) also: the cross-term kernel alone, the same shape untied, peak memory of both."""
+    import torch
+    out, tied_cost = [], None
+    for (name, B, T, dm, nb, tied, pos, sigma) in SWEEP_CELLS:
+        cell, ds = measure_cell(P, dp, name, B, T, dm, nb, tied, pos, sigma, peaks, sampler, seed)
+        if tied:
+            cross_us = cross_term_alone(dp, ds)
+            del ds
+            untied, ds2 = measure_cell(P, dp, name + "-untied", B, T, dm, nb, False, pos, sigma, peaks,
+                                       sampler, seed)
+            del ds2
+            tied_cost = {
+                "shape": "B=%d T=%d, %d blocks, d=%d, V=50257" % (B, T, nb, dm),
+                "cross_term_kernel_us": cross_us,
+                "tied_ms_per_step": cell["ms_per_step"], "untied_same_shape_ms_per_step": untied["ms_per_step"],
+                "step_delta_ms": cell["ms_per_step"] - untied["ms_per_step"],
+                "tied_norms_ms": cell["norms_ms"], "untied_norms_ms": untied["norms_ms"],
+                "tied_max_memory_allocated_bytes": cell["max_memory_allocated_bytes"],
+                "untied_max_memory_allocated_bytes": untied["max_memory_allocated_bytes"],
+                "note": ("tied: one shared 50257 x d matrix receives the head GEMM and the token scatter; "
+                         "untied holds two.  The cross term is 2<g_in, g_out> per example through the "
+                         "T x T pair expansion (no V x d matrix is formed)")}
+        else:
+            del ds
+        out.append(cell)
+        torch.cuda.empty_cache()
+    return out, tied_cost
+
+
 # ------------------------------------------------------------------------------ our arm
 def run_ours(args):
-    import numpy as np
     import torch
     import torch.distributed as dist
 
     from paper_2609_40335_b200 import binding as dp
+    from paper_2609_40335_b200 import parallel
     from paper_2609_40335_b200 import pipeline as P
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -225,28 +453,25 @@ def run_ours(args):
 
     # every rank holds its own batch of the same shape (weak scaling over examples)
     if args.device_inputs:
-        # large sweep cells: inputs drawn on the device (host generation would take minutes)
-        import types
         assert args.workload == "cfg5", "--device-inputs is for the GPT-2-medium sweep"
         B_, T_ = args.B or 16, args.T or 128
         ds = P.synthesize_on_device("cfg5", B_, T_, 1024, 24, seed=rank, device=dev)
-        w = types.SimpleNamespace(
-            name="cfg5", dtype="bf16", B=B_, T=T_, V=50257, d_model=1024, tied=False, positions=False,
-            linears=[types.SimpleNamespace(d=l.d, p=l.p) for l in ds.linears],
-            lm=types.SimpleNamespace(d=ds.lm.d, p=ds.lm.p))
+        w = shape_of(ds, "cfg5")
     else:
         w = make_workload(args.workload, seed=rank, B=args.B, T=args.T, full_model=args.full_model)
         ds = P.upload(w, dev)
     counts = work_counts(w)
     stream = torch.cuda.current_stream()
 
-    from paper_2609_40335_b200 import parallel
-
-    def reduce_sums():
-        # data-parallel exchange: clipped sums are added over ranks before the single noise draw
-        parallel.reduce_clipped_sums(ds.outs)
-
     fused = (world == 1) and not args.unfused     # noise inside the clipped-sum kernels
+    exchange = None
+    if world > 1 and args.exchange == "reduce_scatter":
+        # bucketed reduce-scatter on a communication stream; each rank noises the slices it owns
+        step_box = [0]
+        exchange = parallel.BucketedExchange(
+            ds.outs, lambda t, first, tid, st: dp.dp_add_noise_slice(
+                t, first, ds.sigma, ds.C, 1.0, args.seed, tid, step_box[0], stream=st),
+            gather=args.gather)
 
     def step(k, ev=None):
         ge = (ev[4], ev[5]) if ev else None
@@ -264,17 +489,19 @@ def run_ours(args):
         elif fused:
             P.clip_after_prefill(ds, args.seed, k, filled, gemm_events=ge)
             if ev: ev[2].record(stream)
+        elif exchange is not None:
+            # N > 1 (default): the clipped sums leave bucket by bucket while the next bucket computes
+            step_box[0] = k
+            exchange.begin_step()
+            P.clip_phase_bucketed(ds, exchange)
+            if ev: ev[2].record(stream)
+            exchange.finish()
         else:
             P.clip_phase(ds, gemm_events=ge)
             if ev: ev[2].record(stream)
-            if world > 1 and args.exchange == "reduce_scatter":
-                # each rank noises only the slice it owns (same stream as a single-GPU draw)
-                parallel.reduce_scatter_then_noise(
-                    ds.outs, lambda t, first, tid: dp.dp_add_noise_slice(
-                        t, first, ds.sigma, ds.C, 1.0, args.seed, tid, k))
-            else:
-                reduce_sums()
-                P.noise_phase(ds, seed=args.seed, step=k)
+            if world > 1:
+                parallel.reduce_clipped_sums(ds.outs)
+            P.noise_phase(ds, seed=args.seed, step=k)
         if ev: ev[3].record(stream)
 
     # default at N = 1: the whole step captured once as a CUDA graph and replayed (the noise step
@@ -291,9 +518,8 @@ def run_ours(args):
             use_graph = False
             graph_note = "graph capture failed (%s: %s); the step was issued call by call" % (
                 type(e).__name__, str(e).splitlines()[0][:120] if str(e) else "")
+    eager_step = step
     if use_graph:
-        eager_step = step
-
         def step(k, ev=None):          # noqa: F811  (replaces the eager step for every later use)
             sg.replay()
 
@@ -302,12 +528,12 @@ def run_ours(args):
     torch.cuda.synchronize()
     assert int(ds.dev_status.item()) == 0, "device status %#x flagged a problem during warm-up" % int(ds.dev_status.item())
 
-    sampler = ClockSampler(local)
-    if rank == 0:
+    sampler = ClockSampler(local) if rank == 0 else None
+    if sampler:
         sampler.start()
         time.sleep(0.25)
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    evs = [[_ev() for _ in range(6)] for _ in range(args.steps)] if not use_graph else None
+    e0, e1 = _ev(), _ev()
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
@@ -315,7 +541,7 @@ def run_ours(args):
     t_wall0 = time.time()
     e0.record(stream)
     for k in range(args.steps):
-        step(args.warmup + k, evs[k])
+        step(args.warmup + k, evs[k] if evs else None)
     e1.record(stream)
     torch.cuda.synchronize()
     t_wall1 = time.time()
@@ -324,7 +550,7 @@ def run_ours(args):
     launches = dp.dp_kernel_launches() - launches0
     if use_graph:
         launches = sg.kernels_per_replay * args.steps      # replays do not pass through the library
-    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    clocks = sampler.window(t_wall0, t_wall1) if sampler else None
     ms_total = e0.elapsed_time(e1)
     if world > 1:
         t = torch.tensor([ms_total], device=dev)
@@ -333,88 +559,52 @@ def run_ours(args):
     assert int(ds.dev_status.item()) == 0, "device status flagged a problem in the timed region"
     ms_step = ms_total / args.steps
     value = world * w.B / (ms_step * 1e-3)
+    peak_tf, peak_kind, peak_why = choose_tensor_peak(peaks, ms_total * 1e-3, clocks)
+
     graph_detail = None
     if use_graph:
-        # per-phase and GEMM durations: external CUDA events inside the graph, read after each of
-        # K more replays (the events of the timed region's last replay are read first)
-        sgt = P.StepGraph(ds, seed=args.seed, first_step=args.warmup + args.steps, timing=True)
-        det = []
-        for _ in range(args.steps):
-            sgt.replay()
-            torch.cuda.synchronize()
-            det.append(sgt.phase_ms())
-        ms_norm = statistics.mean(d["norms"] for d in det)
-        ms_clip = statistics.mean(d["clip_accumulate"] for d in det)
-        ms_noise = 0.0
+        ph = graph_phase_times(P, ds, args.seed, args.warmup + args.steps, args.steps)
+        ms_norm, ms_clip, ms_noise, gemm_ms_avg = ph["norms"], ph["clip_accumulate"], 0.0, ph["gemm"]
         graph_detail = {"how": "phases and the GEMM are timed by external CUDA events inside a second "
-                               "capture of the same step (the event nodes cost ~40 us per step, so "
-                               "the timed region replays a capture without them); averages over %d "
-                               "replays, each read after a synchronize" % args.steps,
-                        "step_ms_with_event_nodes": statistics.mean(d["step"] for d in det)}
+                               "capture of the same step (the event nodes cost tens of microseconds per "
+                               "step, so the timed region replays a capture without them): %d runs of "
+                               "%d back-to-back replays, the last replay of each run read, medians"
+                               % (ph["samples"], ph["replays_per_sample"]),
+                        "step_ms_with_event_nodes": ph["step_with_event_nodes"]}
     else:
         ms_norm = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
         ms_clip = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
         ms_noise = statistics.mean(e[2].elapsed_time(e[3]) for e in evs)
+        if fused and args.prefill or exchange is not None:
+            gemm_ms_avg = ms_clip
+        else:
+            gemm_ms_avg = statistics.mean(e[4].elapsed_time(e[5]) for e in evs)
 
-    # dominant kernel: the tensor-core G^T A GEMM of the clipped sums.  Its duration is taken
-    # live inside the timed region: CUDA events bracket the grouped call in every timed step (the
-    # bracket also holds the call's one clip-factor kernel, ~2 us).  With --prefill the GEMM
-    # accumulates onto pre-filled noise and is not bracketed.
-    lin_layers = ds.linears + ([ds.lm] if ds.lm else [])
-    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    if use_graph:
-        gemm_ms_avg = statistics.mean(d["gemm"] for d in det)
-    elif fused and args.prefill:
-        gemm_ms_avg = ms_clip
-    else:
-        gemm_ms_avg = statistics.mean(e[4].elapsed_time(e[5]) for e in evs)
-    n_gemm = 1          # one persistent launch over the output tiles of all layers
+    # dominant kernel: the tensor-core G^T A GEMM of the clipped sums, timed live (see above)
     achieved_tf = counts["acc_flops"] / (gemm_ms_avg * 1e-3) / 1e12
-    peak_tf = peaks["bf16_tflops_sustained"]
     roofline = {"kernel": "gemm_gta_kernel<scale, pair> (%s)" % (
                     "dp_clip_accumulate_noise_grouped, Gaussian noise drawn in the epilogue" if fused
                     else "dp_clip_accumulate_grouped"),
                 "bound": "tensor",
                 "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
-                "frac": achieved_tf / peak_tf, "peak_source": peaks["source"] + " sustained bf16 (kernel timed inside the long step)",
+                "frac": achieved_tf / peak_tf,
+                "peak_source": "%s %s bf16 peak: %s" % (peaks["source"], peak_kind, peak_why),
                 "frac_of_burst_peak": achieved_tf / peaks["bf16_tflops"],
-                "launches_per_step": n_gemm, "ms_per_launch_avg": gemm_ms_avg / n_gemm,
-                "flops_per_launch": counts["acc_flops"], "traffic": GEMM_TRAFFIC_BYTES.get(w.name)}
-    # the norm phase is HBM-bound at T=128: algorithmic bytes = every A and G read once
-    # (five calls captured into one CUDA graph: issued call by call, the host's work per call --
-    # 50 tensor maps -- would be what the events see, not the kernel)
-    reps = 5
-    torch.cuda.synchronize()
-    gg = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(gg):
-        for _ in range(reps):
-            ds.sq.zero_()
-            dp.dp_ghost_norms(lin_layers, ds.B, ds.T, ds.sq, ws=ds.ws, dev_status=ds.dev_status)
-    gg.replay()
-    torch.cuda.synchronize()
-    g0.record(stream)
-    gg.replay()
-    g1.record(stream)
-    torch.cuda.synchronize()
-    ghost_ms = g0.elapsed_time(g1) / reps
-    ghost_gbs = counts["norm_bytes"] / (ghost_ms * 1e-3) / 1e9
-    ghost_tf = counts["gram_flops"] / (ghost_ms * 1e-3) / 1e12
-    floor_ms = max(counts["norm_bytes"] / (peaks["hbm_gbs"] * 1e9),
-                   counts["gram_flops"] / (peak_tf * 1e12)) * 1e3
+                "frac_of_sustained_peak": achieved_tf / peaks["bf16_tflops_sustained"],
+                "launches_per_step": 1 if exchange is None else 4, "ms_per_launch_avg": gemm_ms_avg,
+                "timed_bracket": ("the grouped GEMM call" if exchange is None else
+                                  "the whole clip phase (four GEMM launches, scatters, vectors): N > 1"),
+                "flops_per_launch": counts["acc_flops"],
+                "traffic": int(GEMM_DRAM_OVER_ALGORITHMIC * counts["acc_bytes"]),
+                "traffic_how": ("%.2f x the launch's algorithmic bytes (%d): DRAM read + write of one ncu "
+                                "capture of a three-wave launch of this kernel, scaled by bytes"
+                                % (GEMM_DRAM_OVER_ALGORITHMIC, counts["acc_bytes"]))}
+    ghost = ghost_norm_alone(dp, ds, peaks, peak_tf, counts)
     big = ds.outs["wte"]
     noise_n = big.numel()
-    g0.record(stream)
-    for k in range(reps):
-        dp.dp_add_noise(big, ds.sigma, ds.C, 1.0, args.seed, 0, k)
-    g1.record(stream)
-    torch.cuda.synchronize()
-    noise_ms = g0.elapsed_time(g1) / reps
+    noise_ms = time_graph(lambda: dp.dp_add_noise(big, ds.sigma, ds.C, 1.0, args.seed, 0, 0), reps=5)
     others = {
-        "ghost_norm_tc_kernel (dp_ghost_norms)": {
-            "bound": "hbm" if counts["norm_bytes"] / (peaks["hbm_gbs"] * 1e9) >=
-            counts["gram_flops"] / (peak_tf * 1e12) else "tensor",
-            "ms": ghost_ms, "achieved_GBs": ghost_gbs, "achieved_TFLOPs": ghost_tf,
-            "peak_GBs": peaks["hbm_gbs"], "frac": floor_ms / ghost_ms},
+        "%s (dp_ghost_norms)" % ghost["kernel"]: ghost,
         "add_noise_kernel (dp_add_noise, %d elements)" % noise_n: {
             "bound": "hbm", "ms": noise_ms, "achieved_GBs": 8 * noise_n / (noise_ms * 1e-3) / 1e9,
             "peak_GBs": peaks["hbm_gbs"], "frac": 8 * noise_n / (noise_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
@@ -422,9 +612,10 @@ def run_ours(args):
 
     # end to end through the public API with HOST buffers: every step copies the step's inputs
     # from pinned host memory and reads the per-example norms and clip factors back
+    lin_layers = ds.linears + ([ds.lm] if ds.lm else [])
     host_in, dev_in = [], []
     seen = set()
-    e2e_enabled = ds.input_bytes() < 8e9 and not args.device_inputs
+    e2e_enabled = ds.input_bytes() < 12e9 and not args.device_inputs
     for t in ([ds.ids, ds.G_emb] + [x for l in lin_layers for x in (l.A, l.G)]) if e2e_enabled else []:
         if t.data_ptr() in seen:
             continue
@@ -444,20 +635,23 @@ def run_ours(args):
         host_out[1].copy_(ds.clip, non_blocking=True)
         torch.cuda.synchronize()
 
-    e2e_steps = max(3, min(args.steps, 10)) if e2e_enabled else 1
-    e2e_step(0)
-    if world > 1:
-        dist.barrier()
-    torch.cuda.synchronize()
-    t0 = time.perf_counter()
-    for k in range(e2e_steps):
-        e2e_step(k)
-    t_e2e = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([t_e2e], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        t_e2e = float(t.item())
-    e2e_val = world * w.B * e2e_steps / t_e2e
+    e2e_val, e2e_steps = None, 0
+    if e2e_enabled:
+        e2e_steps = max(3, min(args.steps, 10))
+        e2e_step(0)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for k in range(e2e_steps):
+            e2e_step(k)
+        t_e2e = time.perf_counter() - t0
+        if world > 1:
+            t = torch.tensor([t_e2e], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            t_e2e = float(t.item())
+        e2e_val = world * w.B * e2e_steps / t_e2e
+    del host_in
 
     if rank != 0:
         if world > 1:
@@ -467,7 +661,8 @@ def run_ours(args):
     # CPU baseline: the oracle on a bounded sample, on this machine's host cores (rank 0, N=1 only)
     cpu = None
     if world == 1 and not args.no_cpu_baseline and not args.device_inputs:
-        n_ex = min(w.B, 16)
+        t1 = oracle_sample_step(w, 1)
+        n_ex = max(1, min(w.B, 16, int(20.0 / max(t1, 1e-3))))       # about 20 s of oracle work
         t_ex = oracle_sample_step(w, n_ex)
         n_noise = 4_000_000
         t_noise = oracle_noise_seconds(n_noise)
@@ -481,16 +676,17 @@ def run_ours(args):
     # the same step issued call by call (no graph), for comparison
     graph_info = None
     if use_graph:
+        n_eager = min(args.steps, 100)
         for k in range(3):
             eager_step(k)
-        q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        q0, q1 = _ev(), _ev()
         torch.cuda.synchronize()
         q0.record(stream)
-        for k in range(args.steps):
+        for k in range(n_eager):
             eager_step(k)
         q1.record(stream)
         torch.cuda.synchronize()
-        e_ms = q0.elapsed_time(q1) / args.steps
+        e_ms = q0.elapsed_time(q1) / n_eager
         assert int(ds.dev_status.item()) == 0, "device status flagged a problem in the eager steps"
         graph_info = {"timed_region": "replays of pipeline.StepGraph (one CUDA graph launch per step)",
                       "kernels_per_replay": int(sg.kernels_per_replay),
@@ -498,15 +694,32 @@ def run_ours(args):
     memory = {"max_allocated_bytes": int(torch.cuda.max_memory_allocated(dev)),
               "input_bytes": int(ds.input_bytes())}
 
+    # ghost vs direct per layer shape of this workload, the other configurations, the tied path
+    modes = sweep = tied_cost = None
+    if world == 1 and not args.no_sweep and w.dtype == "bf16":
+        modes = norm_modes(dp, ds, peaks)
+        # free this workload's tensors first: the largest sweep cell needs ~25 GB by itself
+        n_lin, has_lm, n_vec = len(w.linears), bool(w.lm), len(getattr(w, "vectors", []) or [])
+        sg = None
+        eager_step = step = e2e_step = None
+        del ds, lin_layers, dev_in, big
+        torch.cuda.empty_cache()
+        sweep, tied_cost = run_sweep(P, dp, peaks, sampler, args.seed)
+    else:
+        n_lin, has_lm, n_vec = len(w.linears), bool(w.lm), len(getattr(w, "vectors", []) or [])
+    if sampler:
+        sampler.stop()
+
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": w.dtype if w.dtype != "f32" else "f32", "data": "synthetic",
-        "config": {"workload": w.name, "B_per_gpu": w.B, "T": w.T, "V": w.V, "layers": len(w.linears),
-                   "lm_head": bool(w.lm), "tied": w.tied, "positions": w.positions,
-                   "bias_and_layernorm_params": len(getattr(w, "vectors", []) or []),
-                   "accumulate": "fp32", "input_bytes_per_step": ds.input_bytes(),
-                   "l2": "inputs (%.2f GB per step) are larger than the 126 MB L2" % (ds.input_bytes() / 1e9)},
+        "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": w.name, "B_per_gpu": w.B, "T": w.T, "V": w.V, "layers": n_lin,
+                   "lm_head": has_lm, "tied": w.tied, "positions": w.positions,
+                   "bias_and_layernorm_params": n_vec,
+                   "accumulate": "fp32", "input_bytes_per_step": memory["input_bytes"],
+                   "exchange": (args.exchange + (" + all_gather" if args.gather else "")) if world > 1 else None,
+                   "l2": "inputs (%.2f GB per step) are larger than the 126 MB L2" % (memory["input_bytes"] / 1e9)},
         "phases_ms": {"norms": ms_norm, "clip_accumulate": ms_clip, "noise": ms_noise,
                       "norm_plus_clip": ms_norm + ms_clip,
                       "noise_fused_into_clip_accumulate": fused},
@@ -520,6 +733,10 @@ def run_ours(args):
         "e2e": ({"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
                  "d2h_bytes_per_step": int(d2h), "steps": e2e_steps} if e2e_enabled else None),
         "cpu_baseline": cpu,
+        "norm_modes": modes,
+        "tied_extra_cost": tied_cost,
+        "sweep": sweep,
+        "exchange_bytes_per_rank_per_step": exchange.bytes_on_wire if exchange is not None else None,
         "peaks": peaks,
     }
     print(json.dumps(line), flush=True)
@@ -527,20 +744,124 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------- small single-entry-point cases (profilers)
+def run_case(args):
+    """One entry point a few times on a small case: inputs larger than the 126 MB L2 but well
+    under a few GB, so that a multi-pass profiler capture stays short.  Prints one JSON line."""
+    import torch
+
+    from paper_2609_40335_b200 import binding as dp
+
+    torch.cuda.set_device(0)
+    torch.manual_seed(0)
+    dp.load()
+    reps = args.reps
+
+    def rb(*shape, std=1.0):
+        return (torch.randn(*shape, device="cuda") * std).to(torch.bfloat16)
+
+    def timed(fn):
+        fn()
+        a, b = _ev(), _ev()
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    out = {"case": args.case, "reps": reps}
+    c = args.case
+    if c in ("gemm", "gemm_unclipped", "gemm_noise"):
+        # one layer 768 -> 18944 at B=32, T=128: 74 x 3 output tiles of 256 x 256, three waves
+        B, T = 32, 128
+        L = [dp.Linear(rb(B, T, 768), rb(B, T, 148 * 128, std=1e-2))]
+        outs = [torch.empty(148 * 128, 768, device="cuda")]
+        sq = torch.full((B,), 1e-12 if c == "gemm_unclipped" else 4.0, device="cuda")
+        if c == "gemm_noise":
+            ms = timed(lambda: dp.dp_clip_accumulate_noise_grouped(L, B, T, sq, 1.0, outs, 0.8, 1.0, 0, [0], 0))
+        else:
+            ms = timed(lambda: dp.dp_clip_accumulate_grouped(L, B, T, sq, 1.0, outs))
+        out.update(ms=ms, TFLOPs=2 * B * T * 768 * 148 * 128 / ms / 1e9)
+    elif c == "direct":
+        # DIRECT norm (gradient tiles in tensor memory, square-sum epilogue): 768 -> 3072, T = 256
+        B, T = 64, 256
+        L = [dp.Linear(rb(B, T, 768), rb(B, T, 3072, std=1e-2), mode=dp.DP_NORM_DIRECT) for _ in range(4)]
+        sq = torch.zeros(B, device="cuda")
+        ms = timed(lambda: dp.dp_ghost_norms(L, B, T, sq))
+        out.update(ms=ms, TFLOPs=len(L) * 2 * B * T * 768 * 3072 / ms / 1e9)
+    elif c == "ghost":
+        B, T = 32, 128
+        L = [dp.Linear(rb(B, T, 768), rb(B, T, 3072, std=1e-2)) for _ in range(6)]
+        L.append(dp.Linear(rb(B, T, 768), rb(B, T, 16384, std=1e-2)))
+        sq = torch.zeros(B, device="cuda")
+        ms = timed(lambda: dp.dp_ghost_norms(L, B, T, sq))
+        out.update(ms=ms, GBs=sum(2 * B * T * (l.A.shape[-1] + l.G.shape[-1]) for l in L) / ms / 1e6)
+    elif c == "ghost512":
+        B, T = 64, 512
+        L = [dp.Linear(rb(B, T, 1024), rb(B, T, 4096, std=1e-2)) for _ in range(2)]
+        sq = torch.zeros(B, device="cuda")
+        ms = timed(lambda: dp.dp_ghost_norms(L, B, T, sq))
+        out.update(ms=ms, TFLOPs_needed=len(L) * B * T * (T + 1) * 5120 / ms / 1e9,
+                   GBs=len(L) * B * 2 * T * 5120 / ms / 1e6)
+    elif c == "noise":
+        x = torch.zeros(50257 * 768, device="cuda")
+        ms = timed(lambda: dp.dp_add_noise(x, 0.8, 1.0, 1.0, 1234, 0, 0))
+        out.update(ms=ms, GBs=8 * x.numel() / ms / 1e6)
+    elif c in ("embed", "embed_small"):
+        B, T, d, V = (256, 512, 1024, 50257) if c == "embed" else (32, 128, 768, 50257)
+        w = torch.arange(1, V + 1, device="cuda", dtype=torch.float64) ** -1.1
+        ids = torch.multinomial(w / w.sum(), B * T, replacement=True).to(torch.int32).view(B, T)
+        G = rb(B, T, d, std=1e-2)
+        sq = torch.zeros(B, device="cuda")
+        o = torch.empty(V, d, device="cuda")
+
+        def both():
+            dp.dp_embed_norms(ids, G, V, sq)
+            dp.dp_clip_accumulate_embed(ids, G, V, sq, 1.0, o)
+        out.update(ms=timed(both))
+    elif c == "cross":
+        B, T, d, V = 32, 128, 768, 50257
+        ids = torch.randint(0, V, (B, T), device="cuda", dtype=torch.int32)
+        Ge, Al, Gl = rb(B, T, d, std=1e-2), rb(B, T, d), rb(B, T, 50264, std=1e-2)
+        sq = torch.zeros(B, device="cuda")
+        out.update(ms=timed(lambda: dp.dp_tied_cross_term(ids, Ge, Al, Gl, V, sq=sq, d=d)))
+    elif c == "vectors":
+        B, T = 32, 128
+        vec = []
+        for _ in range(6):
+            for p_, with_x in [(768, True), (768, False), (2304, False), (768, False), (768, True),
+                               (768, False), (3072, False), (768, False)]:
+                vec.append(dp.Vector(rb(B, T, p_, std=1e-2), rb(B, T, p_) if with_x else None, p=p_))
+        sq = torch.zeros(B, device="cuda")
+        outs = [torch.empty(v.p, device="cuda") for v in vec]
+
+        def both():
+            dp.dp_vector_norms(vec, B, T, sq)
+            dp.dp_clip_accumulate_vectors(vec, B, T, sq, 1.0, outs)
+        out.update(ms=timed(both))
+    else:
+        raise SystemExit("unknown --case %r" % c)
+    print(json.dumps(out), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    # default long enough (~2 s of back-to-back steps) for the SM clock to settle under the power
-    # cap: the roofline is quoted against the SUSTAINED tensor peak, so the run must be sustained too
-    # (the reference arm, whose steps take ~0.6 s each, defaults to 20)
+    # default: enough back-to-back steps (about two seconds) for the SM clock to settle under the
+    # power cap; the reference arm, whose steps take seconds each, defaults to 20
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--exchange", default="all_reduce", choices=["all_reduce", "reduce_scatter"],
-                    help="N > 1: how the clipped sums are summed over ranks before the noise draw")
+    ap.add_argument("--exchange", default="reduce_scatter", choices=["all_reduce", "reduce_scatter"],
+                    help="N > 1: bucketed reduce-scatter on a communication stream, noise on the owned "
+                         "slice (default), or a blocking all-reduce per tensor followed by the noise pass")
+    ap.add_argument("--gather", action="store_true",
+                    help="N > 1, reduce_scatter: all-gather the noised slices back into the full tensors")
     ap.add_argument("--eager", action="store_true",
                     help="issue the step call by call instead of replaying a captured CUDA graph")
-    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--workload", default="cfg3")
     ap.add_argument("--B", type=int, default=0, help="override the workload's batch size (cfg5 sweep)")
     ap.add_argument("--T", type=int, default=0, help="override the workload's sequence length")
     ap.add_argument("--full-model", action="store_true",
@@ -549,12 +870,19 @@ def main():
                     help="cfg5 only: draw the inputs on the device (big cells)")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true",
+                    help="skip the sweep over the other configurations, norm_modes and the tied cost")
     ap.add_argument("--prefill", action="store_true", help="noise of every tensor filled beside the norms")
     ap.add_argument("--unfused", action="store_true",
-                    help="separate noise pass (what the multi-GPU path uses) instead of fused noise")
+                    help="separate noise pass instead of fused noise (N = 1)")
+    ap.add_argument("--case", default=None, help="run one small single-entry-point case and exit")
+    ap.add_argument("--reps", type=int, default=3)
     args = ap.parse_args()
+    if args.case:
+        run_case(args)
+        return
     if args.steps is None:
-        args.steps = 20 if args.impl == "reference" else 2000
+        args.steps = 20 if args.impl == "reference" else 400
     if args.impl == "reference":
         run_reference(args)      # any K: the per-step sample shrinks so that the run stays bounded
     else:

@@ -225,6 +225,45 @@ def clip_phase(ds: DeviceStep, stream=None, gemm_events=None) -> None:
     _clip_vectors(ds, 0.0, stream=stream)
 
 
+def clip_phase_bucketed(ds: DeviceStep, exchange, n_linear_buckets: int = 3) -> None:
+    """Clipped sums produced bucket by bucket -- the LM head first (tied: together with the token
+    scatter into the shared table), then the block linears in a few groups, then the remaining
+    tables and vectors -- with `exchange.submit(names)` called right after each bucket's kernels
+    were enqueued (a parallel.BucketedExchange: its collectives run on their own stream while the
+    next bucket computes).  ds.clip must already hold the clip factors."""
+    from . import parallel
+    kw = dict(ws=ds.ws, dev_status=ds.dev_status)
+    tied_head = ds.tied and ds.lm is not None
+
+    def scatter_tokens(beta):
+        dp.dp_clip_accumulate_embed(ds.ids, ds.G_emb, ds.V, None, ds.C, ds.outs["wte"], beta=beta,
+                                    d=ds.d_model, clip=ds.clip, **kw)
+
+    lin_names = [f"linear{k}" for k in range(len(ds.linears))]
+    by_name = dict(zip(lin_names, ds.linears))
+    head = None
+    if ds.lm is not None:
+        head = "wte" if ds.tied else "lm_head"
+        by_name[head] = ds.lm
+    last = ([] if tied_head else ["wte"]) + (["wpe"] if ds.positions else []) + \
+           [f"vector{k}" for k in range(len(ds.vectors))]
+    for bucket in parallel.bucket_order(lin_names, head, [], n_linear_buckets):
+        layers = [by_name[n] for n in bucket]
+        dp.dp_clip_accumulate_grouped(layers, ds.B, ds.T, None, ds.C, [ds.outs[n] for n in bucket],
+                                      beta=0.0, clip=ds.clip, **kw)
+        if tied_head and bucket == [head]:
+            scatter_tokens(1.0)              # the shared table receives both contributions (Eq. 8)
+        exchange.submit(bucket)
+    if not tied_head:
+        scatter_tokens(0.0)
+    if ds.positions:
+        dp.dp_clip_accumulate_embed(ds.pos_ids, ds.G_emb, WPE_ROWS, None, ds.C, ds.outs["wpe"],
+                                    beta=0.0, d=ds.d_model, clip=ds.clip, **kw)
+    _clip_vectors(ds, 0.0, factors=True)
+    if last:
+        exchange.submit(last)
+
+
 def noise_phase(ds: DeviceStep, seed: int, step: int, scale: float = 1.0, stream=None) -> None:
     """One Gaussian draw per parameter tensor; tensor_id = position in the sorted key order."""
     for tid, name in enumerate(sorted(ds.outs)):

@@ -65,20 +65,57 @@ def _seed_for(base_seed: int, *tag) -> int:
     return int.from_bytes(h[:8], "little")
 
 
-def _normal(shape, std, dtype, seed, ld=None) -> HostTensor:
+_CHUNK_ELEMS = 1 << 24
+
+
+def _normal_jobs(shape, std, dtype, seed, ld=None):
+    """The tensor (allocated, not yet filled) and the jobs that fill it.
+
+    A tensor is drawn in slabs along its first axis, at most 2^24 elements each and every slab from
+    its own generator (seeded by the tensor's seed and the slab number), so that the slabs can be
+    drawn in parallel and the values depend on the shape and the seed only -- not on how many
+    threads draw them.  A tensor of one slab uses the tensor's seed itself.
+    """
+    shape = tuple(int(v) for v in shape)
     cols = shape[-1]
     ld = cols if ld is None else int(ld)
-    rng = np.random.Generator(np.random.PCG64(seed))
-    x = rng.standard_normal(size=tuple(shape[:-1]) + (cols,), dtype=np.float32)
-    if std != 1.0:
-        x *= np.float32(std)
-    if ld != cols:
-        full = np.full(tuple(shape[:-1]) + (ld,), np.nan, dtype=np.float32)
-        full[..., :cols] = x
-        x = full
-    if dtype == "bf16":
-        return HostTensor(f32_to_bf16_bits(x), "bf16", cols)
-    return HostTensor(x, "f32", cols)
+    out = np.empty(shape[:-1] + (ld,), dtype=np.uint16 if dtype == "bf16" else np.float32)
+    per_row = int(np.prod(shape[1:], dtype=np.int64))
+    rows = max(1, _CHUNK_ELEMS // max(per_row, 1))
+    n_slabs = (shape[0] + rows - 1) // rows
+
+    def fill(k):
+        r0, r1 = k * rows, min(shape[0], (k + 1) * rows)
+        rng = np.random.Generator(np.random.PCG64(seed if n_slabs == 1 else _seed_for(seed, "slab", k)))
+        x = rng.standard_normal(size=(r1 - r0,) + shape[1:], dtype=np.float32)
+        if std != 1.0:
+            x *= np.float32(std)
+        if ld != cols:
+            full = np.full((r1 - r0,) + shape[1:-1] + (ld,), np.nan, dtype=np.float32)
+            full[..., :cols] = x
+            x = full
+        out[r0:r1] = f32_to_bf16_bits(x) if dtype == "bf16" else x
+
+    return HostTensor(out, dtype, cols), [(fill, k) for k in range(n_slabs)]
+
+
+def _run_jobs(jobs) -> None:
+    """Run fill jobs on a thread pool (numpy's generators and ufuncs release the GIL)."""
+    import concurrent.futures as cf
+    import os
+    workers = max(1, min(16, len(os.sched_getaffinity(0)), len(jobs)))
+    if workers == 1:
+        for fn, k in jobs:
+            fn(k)
+        return
+    with cf.ThreadPoolExecutor(max_workers=workers) as ex:
+        list(ex.map(lambda j: j[0](j[1]), jobs))
+
+
+def _normal(shape, std, dtype, seed, ld=None) -> HostTensor:
+    t, jobs = _normal_jobs(shape, std, dtype, seed, ld)
+    _run_jobs(jobs)
+    return t
 
 
 def zipf_ids(B: int, T: int, V: int, s: float, seed: int) -> np.ndarray:
@@ -159,6 +196,13 @@ def make_workload(name: str, *, B: int, T: int, dtype: str,
     biases of the block linears and the LayerNorm gains / shifts of a GPT-2 block (ln_1, ln_2,
     final ln_f), so that the parameter blocks cover the whole model.
     """
+    jobs = []
+
+    def _normal(shape, std, dtype, seed, ld=None):        # deferred: all tensors are drawn together
+        t, j = _normal_jobs(shape, std, dtype, seed, ld)
+        jobs.extend(j)
+        return t
+
     linears: List[LinearIO] = []
     cache = {}
     for blk in range(n_blocks):
@@ -207,6 +251,7 @@ def make_workload(name: str, *, B: int, T: int, dtype: str,
                 l = linears[blk * per_block + li]
                 vectors.append(VectorIO(f"{l.name}.bias", l.p, l.G, None))
         vectors += layer_norm("ln_f")
+    _run_jobs(jobs)
     return Workload(name, dtype, B, T, V, float(C), float(sigma), seed, linears, ids, G_emb,
                     lm, tied, positions, vectors)
 

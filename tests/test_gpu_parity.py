@@ -881,11 +881,46 @@ def test_step_graph_with_positions_and_full_parameter_set():
             assert torch.equal(a.outs[name], b.outs[name]), (k, name)
 
 
+@pytest.mark.parametrize("cfg", ["cfg3", "cfg4"])
+def test_bucketed_clip_phase_equals_the_plain_phases(cfg):
+    """The multi-GPU step order on one GPU: clipped sums produced bucket by bucket (head first), each
+    bucket handed to the exchange, which noises the slices it owns on its own stream -- same numbers
+    as clip phase + noise phase issued in one piece (K may be split differently: 1e-5 Frobenius)."""
+    from paper_2609_40335_b200 import parallel
+    w = W.named_workload(cfg, B=3, T=100, n_blocks=2, V=3001)
+    a, b = P.upload(w), P.upload(w)
+    P.dp_step(a, seed=9, step=4, fused=False)
+    P.norms_phase(b)
+    ex = parallel.BucketedExchange(
+        b.outs, lambda t, first, tid, st: dp.dp_add_noise_slice(t, first, b.sigma, b.C, 1.0, 9, tid, 4, stream=st))
+    ex.begin_step()
+    P.clip_phase_bucketed(b, ex, n_linear_buckets=3)
+    ex.finish()
+    torch.cuda.synchronize()
+    check_status(b.dev_status)
+    assert sorted(ex.submitted) == sorted(b.outs)
+    for name in a.outs:
+        assert frob_rel(b.outs[name].cpu().numpy(), a.outs[name].cpu().numpy()) < 1e-5, name
+        lo, hi, mine = ex.owned[name]
+        assert (lo, hi) == (0, a.outs[name].numel()) and mine.data_ptr() == b.outs[name].data_ptr()
+
+
 # ------------------------------- full-size configurations in the launch configuration of the bench
+def _oracle_example(w, i):
+    """The oracle's squared norm (and, tied, cross term) of example i over every layer of w."""
+    sl = slice(i, i + 1)
+    lin = [(l.A.widened_rows(sl), l.G.widened_rows(sl)) for l in w.linears]
+    return O.dp_step(lin, w.ids[sl], w.G_emb.widened_rows(sl), w.V, w.C,
+                     lm=(w.lm.A.widened_rows(sl), w.lm.G.widened_rows(sl)), tied=w.tied,
+                     positions=w.positions, want_sums=False)
+
+
 def _full_size_graph_check(w, examples, layers, lm_rows, table_rows, seed=7, first_step=3):
-    """One replay of the captured step graph (what bench.py times) at full size; the oracle checks
-    sampled outputs: norms (and cross terms) of `examples`, clip factors of all, the noised clipped
-    sums of `layers`, of rows `lm_rows` of the head and rows `table_rows` of the token table."""
+    """One replay of the captured step graph (what bench.py times) at full size against the oracle:
+    the norms (and cross terms) of `examples` (None: EVERY example of the batch), the clip factors of
+    all, the noised clipped sums of `layers`, of rows `lm_rows` of the head and rows `table_rows` of
+    the token table.  The clip factors that enter the expected sums are the ORACLE's wherever the
+    oracle computed the example's norm, so a wrong norm on the device cannot cancel out."""
     ds = P.upload(w)
     g = P.StepGraph(ds, seed=seed, first_step=first_step)
     g.replay()
@@ -894,18 +929,20 @@ def _full_size_graph_check(w, examples, layers, lm_rows, table_rows, seed=7, fir
     step = first_step                                        # replay k draws step first_step + k
     tid = P.tensor_ids(ds)
     sq_gpu = ds.sq.cpu().numpy().astype(np.float64)
-    for i in examples:
-        sl = slice(i, i + 1)
-        lin = [(l.A.widened_rows(sl), l.G.widened_rows(sl)) for l in w.linears]
-        ref = O.dp_step(lin, w.ids[sl], w.G_emb.widened_rows(sl), w.V, w.C,
-                        lm=(w.lm.A.widened_rows(sl), w.lm.G.widened_rows(sl)), tied=w.tied,
-                        positions=w.positions, want_sums=False)
+    cross_gpu = ds.cross.cpu().numpy() if w.tied else None
+    sq_ref = sq_gpu.copy()                                   # oracle values overwrite the checked entries
+    for i in (range(w.B) if examples is None else examples):
+        ref = _oracle_example(w, i)
         assert abs(sq_gpu[i] - ref["sq"][0]) / ref["sq"][0] < TIGHT_BF16, i
+        sq_ref[i] = ref["sq"][0]
         if w.tied:
             scale = np.sqrt(ref["sq_in"][0] * ref["sq_out"][0])
-            assert abs(ds.cross.cpu().numpy()[i] - ref["cross"][0]) / scale < TIGHT_BF16, i
-    _, R = O.clip_factors(sq_gpu, w.C)                       # Eq. 7 from the (checked) norms
-    assert rel(ds.clip.cpu().numpy(), R).max() < 1e-5
+            assert abs(cross_gpu[i] - ref["cross"][0]) / scale < TIGHT_BF16, i
+    norms_ref, R = O.clip_factors(sq_ref, w.C)               # Eq. 7 on the oracle's norms
+    assert rel(ds.clip.cpu().numpy(), R).max() < TIGHT_BF16
+    assert rel(ds.norms.cpu().numpy(), norms_ref).max() < TIGHT_BF16
+    _, R_own = O.clip_factors(sq_gpu, w.C)                   # the device's own Eq. 7 arithmetic
+    assert rel(ds.clip.cpu().numpy(), R_own).max() < 1e-5
     amp = w.sigma * w.C
 
     def noise(name, n, start=0):
@@ -947,25 +984,88 @@ HEAD_ROWS = [0, 1, 255, 256, 25000, 50175, 50176, 50256]
 def test_cfg2_full_size_graph_replay_sampled():
     w = W.named_workload("cfg2")
     hot = [int(np.bincount(w.ids.reshape(-1)).argmax()), int(w.ids[0, 0]), 0, 50256]
-    _full_size_graph_check(w, examples=(0, 31), layers=(0, 23), lm_rows=HEAD_ROWS, table_rows=hot)
+    # every example's norm against the oracle (about half a second of float64 each)
+    _full_size_graph_check(w, examples=None, layers=(0, 23), lm_rows=HEAD_ROWS, table_rows=hot)
 
 
 def test_cfg4_full_size_tied_graph_replay_sampled():
     w = W.named_workload("cfg4")
     hot = [int(np.bincount(w.ids.reshape(-1)).argmax())]
-    _full_size_graph_check(w, examples=(5,), layers=(2, 47), lm_rows=HEAD_ROWS + hot, table_rows=[])
+    # every example's tied norm and cross term against the oracle's materialised g_in + g_out
+    _full_size_graph_check(w, examples=None, layers=(2, 47), lm_rows=HEAD_ROWS + hot, table_rows=[])
 
 
 def test_cfg3_full_size_graph_replay_sampled():
     w = W.named_workload("cfg3")                             # B = 64, T = 256: the CTA-pair Gram kernel
     hot = [int(np.bincount(w.ids.reshape(-1)).argmax()), 50256]
-    _full_size_graph_check(w, examples=(63,), layers=(1,), lm_rows=HEAD_ROWS[:4], table_rows=hot)
+    spread = (0, 9, 17, 26, 34, 45, 54, 63)                  # eight examples across the batch
+    _full_size_graph_check(w, examples=spread, layers=(1,), lm_rows=HEAD_ROWS[:4], table_rows=hot)
 
 
 def test_cfg5_cell_full_size_graph_replay_sampled():
     w = W.named_workload("cfg5", B=16, T=128)                # GPT-2-medium shape, 97 layers
     hot = [int(np.bincount(w.ids.reshape(-1)).argmax())]
-    _full_size_graph_check(w, examples=(7,), layers=(3, 95), lm_rows=HEAD_ROWS[:4], table_rows=hot)
+    _full_size_graph_check(w, examples=(0, 7, 15), layers=(3, 95), lm_rows=HEAD_ROWS[:4], table_rows=hot)
+
+
+def _host_rows(t, i, cols):
+    """Example i of a device tensor (B, T, ld) as float64 on the host, padding columns dropped."""
+    return t[i:i + 1, :, :cols].float().cpu().numpy().astype(np.float64)
+
+
+@pytest.mark.parametrize("B,T", [(16, 128), (64, 128), (256, 128), (16, 512), (64, 512), (256, 512)])
+def test_cfg5_every_cell_one_example_against_the_oracle(B, T):
+    """Each (B, T) cell of the GPT-2-medium sweep at full size (inputs drawn on the device, 97
+    layers): one step, then the rows of a few examples are copied to the host and the float64
+    oracle materialises their per-example gradients layer by layer -- norm, clip factor, and the
+    device's whole vector of norms must be finite and deterministic."""
+    ds = P.synthesize_on_device("cfg5", B, T, 1024, 24, seed=11)
+    P.dp_step(ds, seed=5, step=2)
+    torch.cuda.synchronize()
+    check_status(ds.dev_status)
+    sq = ds.sq.cpu().numpy().astype(np.float64)
+    clip = ds.clip.cpu().numpy().astype(np.float64)
+    assert np.isfinite(sq).all() and (sq > 0).all()
+    every = ds.linears + [ds.lm]
+    for i in sorted({0, B // 2 + 1, B - 1})[: (3 if T == 128 else 2)]:
+        lin = [(_host_rows(l.A, i, l.d), _host_rows(l.G, i, l.p)) for l in ds.linears]
+        ref = O.dp_step(lin, ds.ids[i:i + 1].cpu().numpy(), _host_rows(ds.G_emb, i, ds.d_model), ds.V,
+                        ds.C, lm=(_host_rows(ds.lm.A, i, ds.lm.d), _host_rows(ds.lm.G, i, ds.lm.p)),
+                        want_sums=False)
+        assert abs(sq[i] - ref["sq"][0]) / ref["sq"][0] < TIGHT_BF16, (B, T, i)
+        assert abs(clip[i] - ref["clip"][0]) / ref["clip"][0] < TIGHT_BF16, (B, T, i)
+    assert len(every) == 97
+
+
+@pytest.mark.parametrize("T", [256, 200])
+def test_direct_norm_forced_on_every_gpt2_small_layer(T):
+    """The per-layer switch at GPT-2-small shapes (config 3): DIRECT forced on all four block
+    shapes and on the LM head (p = V), GHOST forced on the same layers, AUTO reported -- all three
+    against the oracle's materialised per-example gradients."""
+    B, V = 2, 50257
+    shapes = [(768, 2304), (768, 768), (768, 3072), (3072, 768), (768, V)]
+    host = [host_linear(B, T, d, p, "bf16", seed=31 * T + p + d, ldg=W.round_up(p, 8)) for d, p in shapes]
+    want = [O.linear_sq_norms(A.widened(), G.widened()) for A, G in host]
+    up = [(P.to_device(A), P.to_device(G)) for A, G in host]
+    st = torch.zeros(1, dtype=torch.int32, device=dev())
+    for mode in (dp.DP_NORM_DIRECT, dp.DP_NORM_GHOST, dp.DP_NORM_AUTO):
+        layers = [dp.Linear(a, g, d=d, p=p, mode=mode) for (a, g), (d, p) in zip(up, shapes)]
+        # one call over all layers (the grouped launch) and one call per layer
+        sq_all = torch.zeros(B, device=dev())
+        used = dp.dp_ghost_norms(layers, B, T, sq_all, dev_status=st)
+        torch.cuda.synchronize()
+        check_status(st)
+        if mode == dp.DP_NORM_AUTO:                          # T^2 <= d p everywhere: the rule picks GHOST
+            assert used == [dp.DP_NORM_GHOST] * len(layers)
+        else:
+            assert used == [mode] * len(layers)
+        assert rel(sq_all.cpu().numpy(), sum(want)).max() < TIGHT_BF16, mode
+        for k, l in enumerate(layers):
+            sq = torch.zeros(B, device=dev())
+            dp.dp_ghost_norms([l], B, T, sq, dev_status=st)
+            torch.cuda.synchronize()
+            check_status(st)
+            assert rel(sq.cpu().numpy(), want[k]).max() < TIGHT_BF16, (mode, shapes[k])
 
 
 @pytest.mark.parametrize("B,T", [(64, 512), (256, 128), (256, 512)])

@@ -45,6 +45,32 @@ def _worker(rank, world, port, ret):
     ret[f"rs{rank}"] = {k: v.numpy().copy() for k, v in outs2.items()}
     ret[f"own{rank}"] = {k: (lo, hi) for k, (lo, hi, _) in owned.items()}
     ret[f"clip{rank}"] = (lo, hi, res["clip"])
+
+    # bucketed form (what bench.py --gpus N runs): the tensors leave in the production order of the
+    # clipped sums, each bucket as soon as it exists; the owned slices tile every tensor
+    outs3 = {k: torch.from_numpy(v.copy()) for k, v in res["sums"].items()}
+    for gather in (False, True):
+        work = {k: v.clone() for k, v in outs3.items()}
+        ex = parallel.BucketedExchange(work, lambda t, first, tid, st: add_noise_slice(t, first, tid),
+                                       gather=gather)
+        ex.begin_step()
+        order = parallel.bucket_order(["linear0"], None, ["wte"], n_linear_buckets=3)
+        for bucket in order:
+            ex.submit(bucket)
+        ex.finish()
+        ret[f"bk{int(gather)}_{rank}"] = {k: (lo_, hi_, t.numpy().copy()) for k, (lo_, hi_, t) in ex.owned.items()}
+        if gather:
+            ret[f"bkfull{rank}"] = {k: v.numpy().copy() for k, v in work.items()}
+        ret[f"wire{int(gather)}_{rank}"] = ex.bytes_on_wire
+    try:                                   # a tensor that is never submitted is an error, not a silent skip
+        ex2 = parallel.BucketedExchange({k: v.clone() for k, v in outs3.items()},
+                                        lambda t, first, tid, st: None)
+        ex2.begin_step()
+        ex2.submit(["linear0"])
+        ex2.finish()
+        ret[f"missing{rank}"] = "not raised"
+    except RuntimeError as e:
+        ret[f"missing{rank}"] = str(e)
     dist.destroy_process_group()
 
 
@@ -84,3 +110,22 @@ def test_two_ranks_reproduce_the_single_process_step():
     for r in range(2):
         lo, hi, clip = ret[f"clip{r}"]
         np.testing.assert_allclose(clip, full["clip"][lo:hi], rtol=1e-12)
+    # bucketed exchange: every rank's owned slice holds the single-process values of that slice
+    for tid, k in enumerate(sorted(full["sums"])):
+        want = NO.add_noise(full["sums"][k], 0.5, C, 1.0, 3, tid, 11).reshape(-1)
+        for gather in (0, 1):
+            covered = 0
+            for r in range(2):
+                lo, hi, t = ret[f"bk{gather}_{r}"][k]
+                np.testing.assert_allclose(t, want[lo:hi], rtol=1e-12, atol=1e-12)
+                covered += hi - lo
+            assert covered == want.size
+        for r in range(2):
+            np.testing.assert_allclose(ret[f"bkfull{r}"][k].reshape(-1), want, rtol=1e-12, atol=1e-12)
+    assert ret["wire1_0"] == 2 * ret["wire0_0"] > 0
+    assert "never exchanged" in ret["missing0"] and "wte" in ret["missing0"]
+    # the bucket order: head first, the linears in contiguous groups, tables last, nothing lost
+    order = parallel.bucket_order([f"linear{k}" for k in range(7)], "lm_head", ["wte", "wpe"], 3)
+    assert order[0] == ["lm_head"] and order[-1] == ["wte", "wpe"]
+    assert [n for b in order[1:-1] for n in b] == [f"linear{k}" for k in range(7)]
+    assert len(order) == 5 and parallel.bucket_order([], None, ["wte"]) == [["wte"]]

@@ -1,10 +1,12 @@
 """dp_embed_norms_static: the embedding norm for callers that cannot allocate (its scratch is a
-fixed array inside the library).  Checked through the C ABI against dp_embed_norms on two calls
-in a row; collected last so that a run stopping at the first failure has run everything else."""
+fixed array inside the library).  Checked through the C ABI against dp_embed_norms, and against
+the float64 oracle's materialised embedding gradient, on two calls in a row; collected last so
+that a run stopping at the first failure has run everything else."""
 import numpy as np
 import pytest
 import torch
 
+from oracle import dp_oracle as O
 from paper_2609_40335_b200 import binding as dp
 from paper_2609_40335_b200 import pipeline as P
 from paper_2609_40335_b200 import workloads as W
@@ -36,6 +38,12 @@ def test_static_scratch_entry_point_matches_workspace_entry_point_twice():
         err = ((got - 0.5) - ref).abs() / ref
         assert float(err.max()) < 2e-3, (call, err)
         assert torch.equal(fo, fo_ref)
+        # and the oracle: the (V, d) embedding gradient of every example, materialised in float64
+        ids_h = ids.cpu().numpy()
+        G_h = G.float().cpu().numpy().astype(np.float64)
+        want = O.embed_sq_norms(ids_h, G_h, V)
+        assert np.abs((got.cpu().numpy() - 0.5) - want).max() / want.max() < 2e-3, call
+        assert np.array_equal(fo.cpu().numpy(), O.first_occurrence(ids_h))
     # sizes beyond the built-in array are refused with their own status, nothing is enqueued
     B, T, d = 1024, 8, 8192                                  # 1024 * 32 slabs > 16384 floats
     ids = torch.zeros(B, T, dtype=torch.int32, device=dev)
