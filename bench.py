@@ -761,15 +761,8 @@ def run_case(args):
         return (torch.randn(*shape, device="cuda") * std).to(torch.bfloat16)
 
     def timed(fn):
-        fn()
-        a, b = _ev(), _ev()
-        torch.cuda.synchronize()
-        a.record()
-        for _ in range(reps):
-            fn()
-        b.record()
-        torch.cuda.synchronize()
-        return a.elapsed_time(b) / reps
+        # device time per call: `reps` calls captured in one CUDA graph (host work stays outside)
+        return time_graph(fn, reps)
 
     out = {"case": args.case, "reps": reps}
     c = args.case
@@ -805,6 +798,15 @@ def run_case(args):
         ms = timed(lambda: dp.dp_ghost_norms(L, B, T, sq))
         out.update(ms=ms, TFLOPs_needed=len(L) * B * T * (T + 1) * 5120 / ms / 1e9,
                    GBs=len(L) * B * 2 * T * 5120 / ms / 1e6)
+    elif c == "ghost256":
+        # T = 256: one diagonal 256 x 256 tile pair per (example, layer), the HBM-bound regime of
+        # the CTA-pair kernel
+        B, T = 64, 256
+        L = [dp.Linear(rb(B, T, 768), rb(B, T, 3072, std=1e-2)) for _ in range(6)]
+        sq = torch.zeros(B, device="cuda")
+        ms = timed(lambda: dp.dp_ghost_norms(L, B, T, sq))
+        out.update(ms=ms, GBs=len(L) * B * 2 * T * 3840 / ms / 1e6,
+                   TFLOPs_needed=len(L) * B * T * (T + 1) * 3840 / ms / 1e9)
     elif c == "noise":
         x = torch.zeros(50257 * 768, device="cuda")
         ms = timed(lambda: dp.dp_add_noise(x, 0.8, 1.0, 1.0, 1234, 0, 0))

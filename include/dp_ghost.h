@@ -28,7 +28,8 @@
  *     the logical width are never read.
  *   - Norm functions ADD into sq; the caller zeroes sq once per step.
  *   - `dev_status` [dev, int32, may be NULL] collects device-side problems by bitwise OR:
- *     DP_DEV_BAD_ID (a token id outside [0,V): that token is skipped) and DP_DEV_TIMEOUT
+ *     DP_DEV_BAD_ID (a token id outside [0,V): that token is skipped), DP_DEV_BOUNDS (checked
+ *     build only: a computed index fell outside its array and the access was skipped) and DP_DEV_TIMEOUT
  *     (a bounded barrier wait gave up: the launch's results are invalid).  The caller
  *     zeroes it and reads it after its own synchronisation.
  *   - Return value: DP_OK or an error found BEFORE anything was enqueued, except
@@ -63,7 +64,7 @@ typedef enum { DP_F32 = 0, DP_BF16 = 1 } dp_dtype;
  * DIRECT iff T*T > d*p, else GHOST. */
 typedef enum { DP_NORM_AUTO = 0, DP_NORM_GHOST = 1, DP_NORM_DIRECT = 2 } dp_norm_mode;
 
-enum { DP_DEV_BAD_ID = 1, DP_DEV_TIMEOUT = 2 };
+enum { DP_DEV_BAD_ID = 1, DP_DEV_TIMEOUT = 2, DP_DEV_BOUNDS = 4 };
 
 /* One linear layer d -> p as seen by the backward pass (Eq. 4: a_i and delta_i). */
 typedef struct {
@@ -160,7 +161,10 @@ size_t dp_tied_cross_term_ws_bytes(int32_t B, int32_t T, int32_t d, int32_t V);
 
 /* ---- clip coefficients (Eq. 2, Eq. 7) ----
  * clip[i] = min(1, C / sqrt(sq[i])), 1 when sq[i] == 0 (no stabiliser is added);
- * norms [dev, B or NULL] receives sqrt(sq[i]).  C > 0 and finite. */
+ * norms [dev, B or NULL] receives sqrt(sq[i]).  C > 0 and finite.
+ * Bad norms fail closed: a squared norm that is NaN or infinite gives clip[i] = 0 (the example
+ * drops out of every clipped sum instead of entering it unclipped); a slightly negative one (the
+ * tied sum in + out + 2 cross can round below zero when the true norm is ~0) counts as 0. */
 dp_status dp_clip_factors(const float* sq, int32_t B, float C, float* clip, float* norms,
                           void* stream);
 /* The same after joining a second accumulator: sq[i] += sq_extra[i] (one addition, fixed order),
@@ -320,6 +324,16 @@ int32_t dp_debug_ghost_single(int32_t on);
  * r^2 <= t_max (t_max <= 0: the threshold in use), max absolute error of cos/sin, largest radius
  * seen, the compiled r^2 threshold}. */
 dp_status dp_debug_noise_error_scan(float t_max, double* out4, void* stream);
+/* The checked build (libdp_ghost_check.so, compiled with -DDP_BOUNDS_CHECK) compares every index
+ * that a kernel computes from data with the extent of the array it addresses, ORs DP_DEV_BOUNDS
+ * into dev_status for an index outside and skips that access: a stand-in for a memory checker.
+ * dp_debug_bounds_checked: 1 in the checked build, 0 otherwise.  dp_debug_bounds_probe: runs the
+ * range test on (idx, n) in a one-thread kernel that touches no memory, so that a test can see an
+ * out-of-range index being reported without any invalid access.  dp_debug_tensor_map_encodes:
+ * TMA tensor maps encoded by the driver so far (maps are cached per tensor and box shape). */
+int32_t dp_debug_bounds_checked(void);
+dp_status dp_debug_bounds_probe(int64_t idx, int64_t n, int32_t* dev_status, void* stream);
+int64_t dp_debug_tensor_map_encodes(void);
 /* Test knob for the failure path: device-side barrier waits give up after `cycles` (0: at the
  * first miss; negative: back to the default of about a second).  A kernel whose wait gives up
  * ORs DP_DEV_TIMEOUT into dev_status, lets its copies and MMAs in flight finish, frees its

@@ -15,7 +15,7 @@ import torch
 
 DP_F32, DP_BF16 = 0, 1
 DP_NORM_AUTO, DP_NORM_GHOST, DP_NORM_DIRECT = 0, 1, 2
-DP_DEV_BAD_ID, DP_DEV_TIMEOUT = 1, 2
+DP_DEV_BAD_ID, DP_DEV_TIMEOUT, DP_DEV_BOUNDS = 1, 2, 4
 
 _LIB_PATH = os.environ.get("DP_GHOST_LIB") or os.path.join(os.path.dirname(os.path.abspath(__file__)),
                                                        "libdp_ghost.so")
@@ -50,7 +50,8 @@ EXPORTS = ["dp_vector_norms", "dp_vector_norms_ws_bytes", "dp_clip_accumulate_ve
            "dp_clip_accumulate_embed_sorted", "dp_add_noise", "dp_add_noise_slice", "dp_noise_step_device",
            "dp_fill_noise", "dp_rdp_epsilon", "dp_sigma_for_epsilon", "dp_status_string",
            "dp_last_cuda_error", "dp_version", "dp_kernel_launches", "dp_debug_force_fma",
-           "dp_debug_noise_error_scan", "dp_debug_set_wait_limit",
+           "dp_debug_noise_error_scan", "dp_debug_bounds_checked", "dp_debug_bounds_probe",
+           "dp_debug_tensor_map_encodes", "dp_debug_set_wait_limit",
            "dp_debug_ghost_single"]
 
 
@@ -125,6 +126,8 @@ def load():
     L.dp_version.restype = C.c_char_p
     L.dp_kernel_launches.restype = C.c_int64
     L.dp_debug_noise_error_scan.argtypes = [f32, vp, vp]
+    L.dp_debug_bounds_probe.argtypes = [i64, i64, vp, vp]
+    L.dp_debug_tensor_map_encodes.restype = i64
     L.dp_debug_set_wait_limit.argtypes = [i64]
     L.dp_debug_set_wait_limit.restype = i64
     L.dp_debug_ghost_single.argtypes = [i32]

@@ -1,6 +1,10 @@
 """Builds csrc/*.cu into libdp_ghost.so (sm_100a only) next to this file.
 
-    python -m paper_2609_40335_b200.build [--force] [--verbose]
+    python -m paper_2609_40335_b200.build [--force] [--verbose] [--check]
+
+--check also builds libdp_ghost_check.so: the same sources with -DDP_BOUNDS_CHECK (every index a
+kernel computes from data is range-checked before the access).  Load it in place of the normal
+library by setting DP_GHOST_LIB to its path.
 
 nvcc cross-compiles without a GPU.  The shared library is kept in-tree so that it travels
 with the source to the machine that has the GPU.
@@ -16,6 +20,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ_DIR = os.path.join(HERE, "build")
 LIB_PATH = os.path.join(HERE, "libdp_ghost.so")
+CHECK_LIB_PATH = os.path.join(HERE, "libdp_ghost_check.so")
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 FLAGS = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC"]
 
@@ -38,17 +43,21 @@ def _stale(target, deps):
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, check: bool = False) -> str:
+    """Compile the library; check=True builds the range-checked variant instead."""
     nvcc = os.environ.get("NVCC", "nvcc")
-    os.makedirs(OBJ_DIR, exist_ok=True)
+    obj_dir = os.path.join(OBJ_DIR, "check") if check else OBJ_DIR
+    lib_path = CHECK_LIB_PATH if check else LIB_PATH
+    extra = ["-DDP_BOUNDS_CHECK"] if check else []
+    os.makedirs(obj_dir, exist_ok=True)
     hdrs = _headers()
     jobs = []
     objs = []
     for src in _sources():
-        obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")
+        obj = os.path.join(obj_dir, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
         if force or _stale(obj, [src] + hdrs):
-            cmd = [nvcc, *ARCH, *FLAGS, "-c", src, "-o", obj]
+            cmd = [nvcc, *ARCH, *FLAGS, *extra, "-c", src, "-o", obj]
             if verbose:
                 cmd.insert(1, "-Xptxas=-v")
             jobs.append(cmd)
@@ -63,14 +72,16 @@ def build(force: bool = False, verbose: bool = False) -> str:
                 sys.stderr.write(" ".join(cmd) + "\n" + r.stdout + r.stderr)
             if r.returncode != 0:
                 raise RuntimeError(f"nvcc failed on {cmd[-3]}")
-    if force or jobs or _stale(LIB_PATH, objs):
-        cmd = [nvcc, *ARCH, "-shared", "-o", LIB_PATH, *objs]
+    if force or jobs or _stale(lib_path, objs):
+        cmd = [nvcc, *ARCH, "-shared", "-o", lib_path, *objs]
         r = subprocess.run(cmd, capture_output=True, text=True)
         if r.returncode != 0:
             sys.stderr.write(r.stdout + r.stderr)
             raise RuntimeError("link failed")
-    return LIB_PATH
+    return lib_path
 
 
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    if "--check" in sys.argv:
+        print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, check=True))

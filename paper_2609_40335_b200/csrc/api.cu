@@ -11,6 +11,7 @@
 #include "fma_kernels.cuh"
 #include "gemm_gta.cuh"
 #include "ghost_plan.cuh"
+#include "tma_host.cuh"
 #include "vector_kernels.cuh"
 
 namespace dpg {
@@ -176,6 +177,12 @@ dp_status dp_debug_noise_error_scan(float t_max, double* out3, void* stream) {
   if (!out3) return DP_ERR_INVALID_ARG;
   return launch_noise_error_scan(t_max, out3, (cudaStream_t)stream);
 }
+int32_t dp_debug_bounds_checked(void) { return kBoundsChecked; }
+dp_status dp_debug_bounds_probe(int64_t idx, int64_t n, int32_t* dev_status, void* stream) {
+  if (!dev_status) return DP_ERR_INVALID_ARG;
+  return launch_bounds_probe(idx, n, dev_status, (cudaStream_t)stream);
+}
+int64_t dp_debug_tensor_map_encodes(void) { return tmap_encode_count(); }
 int32_t dp_debug_force_fma(int32_t on) {
   const int prev = g_force_fma;
   g_force_fma = on ? 1 : 0;
@@ -550,7 +557,7 @@ static dp_status clip_accumulate_embed_impl(const int32_t* ids, const void* G, i
     }
   }
   return launch_embed_scatter(ids, G, ldg, dt, n, T, d, V, clip_ws, sw.perm, sw.seg, out, ldo, beta,
-                              scale, clear, reinterpret_cast<float*>(w + o_part), st);
+                              scale, clear, reinterpret_cast<float*>(w + o_part), st, dev_status);
 }
 
 dp_status dp_clip_accumulate_embed(const int32_t* ids, const void* G, int64_t ldg, dp_dtype dt,

@@ -159,8 +159,14 @@ cross_term_tc_kernel(const __grid_constant__ CrossParams P) {
         const int s0 = tj * kTile + c * 32;
         float wv[32];
 #pragma unroll
-        for (int j = 0; j < 32; ++j)
-          wv[j] = (id >= 0 && s0 + j < P.T) ? __bfloat162float(gcol[size_t(s0 + j) * P.ldgl]) : 0.f;
+        for (int j = 0; j < 32; ++j) {
+          // gathered logit gradient G_lm[ex, s0 + j, id]: the flat element index is computed from
+          // the token id, so the checked build compares it with the tensor's extent
+          const bool take = id >= 0 && s0 + j < P.T &&
+                            dp_in_range((long long)(size_t(ex) * P.T + s0 + j) * P.ldgl + id,
+                                        (long long)P.B * P.T * P.ldgl, P.dev_status);
+          wv[j] = take ? __bfloat162float(gcol[size_t(s0 + j) * P.ldgl]) : 0.f;
+        }
 #pragma unroll
         for (int j = 0; j < 32; ++j) acc = fmaf(__uint_as_float(r[j]), wv[j], acc);
       }
@@ -175,7 +181,7 @@ cross_term_tc_kernel(const __grid_constant__ CrossParams P) {
       if (lane == 0) { epi_red[slot * 4 + ew] = acc; ptx::mbar_arrive(&red_bar[slot]); }
       if (ew == 0) {
         if (!ptx::mbar_wait_relaxed(&red_bar[slot], red_phase, abort_flag, P.wait_limit)) { ok = false; break; }
-        if (lane == 0)
+        if (lane == 0 && dp_in_range(item, P.total_items, P.dev_status))
           P.partials[item] = (epi_red[slot * 4 + 0] + epi_red[slot * 4 + 1]) +
                              (epi_red[slot * 4 + 2] + epi_red[slot * 4 + 3]);
       }

@@ -120,6 +120,25 @@ __device__ __forceinline__ float clip_from_sq(float sq, float C) {
   return nrm > 0.f ? fminf(1.f, __fdiv_rn(C, nrm)) : 1.f;
 }
 
+// ---- checked build ------------------------------------------------------------------------
+// Compiled with -DDP_BOUNDS_CHECK (python -m paper_2609_40335_b200.build --check, which writes
+// libdp_ghost_check.so), every index that a kernel COMPUTES from data -- a gathered column, a
+// sorted position, a rank, a partial-sum slot -- is compared with the extent of the array it
+// addresses before the access; an index outside ORs DP_DEV_BOUNDS into dev_status and the access
+// is skipped.  It stands in for a memory checker on machines where none may be run.  In the
+// normal build the test costs nothing.
+#ifdef DP_BOUNDS_CHECK
+__device__ __forceinline__ bool dp_in_range(long long idx, long long n, int* dev_status) {
+  if (idx >= 0 && idx < n) return true;
+  if (dev_status) atomicOr(dev_status, DP_DEV_BOUNDS);
+  return false;
+}
+constexpr int kBoundsChecked = 1;
+#else
+__device__ __forceinline__ bool dp_in_range(long long, long long, int*) { return true; }
+constexpr int kBoundsChecked = 0;
+#endif
+
 // ---- launchers implemented across the .cu files (all enqueue on `st`, no sync) ----
 // sq[i] += factor * sum_j partials[i*n_per + j] (fixed order); plain_out[i] = that sum if given
 dp_status launch_reduce_partials(const float* partials, int n_per, int B, float* sq,

@@ -94,7 +94,7 @@ embed_norm_kernel(const int* __restrict__ ids, const T* __restrict__ G, long lon
       const int f = s_fo[s];
       rank += (f < fo) || (f == fo && s < t);
     }
-    s_ord[rank] = t;
+    if (dp_in_range(rank, Tn, dev_status)) s_ord[rank] = t;
     if (slab == 0 && first_occ) first_occ[size_t(i) * Tn + t] = fo;
   }
   __syncthreads();
@@ -134,7 +134,7 @@ embed_norm_kernel(const int* __restrict__ ids, const T* __restrict__ G, long lon
         const int r = r0 + b;
         o[b] = r < hi ? s_ord[r] : 0;
         const int t = o[b] & 0x7fffffff;
-        if (r < hi && s_id[t] >= 0) {
+        if (r < hi && dp_in_range(t, Tn, dev_status) && s_id[t] >= 0) {
           load8<T>(Gi + size_t(t) * ldg, nvalid, vec, v[b]);
         } else {
 #pragma unroll
@@ -242,7 +242,7 @@ sort_scan_kernel(int* __restrict__ seg, int V, const int* __restrict__ blk) {
 
 __global__ void __launch_bounds__(kSortChunk)
 sort_place_kernel(const int* __restrict__ ids, int n, int V, const int* __restrict__ counts,
-                  const int* __restrict__ seg, int* __restrict__ perm) {
+                  const int* __restrict__ seg, int* __restrict__ perm, int* __restrict__ dev_status) {
   __shared__ int s_id[kSortChunk];
   const int chunk = blockIdx.x;
   const int j = chunk * kSortChunk + threadIdx.x;
@@ -253,7 +253,8 @@ sort_place_kernel(const int* __restrict__ ids, int n, int V, const int* __restri
   if (id < 0) return;
   int r = 0;
   for (int s = 0; s < (int)threadIdx.x; ++s) r += (s_id[s] == id);
-  perm[seg[id] + counts[size_t(chunk) * V + id] + r] = j;
+  const int dst = seg[id] + counts[size_t(chunk) * V + id] + r;
+  if (dp_in_range(dst, n, dev_status)) perm[dst] = j;
 }
 
 // ------------------------------------------------------------------ segmented row sum
@@ -278,7 +279,8 @@ __global__ void __launch_bounds__(256)
 embed_scatter_kernel(const int* __restrict__ ids, const T* __restrict__ G, long long ldg, int Tn,
                      int d, const float* __restrict__ clip, const int* __restrict__ perm,
                      const int* __restrict__ seg, int V, float* __restrict__ out, long long ldo,
-                     float beta, float scale, float* __restrict__ long_part) {
+                     float beta, float scale, float* __restrict__ long_part, int n_rows,
+                     int* __restrict__ dev_status) {
   __shared__ float part[8][kEmbedColsPerBlock];
   __shared__ int s_pos[kScatChunk + kScatShort];
   __shared__ float s_r[kScatChunk + kScatShort];
@@ -297,10 +299,13 @@ embed_scatter_kernel(const int* __restrict__ ids, const T* __restrict__ G, long 
     const int k = kc + threadIdx.x;
     int s0 = 0;
     if (k < n_valid) {
-      my_v = ids[perm[k]];
-      s0 = seg[my_v];
-      my_n = seg[my_v + 1] - s0;
-      head = (s0 == k);
+      const int pos = perm[k];
+      if (dp_in_range(pos, n_rows, dev_status)) my_v = ids[pos];
+      if (dp_in_range(my_v, V, dev_status)) {
+        s0 = seg[my_v];
+        my_n = seg[my_v + 1] - s0;
+        head = (s0 == k);
+      }
     }
     const bool is_long = my_n > kScatShort;
     const unsigned m = __ballot_sync(0xffffffffu, head);
@@ -311,7 +316,8 @@ embed_scatter_kernel(const int* __restrict__ ids, const T* __restrict__ G, long 
   if (threadIdx.x < kScatChunk + kScatShort) {
     const int k = kc + threadIdx.x;
     if (k < n_valid) {
-      const int pos = perm[k];
+      int pos = perm[k];
+      if (!dp_in_range(pos, n_rows, dev_status)) pos = 0;   // checked build: flagged, row 0 stands in
       s_pos[threadIdx.x] = pos;
       s_r[threadIdx.x] = clip[pos / Tn];
     }
@@ -424,7 +430,8 @@ __global__ void __launch_bounds__(256)
 embed_scatter_combine_kernel(const int* __restrict__ ids, const int* __restrict__ perm,
                              const int* __restrict__ seg, int V, int d,
                              const float* __restrict__ long_part, float* __restrict__ out,
-                             long long ldo, float beta, float scale) {
+                             long long ldo, float beta, float scale, int n_rows,
+                             int* __restrict__ dev_status) {
   __shared__ int s_v, s_k0, s_n;
   const int n_valid = seg[V];
   const int kc = blockIdx.x * kScatChunk;
@@ -434,10 +441,13 @@ embed_scatter_combine_kernel(const int* __restrict__ ids, const int* __restrict_
     int v = -1, n = 0;
     bool long_head = false;
     if (k < n_valid) {
-      v = ids[perm[k]];
-      const int s0 = seg[v];
-      n = seg[v + 1] - s0;
-      long_head = (s0 == k) && (n > kScatShort);
+      const int pos = perm[k];
+      if (dp_in_range(pos, n_rows, dev_status)) v = ids[pos];
+      if (dp_in_range(v, V, dev_status)) {
+        const int s0 = seg[v];
+        n = seg[v + 1] - s0;
+        long_head = (s0 == k) && (n > kScatShort);
+      }
     }
     const unsigned m = __ballot_sync(0xffffffffu, long_head);
     if (threadIdx.x == 0) s_n = 0;
@@ -493,7 +503,18 @@ dp_status launch_embed_sort(const int* ids, int n, int V, const EmbedSortWs& ws,
   DP_LAUNCH_OK();
   sort_scan_kernel<<<ceil_div(V, 1024), 1024, 0, st>>>(ws.seg, V, ws.block_sums);
   DP_LAUNCH_OK();
-  sort_place_kernel<<<ws.chunks, kSortChunk, 0, st>>>(ids, n, V, ws.counts, ws.seg, ws.perm);
+  sort_place_kernel<<<ws.chunks, kSortChunk, 0, st>>>(ids, n, V, ws.counts, ws.seg, ws.perm, dev_status);
+  DP_LAUNCH_OK();
+  return DP_OK;
+}
+
+// Test hook of the checked build: one thread runs the range test on (idx, n) and touches no
+// memory -- shows that an index outside its array is reported (and only in the checked build).
+__global__ void bounds_probe_kernel(long long idx, long long n, int* dev_status) {
+  (void)dp_in_range(idx, n, dev_status);
+}
+dp_status launch_bounds_probe(long long idx, long long n, int* dev_status, cudaStream_t st) {
+  bounds_probe_kernel<<<1, 1, 0, st>>>(idx, n, dev_status);
   DP_LAUNCH_OK();
   return DP_OK;
 }
@@ -505,7 +526,7 @@ size_t embed_scatter_partial_bytes(long long n, int d) {
 dp_status launch_embed_scatter(const int* ids, const void* G, int64_t ldg, dp_dtype dt, int n,
                                int T, int d, int V, const float* clip, const int* perm,
                                const int* seg, float* out, int64_t ldo, float beta, float scale,
-                               bool clear, float* long_part, cudaStream_t st) {
+                               bool clear, float* long_part, cudaStream_t st, int* dev_status) {
   // beta == 0: the table is cleared once (unless the caller already filled it, e.g. with
   // noise), then every touched row receives table + scale*sum
   if (beta == 0.f && clear) {
@@ -515,14 +536,15 @@ dp_status launch_embed_scatter(const int* ids, const void* G, int64_t ldg, dp_dt
   dim3 grid(ceil_div(n, kScatChunk), ceil_div(d, kEmbedColsPerBlock));
   if (dt == DP_F32)
     embed_scatter_kernel<float><<<grid, 256, 0, st>>>(ids, (const float*)G, ldg, T, d, clip, perm,
-                                                     seg, V, out, ldo, 1.f, scale, long_part);
+                                                     seg, V, out, ldo, 1.f, scale, long_part, n,
+                                                     dev_status);
   else
     embed_scatter_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(ids, (const __nv_bfloat16*)G, ldg, T,
                                                              d, clip, perm, seg, V, out, ldo, 1.f,
-                                                             scale, long_part);
+                                                             scale, long_part, n, dev_status);
   DP_LAUNCH_OK();
   embed_scatter_combine_kernel<<<grid, 256, 0, st>>>(ids, perm, seg, V, d, long_part, out, ldo, 1.f,
-                                                     scale);
+                                                     scale, n, dev_status);
   DP_LAUNCH_OK();
   return DP_OK;
 }

@@ -39,7 +39,9 @@ dp_status launch_embed_sort(const int* ids, int n, int V, const EmbedSortWs& ws,
 dp_status launch_embed_scatter(const int* ids, const void* G, int64_t ldg, dp_dtype dt, int n,
                                int T, int d, int V, const float* clip, const int* perm,
                                const int* seg, float* out, int64_t ldo, float beta, float scale,
-                               bool clear, float* long_part, cudaStream_t st);
+                               bool clear, float* long_part, cudaStream_t st,
+                               int* dev_status = nullptr);
+dp_status launch_bounds_probe(long long idx, long long n, int* dev_status, cudaStream_t st);
 // bytes of the per-chunk partial sums of long segments: [chunks][2][d] floats
 size_t embed_scatter_partial_bytes(long long n, int d);
 

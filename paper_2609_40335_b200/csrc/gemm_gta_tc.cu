@@ -391,7 +391,8 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
         if (lane == 0) { epi_red[slot * kEpiWarps + ew] = acc; ptx::mbar_arrive(&red_bar[slot]); }
         if (ew == 0) {
           if (!ptx::mbar_wait_relaxed(&red_bar[slot], red_phase, abort_flag, P.wait_limit)) { ok = false; break; }
-          if (lane == 0) {
+          const long long slot_idx = (long long)it.example * P.n_per + L.col_begin + it.tm * L.tiles_n + it.tn;
+          if (lane == 0 && dp_in_range(slot_idx, (long long)P.B * P.n_per, P.dev_status)) {
             float s = 0.f;
 #pragma unroll
             for (int e = 0; e < kEpiWarps; ++e) s += epi_red[slot * kEpiWarps + e];

@@ -231,7 +231,7 @@ ghost_norm_tc_kernel(const __grid_constant__ GhostParams P) {
       if (lane == 0) { epi_red[slot * 4 + ew] = acc; ptx::mbar_arrive(&red_bar[slot]); }
       if (ew == 0) {
         if (!ptx::mbar_wait_relaxed(&red_bar[slot], red_phase, abort_flag, P.wait_limit)) { ok = false; break; }
-        if (lane == 0) {
+        if (lane == 0 && dp_in_range(it.pidx, (long long)P.B * P.n_per, P.dev_status)) {
           const float s = (epi_red[slot * 4 + 0] + epi_red[slot * 4 + 1]) +
                           (epi_red[slot * 4 + 2] + epi_red[slot * 4 + 3]);
           P.partials[it.pidx] = (it.ti == it.tj) ? s : 2.f * s;

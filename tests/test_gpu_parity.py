@@ -1112,6 +1112,78 @@ def test_cfg5_large_cells_against_library_gemms_on_the_device(B, T):
     assert torch.equal(ds.sq, sq1) and torch.equal(ds.outs["linear2"], out1)
 
 
+def test_tensor_maps_are_encoded_once_per_tensor():
+    """Calls issued one by one (no CUDA graph) reuse the TMA tensor maps of tensors they have seen:
+    the second identical call makes no driver encode at all."""
+    B, T = 2, 128
+    layers = [dev_linear(*host_linear(B, T, 128, 256, "bf16", seed=k)) for k in range(3)]
+    sq = torch.zeros(B, device=dev())
+    outs = [torch.empty(256, 128, device=dev()) for _ in layers]
+    L = dp.load()
+
+    def one_step():
+        dp.dp_ghost_norms(layers, B, T, sq)
+        dp.dp_clip_accumulate_grouped(layers, B, T, sq, 1.0, outs)
+    one_step()
+    n0 = L.dp_debug_tensor_map_encodes()
+    one_step()
+    one_step()
+    torch.cuda.synchronize()
+    assert L.dp_debug_tensor_map_encodes() == n0
+    other = dev_linear(*host_linear(B, T, 128, 256, "bf16", seed=99))
+    dp.dp_ghost_norms([other], B, T, sq)
+    assert L.dp_debug_tensor_map_encodes() == n0 + 2          # a new tensor pair: two new maps
+
+
+def test_bad_squared_norms_fail_closed():
+    """Eq. 7 on corrupted norms: NaN / inf give a factor of 0 (the example leaves the sum, it is
+    never added unclipped); a tiny negative value (rounding of in + out + 2 cross) counts as 0."""
+    sq = torch.tensor([float("nan"), float("inf"), -1e-9, 0.0, 4.0, 0.25, -float("inf")], device=dev())
+    clip, norms = torch.empty_like(sq), torch.empty_like(sq)
+    dp.dp_clip_factors(sq, 1.0, clip=clip, norms=norms)
+    torch.cuda.synchronize()
+    assert clip.cpu().tolist() == [0.0, 0.0, 1.0, 1.0, 0.5, 1.0, 0.0]
+    # and inside a clipped sum: the NaN example contributes nothing
+    B, T, d, p = 3, 64, 64, 128
+    A, G = host_linear(B, T, d, p, "bf16", seed=77)
+    lin = dev_linear(A, G)
+    sq3 = torch.tensor([4.0, float("nan"), 1e-12], device=dev())
+    out = torch.empty(p, d, device=dev())
+    dp.dp_clip_accumulate_grouped([lin], B, T, sq3, 1.0, [out])
+    torch.cuda.synchronize()
+    want = O.clipped_sum_linear(A.widened(), G.widened(), np.array([0.5, 0.0, 1.0]))
+    assert np.isfinite(out.cpu().numpy()).all()
+    assert frob_rel(out.cpu().numpy(), want) < 5e-3
+
+
+def test_fused_noise_on_outputs_that_are_only_4_byte_aligned():
+    """The fused entry points accept any fp32 output tensor: a base that is 4-byte but not 16-byte
+    aligned takes the scalar branch of the noise pass (same values as the aligned call, no fault)."""
+    B, T, d, V = 4, 64, 64, 301
+    ids = torch.from_numpy(W.zipf_ids(B, T, V, 1.1, 3)).to(dev())
+    Ge = P.to_device(W._normal((B, T, d), 1e-2, "bf16", 4))
+    sq = torch.full((B,), 9.0, device=dev())
+    st = torch.zeros(1, dtype=torch.int32, device=dev())
+    aligned = torch.empty(V, d, device=dev())
+    buf = torch.empty(V * d + 8, device=dev())
+    odd = buf[1:1 + V * d].view(V, d)                       # data_ptr() % 16 == 4
+    assert odd.data_ptr() % 16 == 4
+    for out in (aligned, odd):
+        dp.dp_clip_accumulate_embed_noise(ids, Ge, V, sq, 1.0, out, 0.7, 1.0, 5, 2, 9, beta=0.0,
+                                          dev_status=st)
+    # fp32 linear layer with fused noise: the unfused path adds noise with the same kernel
+    A, G = host_linear(B, T, d, 96, "f32", seed=8)
+    lin = dev_linear(A, G)
+    o1 = torch.empty(96, d, device=dev())
+    buf2 = torch.empty(96 * d + 8, device=dev())
+    o2 = buf2[1:1 + 96 * d].view(96, d)
+    for out in (o1, o2):
+        dp.dp_clip_accumulate_noise_grouped([lin], B, T, sq, 1.0, [out], 0.7, 1.0, 5, [3], 9, dev_status=st)
+    torch.cuda.synchronize()
+    check_status(st)
+    assert torch.equal(aligned, odd) and torch.equal(o1, o2)
+
+
 def test_precomputed_clip_factors_and_fused_accumulator_join():
     """sq = None makes `clip` an input of the clip-accumulate calls; dp_clip_factors_sum joins two
     norm accumulators and takes Eq. 7 in one kernel.  Both must equal the plain calls bit for bit."""
