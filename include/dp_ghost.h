@@ -80,7 +80,12 @@ typedef struct {
 
 /* ---- per-example norms of linear layers (Eq. 4 - Eq. 6; LM head = a layer with p = V) ----
  * layers [host, n_layers entries, mode_used written back]; sq [dev, B floats, +=].
- * All layers share B, T and dt.  DP_BF16 runs on tcgen05 tensor cores, DP_F32 on fp32 FMA. */
+ * All layers share B, T and dt.  DP_BF16 runs on tcgen05 tensor cores.  DP_F32 layers with
+ * T >= 32 and d, p >= 64 run there too: every fp32 operand is split into two bf16 terms in the
+ * workspace (x = hi + lo up to 2^-17) and each product is taken as hi*hi' + hi*lo' + lo*hi' with
+ * fp32 accumulation -- about 1e-5 relative, inside the 1e-4 of fp32 inputs; it needs a workspace of
+ * about three times the layer's inputs (dp_ghost_norms_ws_bytes says how much; layers run one after
+ * the other through it).  Smaller fp32 layers run on plain fp32 FMA kernels and need none. */
 dp_status dp_ghost_norms(dp_linear_desc* layers, int32_t n_layers, dp_dtype dt,
                          int32_t B, int32_t T, float* sq,
                          void* ws, size_t ws_bytes, int32_t* dev_status, void* stream);
@@ -180,7 +185,9 @@ dp_status dp_clip_factors_sum(float* sq, const float* sq_extra, int32_t B, float
  * One GEMM with M = p, N = d, K = B*T whose K rows are scaled by R_i = min(1, C/sqrt(sq[i]))
  * on chip.  out [dev, (p,d) fp32, leading dimension ldo] has the layout of a linear layer's
  * weight gradient.  beta is 0 (overwrite) or 1 (accumulate).  clip [dev, B or NULL] receives
- * R.  This replaces the re-weighted second backward pass of ghost clipping by its result. */
+ * R.  This replaces the re-weighted second backward pass of ghost clipping by its result.
+ * DP_F32 layers with T >= 32 and d, p >= 64 take the split-bf16 tensor-core path described at
+ * dp_ghost_norms (R_i multiplies G in fp32 before the split); the workspace grows accordingly. */
 dp_status dp_clip_accumulate(const void* A, int64_t lda, const void* G, int64_t ldg,
                              dp_dtype dt, int32_t B, int32_t T, int32_t d, int32_t p,
                              const float* sq, float C, float* clip,
@@ -311,8 +318,8 @@ const char* dp_version(void);
 /* Number of CUDA kernels this library has enqueued since it was loaded (memsets and copies
  * are not counted).  Lets a caller report how many of its launches a timed region held. */
 int64_t dp_kernel_launches(void);
-/* Test hook: when non-zero, DP_BF16 linear-layer calls run the plain fp32-FMA kernels
- * instead of the tensor-core ones (used to cross-check the two on the device).  Returns
+/* Test hook: when non-zero, linear-layer calls (DP_BF16 and DP_F32 alike) run the plain fp32-FMA
+ * kernels instead of the tensor-core ones (used to cross-check the two on the device).  Returns
  * the previous value.  Off by default; not meant for production use. */
 int32_t dp_debug_force_fma(int32_t on);
 /* Test hook: when non-zero, sequences longer than 128 tokens keep the single-CTA 128 x 128 Gram

@@ -11,6 +11,7 @@
 #include "fma_kernels.cuh"
 #include "gemm_gta.cuh"
 #include "ghost_plan.cuh"
+#include "split_kernels.cuh"
 #include "tma_host.cuh"
 #include "vector_kernels.cuh"
 
@@ -50,9 +51,10 @@ bool first_use_on_this_device(const void* key) {
 }
 
 // ---- planning of dp_ghost_norms ------------------------------------------------------------
-GhostPlan plan_ghost_norms(const dp_linear_desc* layers, int n_layers, int B, int T, int sms) {
+GhostPlan plan_ghost_norms(const dp_linear_desc* layers, int n_layers, int B, int T, int sms,
+                           bool allow_pair) {
   GhostPlan plan;
-  plan.pair = T > 128 && !g_ghost_single;
+  plan.pair = allow_pair && T > 128 && !g_ghost_single;
   const int nt = ceil_div(T, plan.pair ? 256 : 128);
   const int slots = plan.pair ? 2 : 1;           // partial sums per work item
   const int units = plan.pair ? sms / 2 : sms;   // persistent CTAs or CTA pairs
@@ -125,6 +127,83 @@ static dp_status check_linear(const dp_linear_desc& L, dp_dtype dt, bool tc) {
   return DP_OK;
 }
 
+// ---- fp32 inputs on the tensor cores (operands split into two bf16 terms, see split_kernels.cu)
+// Taken for layers that are large enough for a tensor-core tile to pay; tiny layers (and the test
+// hook dp_debug_force_fma) stay on the plain fp32 kernels.
+static bool f32_on_tensor_cores(const dp_linear_desc& L, int T) {
+  return !g_force_fma && T >= 32 && L.d >= 64 && L.p >= 64;
+}
+
+// One layer's widened operands inside a workspace: `a` and `g` (and, column form, their second
+// sides `a2`, `g2`), then whatever the kernels need behind them.
+struct SplitLayer {
+  dp_linear_desc one, other;     // descriptors of the widened bf16 operands
+  size_t bytes;                  // workspace taken by the operands
+};
+
+static SplitLayer split_layout(const dp_linear_desc& L, int B, int T, bool column_form, char* base) {
+  SplitLayer S;
+  memset(&S, 0, sizeof(S));
+  const size_t na = split_bytes((long long)B * T, L.d), ng = split_bytes((long long)B * T, L.p);
+  const int dp_ = split_padded(L.d), pp = split_padded(L.p);
+  S.one.mode = S.other.mode = DP_NORM_GHOST;
+  if (column_form) {             // (B*T, 3*padded) operands, two sides each
+    S.one.A = base; S.one.G = base + na; S.other.A = base + na + ng; S.other.G = base + 2 * na + ng;
+    S.one.d = S.other.d = 3 * dp_; S.one.p = S.other.p = 3 * pp;
+    S.one.lda = S.other.lda = 3 * dp_; S.one.ldg = S.other.ldg = 3 * pp;
+    S.bytes = 2 * (na + ng);
+  } else {                       // (B, 3T, padded) operands
+    S.one.A = base; S.one.G = base + na;
+    S.one.d = L.d; S.one.p = L.p; S.one.lda = dp_; S.one.ldg = pp;
+    S.bytes = na + ng;
+  }
+  return S;
+}
+
+static size_t f32_norm_ws_bytes(const dp_linear_desc& L, int B, int T, int mode, int sms) {
+  const bool direct = mode == DP_NORM_DIRECT;
+  SplitLayer S = split_layout(L, B, T, !direct, nullptr);
+  S.one.mode = mode;
+  const GhostPlan plan = plan_ghost_norms(&S.one, 1, B, direct ? 3 * T : T, sms, false);
+  return S.bytes + align_up(size_t(B) * plan.n_per * sizeof(float), 256);
+}
+
+static int resolve_mode(const dp_linear_desc& L, int T) {
+  if (L.mode != DP_NORM_AUTO) return L.mode;
+  return ((long long)T * T > (long long)L.d * L.p) ? DP_NORM_DIRECT : DP_NORM_GHOST;
+}
+
+// norm of one fp32 layer on the tensor cores; ws holds the widened operands and the partial sums
+static dp_status f32_norm_tc(const dp_linear_desc& L, int B, int T, int mode, float* sq, char* ws,
+                             int* dev_status, cudaStream_t st) {
+  const bool direct = mode == DP_NORM_DIRECT;
+  SplitLayer S = split_layout(L, B, T, !direct, ws);
+  float* partials = reinterpret_cast<float*>(ws + S.bytes);
+  dp_status s;
+  const float* A = static_cast<const float*>(L.A);
+  const float* G = static_cast<const float*>(L.G);
+  if (!direct) {
+    s = launch_split_cols(A, L.lda, (int64_t)B * T, L.d, const_cast<void*>(S.one.A), const_cast<void*>(S.other.A), st);
+    if (s != DP_OK) return s;
+    s = launch_split_cols(G, L.ldg, (int64_t)B * T, L.p, const_cast<void*>(S.one.G), const_cast<void*>(S.other.G), st);
+    if (s != DP_OK) return s;
+    const GhostPlan plan = plan_ghost_norms(&S.one, 1, B, T, sm_count(), false);
+    s = launch_ghost_norm_tc(&S.one, plan, B, T, partials, dev_status, st, &S.other);
+    if (s != DP_OK) return s;
+    return launch_reduce_partials(partials, plan.n_per, B, sq, 1.f, nullptr, st);
+  }
+  // DIRECT: G'^T A' per example over 3T token rows
+  s = launch_split_rows(A, L.lda, B, T, L.d, nullptr, 1, const_cast<void*>(S.one.A), st);
+  if (s != DP_OK) return s;
+  s = launch_split_rows(G, L.ldg, B, T, L.p, nullptr, 2, const_cast<void*>(S.one.G), st);
+  if (s != DP_OK) return s;
+  S.one.mode = DP_NORM_DIRECT;
+  const GhostPlan plan = plan_ghost_norms(&S.one, 1, B, 3 * T, sm_count(), false);
+  s = launch_direct_norm_tc(&S.one, plan, B, 3 * T, partials, dev_status, st);
+  if (s != DP_OK) return s;
+  return launch_reduce_partials(partials, plan.n_per, B, sq, 1.f, nullptr, st);
+}
+
 }  // namespace dpg
 
 using namespace dpg;
@@ -193,7 +272,14 @@ int32_t dp_debug_force_fma(int32_t on) {
 size_t dp_ghost_norms_ws_bytes(const dp_linear_desc* layers, int32_t n_layers, dp_dtype dt,
                                int32_t B, int32_t T) {
   if (!layers || n_layers <= 0 || B <= 0 || T <= 0) return 0;
-  if (dt == DP_F32 || g_force_fma) return 0;
+  if (g_force_fma) return 0;
+  if (dt == DP_F32) {            // layers run one after the other through the same workspace
+    size_t need = 0;
+    for (int l = 0; l < n_layers; ++l)
+      if (f32_on_tensor_cores(layers[l], T))
+        need = std::max(need, f32_norm_ws_bytes(layers[l], B, T, resolve_mode(layers[l], T), sm_count()));
+    return need;
+  }
   const GhostPlan plan = plan_ghost_norms(layers, n_layers, B, T, sm_count());
   return align_up(size_t(B) * plan.n_per * sizeof(float), 256);
 }
@@ -211,8 +297,15 @@ dp_status dp_ghost_norms(dp_linear_desc* layers, int32_t n_layers, dp_dtype dt, 
   }
   const GhostPlan plan = plan_ghost_norms(layers, n_layers, B, T, sm_count());
   if (!tc) {
+    if (dt == DP_F32 && dp_ghost_norms_ws_bytes(layers, n_layers, dt, B, T) > ws_bytes) return DP_ERR_WORKSPACE;
     for (int l = 0; l < n_layers; ++l) {
-      const dp_status s = launch_norms_fma(layers[l], dt, plan.mode_used[l], B, T, sq, st);
+      dp_status s;
+      if (dt == DP_F32 && f32_on_tensor_cores(layers[l], T)) {
+        if (!ws || !aligned16(ws)) return DP_ERR_WORKSPACE;
+        s = f32_norm_tc(layers[l], B, T, plan.mode_used[l], sq, static_cast<char*>(ws), dev_status, st);
+      } else {
+        s = launch_norms_fma(layers[l], dt, plan.mode_used[l], B, T, sq, st);
+      }
       if (s != DP_OK) return s;
       layers[l].mode_used = plan.mode_used[l];
     }
@@ -383,6 +476,15 @@ size_t dp_clip_accumulate_grouped_ws_bytes(const dp_linear_desc* layers, int32_t
   if (!layers || n_layers <= 0 || B <= 0 || T <= 0) return 0;
   size_t n = align_up(size_t(B) * sizeof(float), 256);          // clip factors
   if (dt == DP_BF16 && !g_force_fma) n += gta_partial_bytes(layers, n_layers, B, T, sm_count());
+  if (dt == DP_F32) {            // widened operands of one layer at a time + its K-split planes
+    size_t need = 0;
+    for (int l = 0; l < n_layers; ++l)
+      if (f32_on_tensor_cores(layers[l], T)) {
+        SplitLayer S = split_layout(layers[l], B, T, false, nullptr);
+        need = std::max(need, S.bytes + gta_partial_bytes(&S.one, 1, B, 3 * T, sm_count()));
+      }
+    n += need;
+  }
   return n;
 }
 
@@ -409,7 +511,25 @@ static dp_status clip_accumulate_impl(const dp_linear_desc* layers, int32_t n_la
   dp_status s = resolve_clip(sq, B, C, clip, &clip_ws, st);
   if (s != DP_OK) return s;
   if (!tc) {
+    char* split_ws = static_cast<char*>(ws) + align_up(size_t(B) * sizeof(float), 256);
     for (int l = 0; l < n_layers; ++l) {
+      if (dt == DP_F32 && f32_on_tensor_cores(layers[l], T)) {
+        // R_i multiplies G in fp32 before the split, so the GEMM runs unscaled (clip = NULL)
+        SplitLayer S = split_layout(layers[l], B, T, false, split_ws);
+        s = launch_split_rows(static_cast<const float*>(layers[l].A), layers[l].lda, B, T, layers[l].d,
+                              nullptr, 1, const_cast<void*>(S.one.A), st);
+        if (s != DP_OK) return s;
+        s = launch_split_rows(static_cast<const float*>(layers[l].G), layers[l].ldg, B, T, layers[l].p,
+                              clip_ws, 2, const_cast<void*>(S.one.G), st);
+        if (s != DP_OK) return s;
+        GtaNoise one_noise;
+        if (noise) { one_noise = *noise; one_noise.tensor_ids = noise->tensor_ids + l; }
+        s = launch_clip_accumulate_tc(&S.one, 1, B, 3 * T, nullptr, outs + l, ldos + l, beta,
+                                      noise ? &one_noise : nullptr,
+                                      reinterpret_cast<float*>(split_ws + S.bytes), dev_status, st);
+        if (s != DP_OK) return s;
+        continue;
+      }
       s = launch_clip_accumulate_fma(layers[l].A, layers[l].lda, layers[l].G, layers[l].ldg, dt, B, T,
                                      layers[l].d, layers[l].p, clip_ws, outs[l], ldos[l], beta, st);
       if (s != DP_OK) return s;

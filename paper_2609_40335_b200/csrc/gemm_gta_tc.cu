@@ -298,11 +298,12 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
         // first K step of this item that belongs to this warp
         int ks = it.k0 + int((uint32_t(sw) + kScalerWarps - cnt % kScalerWarps) % kScalerWarps);
         uint32_t c = cnt + uint32_t(ks - it.k0);
-        float r_next = ks < it.k1 ? __ldg(P.clip + ks / P.tsteps) : 1.f;
+        // clip == NULL: the operand is already scaled (the split fp32 path)
+        float r_next = (P.clip && ks < it.k1) ? __ldg(P.clip + ks / P.tsteps) : 1.f;
         for (; ks < it.k1; ks += kScalerWarps, c += kScalerWarps) {
           const float r = r_next;
           // the factor of this warp's next K step is fetched before the waits, off the stage's path
-          if (ks + kScalerWarps < it.k1) r_next = __ldg(P.clip + (ks + kScalerWarps) / P.tsteps);
+          if (P.clip && ks + kScalerWarps < it.k1) r_next = __ldg(P.clip + (ks + kScalerWarps) / P.tsteps);
           const uint32_t stage = c % kStages, fill = c / kStages, phase = fill & 1u;
           // A warp hops between stages, so it has not seen the previous fill of this one, and the
           // parity of `full` alone cannot tell "fill n landed" from "fill n-1 still in flight".

@@ -85,9 +85,14 @@ __device__ __forceinline__ Item decode_item(const GhostParams& P, int item) {
   return it;
 }
 
-template <bool kDiagOnly>
+// kDual: the two sides of each Gram product come from two different tensors (maps 2l and 2l+1 of
+// a layer): the fp32 path, where S = X Y^T with X = [hi | hi | lo] and Y = [hi | lo | hi] of the
+// operand split into two bf16 terms.  S is still symmetric, so tile pairs are enumerated as before,
+// but a diagonal pair also needs both loads.
+template <bool kDiagOnly, bool kDual = false>
 __global__ void __launch_bounds__(kThreads, 1)
 ghost_norm_tc_kernel(const __grid_constant__ GhostParams P) {
+  static_assert(!(kDiagOnly && kDual), "the two-tensor form always loads two tiles per stage");
   constexpr int kStages = GhostGeo<kDiagOnly>::kStages;
   constexpr int kStageBytes = GhostGeo<kDiagOnly>::kStageBytes;
   extern __shared__ uint8_t smem_raw[];
@@ -132,10 +137,12 @@ ghost_norm_tc_kernel(const __grid_constant__ GhostParams P) {
       bool ok = true;
       for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x) {
         const Item it = decode_item(P, item);
-        const bool diag = kDiagOnly || (it.ti == it.tj);
+        const bool diag = !kDual && (kDiagOnly || (it.ti == it.tj));
         const uint32_t bytes = diag ? kTileBytes : kStageBytes;
+        const int li = kDual ? 2 * it.layer : it.layer;
         for (int pass = 0; pass < 2 && ok; ++pass) {
-          const CUtensorMap* tm = pass == 0 ? &P.tmA[it.layer] : &P.tmG[it.layer];
+          const CUtensorMap* tm = pass == 0 ? &P.tmA[li] : &P.tmG[li];
+          const CUtensorMap* tm2 = kDual ? tm + 1 : tm;     // the other side of the product
           const int k0 = pass == 0 ? it.a0 : it.g0, k1 = pass == 0 ? it.a1 : it.g1;
           for (int k = k0; k < k1; ++k) {
             if (!ptx::mbar_wait(&empty[stage], phase ^ 1, abort_flag, P.wait_limit)) { ok = false; break; }
@@ -143,7 +150,7 @@ ghost_norm_tc_kernel(const __grid_constant__ GhostParams P) {
             ptx::mbar_arrive_expect_tx(&full[stage], bytes);
             ptx::tma_load_3d(dst, tm, &full[stage], k * kKStep, it.ti * kTile, it.example);
             if (!diag)
-              ptx::tma_load_3d(dst + kTileBytes, tm, &full[stage], k * kKStep, it.tj * kTile,
+              ptx::tma_load_3d(dst + kTileBytes, tm2, &full[stage], k * kKStep, it.tj * kTile,
                                it.example);
             ++issued;
             if (++stage == kStages) { stage = 0; phase ^= 1; }
@@ -166,7 +173,7 @@ ghost_norm_tc_kernel(const __grid_constant__ GhostParams P) {
       bool ok = true;
       for (int item = blockIdx.x; item < P.total_items && ok; item += gridDim.x, ++n_item) {
         const Item it = decode_item(P, item);
-        const bool diag = kDiagOnly || (it.ti == it.tj);
+        const bool diag = !kDual && (kDiagOnly || (it.ti == it.tj));
         const uint32_t buf = n_item & 1, acc_phase = (n_item >> 1) & 1;
         if (!ptx::mbar_wait(&acc_empty[buf], acc_phase ^ 1, abort_flag, P.wait_limit)) { ok = false; break; }
         ptx::tc_fence_after();
@@ -281,7 +288,8 @@ dp_status launch_reduce_partials(const float* partials, int n_per, int B, float*
 // Enqueue the tensor-core ghost norm for the planned layers; partial sums land in
 // plan.partials layout inside `partials` (the caller reduces them afterwards).
 dp_status launch_ghost_norm_tc(const dp_linear_desc* layers, const GhostPlan& plan, int B, int T,
-                               float* partials, int* dev_status, cudaStream_t st) {
+                               float* partials, int* dev_status, cudaStream_t st,
+                               const dp_linear_desc* other_side) {
   if (first_use_on_this_device(reinterpret_cast<const void*>(&launch_ghost_norm_tc))) {
     DP_CUDA_OK(cudaFuncSetAttribute(ghost_norm_tc_kernel<true>,
                                     cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -289,21 +297,34 @@ dp_status launch_ghost_norm_tc(const dp_linear_desc* layers, const GhostPlan& pl
     DP_CUDA_OK(cudaFuncSetAttribute(ghost_norm_tc_kernel<false>,
                                     cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)GhostGeo<false>::kSmemBytes));
+    DP_CUDA_OK(cudaFuncSetAttribute(ghost_norm_tc_kernel<false, true>,
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)GhostGeo<false>::kSmemBytes));
   }
+  const bool dual = other_side != nullptr;
+  const size_t per_launch = dual ? kGhostMaxLayers / 2 : kGhostMaxLayers;
   const int nt = ceil_div(T, kTile);
   // layers are processed in groups that fit one parameter block
-  for (size_t g0 = 0; g0 < plan.ghost_layers.size(); g0 += kGhostMaxLayers) {
-    const size_t g1 = std::min(plan.ghost_layers.size(), g0 + kGhostMaxLayers);
+  for (size_t g0 = 0; g0 < plan.ghost_layers.size(); g0 += per_launch) {
+    const size_t g1 = std::min(plan.ghost_layers.size(), g0 + per_launch);
     GhostParams P;
     memset(&P, 0, sizeof(P));
     int items = 0;
     for (size_t g = g0; g < g1; ++g) {
       const int li = plan.ghost_layers[g];
       const dp_linear_desc& L = layers[li];
-      dp_status s = make_tmap_bf16_3d(&P.tmA[g - g0], L.A, L.lda, L.d, T, B, kKStep, kTile);
+      const size_t slot = dual ? 2 * (g - g0) : (g - g0);
+      dp_status s = make_tmap_bf16_3d(&P.tmA[slot], L.A, L.lda, L.d, T, B, kKStep, kTile);
       if (s != DP_OK) return s;
-      s = make_tmap_bf16_3d(&P.tmG[g - g0], L.G, L.ldg, L.p, T, B, kKStep, kTile);
+      s = make_tmap_bf16_3d(&P.tmG[slot], L.G, L.ldg, L.p, T, B, kKStep, kTile);
       if (s != DP_OK) return s;
+      if (dual) {
+        const dp_linear_desc& R = other_side[li];
+        s = make_tmap_bf16_3d(&P.tmA[slot + 1], R.A, R.lda, R.d, T, B, kKStep, kTile);
+        if (s != DP_OK) return s;
+        s = make_tmap_bf16_3d(&P.tmG[slot + 1], R.G, R.ldg, R.p, T, B, kKStep, kTile);
+        if (s != DP_OK) return s;
+      }
       GhostLayerPlan lp = plan.layer[li];
       lp.item_begin = items;
       items += B * plan.ntp * lp.nsplit;
@@ -317,7 +338,9 @@ dp_status launch_ghost_norm_tc(const dp_linear_desc* layers, const GhostPlan& pl
     P.dev_status = dev_status;
     P.wait_limit = g_wait_limit;
     const int grid = std::min(items, sm_count());
-    if (nt == 1)
+    if (dual)
+      ghost_norm_tc_kernel<false, true><<<grid, kThreads, GhostGeo<false>::kSmemBytes, st>>>(P);
+    else if (nt == 1)
       ghost_norm_tc_kernel<true><<<grid, kThreads, GhostGeo<true>::kSmemBytes, st>>>(P);
     else
       ghost_norm_tc_kernel<false><<<grid, kThreads, GhostGeo<false>::kSmemBytes, st>>>(P);

@@ -38,12 +38,17 @@ struct GhostPlan {
 };
 
 // T*T > d*p selects DIRECT under AUTO (strict), otherwise GHOST.
-GhostPlan plan_ghost_norms(const dp_linear_desc* layers, int n_layers, int B, int T, int sms);
+// allow_pair = false keeps the single-CTA Gram kernel whatever T is.
+GhostPlan plan_ghost_norms(const dp_linear_desc* layers, int n_layers, int B, int T, int sms,
+                           bool allow_pair = true);
 
 dp_status launch_ghost_norm_pair(const dp_linear_desc* layers, const GhostPlan& plan, int B, int T,
                                  float* partials, int* dev_status, cudaStream_t st);
 
+// other_side != NULL: the second operand of every Gram product is taken from other_side[l] (same
+// shapes as layers[l]) instead of layers[l] itself (the split fp32 path).
 dp_status launch_ghost_norm_tc(const dp_linear_desc* layers, const GhostPlan& plan, int B, int T,
-                               float* partials, int* dev_status, cudaStream_t st);
+                               float* partials, int* dev_status, cudaStream_t st,
+                               const dp_linear_desc* other_side = nullptr);
 
 }  // namespace dpg

@@ -1112,6 +1112,66 @@ def test_cfg5_large_cells_against_library_gemms_on_the_device(B, T):
     assert torch.equal(ds.sq, sq1) and torch.equal(ds.outs["linear2"], out1)
 
 
+F32_TC_CASES = [(8, 128, 768, 3072), (3, 100, 72, 136), (2, 200, 192, 320), (2, 64, 3072, 768)]
+
+
+@pytest.mark.parametrize("B,T,d,p", F32_TC_CASES)
+@pytest.mark.parametrize("mode", [dp.DP_NORM_GHOST, dp.DP_NORM_DIRECT])
+def test_fp32_inputs_on_tensor_cores_norms(B, T, d, p, mode):
+    """DP_F32 layers that are large enough run on the bf16 tensor cores with every operand split
+    into two bf16 terms (three products per product).  Norms against the oracle at the fp32
+    tolerance 1e-4, and against the plain fp32 FMA kernels (the cross-check path)."""
+    A, G = host_linear(B, T, d, p, "f32", seed=17 * T + d + p)
+    lin = dev_linear(A, G, mode)
+    st = torch.zeros(1, dtype=torch.int32, device=dev())
+    sq = torch.zeros(B, device=dev())
+    assert dp.dp_ghost_norms_ws_bytes([lin], B, T) > 0                 # the split path is the one taken
+    used = dp.dp_ghost_norms([lin], B, T, sq, dev_status=st)
+    torch.cuda.synchronize()
+    check_status(st)
+    assert used == [mode]
+    want = O.linear_sq_norms(A.widened(), G.widened())
+    assert rel(sq.cpu().numpy(), want).max() < TOL_F32
+    assert rel(sq.cpu().numpy(), want).max() < 2e-5                    # what two bf16 terms give
+    prev = dp.dp_debug_force_fma(1)
+    try:
+        sq_fma = torch.zeros(B, device=dev())
+        dp.dp_ghost_norms([lin], B, T, sq_fma, dev_status=st)
+        torch.cuda.synchronize()
+    finally:
+        dp.dp_debug_force_fma(prev)
+    assert rel(sq.cpu().numpy(), sq_fma.cpu().numpy()).max() < 5e-5
+
+
+@pytest.mark.parametrize("B,T,d,p", F32_TC_CASES)
+@pytest.mark.parametrize("beta", [0.0, 1.0])
+def test_fp32_inputs_on_tensor_cores_clipped_sums(B, T, d, p, beta):
+    """Clipped sum of a DP_F32 layer on the tensor cores: R_i multiplies G in fp32 before the split,
+    so the result keeps fp32-class accuracy (1e-4 Frobenius asserted; bf16 inputs get 5e-3)."""
+    A, G = host_linear(B, T, d, p, "f32", seed=5 * T + d + p)
+    lin = dev_linear(A, G)
+    rng = np.random.default_rng(B + T)
+    sq = torch.from_numpy(rng.uniform(0.25, 9.0, B).astype(np.float32)).to(dev())   # both branches of min
+    Cc = 1.5
+    _, R = O.clip_factors(sq.cpu().numpy().astype(np.float64), Cc)
+    st = torch.zeros(1, dtype=torch.int32, device=dev())
+    init = torch.from_numpy(rng.standard_normal((p, d)).astype(np.float32)).to(dev())
+    out = init.clone()
+    dp.dp_clip_accumulate_grouped([lin], B, T, sq, Cc, [out], beta=beta, dev_status=st)
+    torch.cuda.synchronize()
+    check_status(st)
+    want = O.clipped_sum_linear(A.widened(), G.widened(), R) + beta * init.cpu().numpy().astype(np.float64)
+    assert frob_rel(out.cpu().numpy(), want) < 1e-4
+    # fused noise equals clipped sum + stand-alone noise, bit for bit
+    a, b = init.clone(), init.clone()
+    dp.dp_clip_accumulate_noise_grouped([lin], B, T, sq, Cc, [a], 0.7, 1.0, 5, [3], 9, beta=beta, dev_status=st)
+    dp.dp_clip_accumulate_grouped([lin], B, T, sq, Cc, [b], beta=beta, dev_status=st)
+    dp.dp_add_noise(b, 0.7, Cc, 1.0, 5, 3, 9)
+    torch.cuda.synchronize()
+    check_status(st)
+    assert torch.equal(a, b)
+
+
 def test_tensor_maps_are_encoded_once_per_tensor():
     """Calls issued one by one (no CUDA graph) reuse the TMA tensor maps of tensors they have seen:
     the second identical call makes no driver encode at all."""
