@@ -66,7 +66,15 @@ def test_workspace_sizes_follow_the_plan(lib):
     n = lib.dp_ghost_norms_ws_bytes(d, 2, 1, B, T)
     # one partial per (example, layer, column chunk): the head is split into several chunks
     assert n >= B * (1 + 8) * 4 and n % 256 == 0
-    assert lib.dp_ghost_norms_ws_bytes(d, 2, 0, B, T) == 0          # fp32 path needs none
+    # fp32 layers of this size run on the tensor cores with their operands split into two bf16
+    # terms: the widened operands of the LARGEST layer (two sides, three column blocks, 2 bytes)
+    # plus its partial sums; layers too small for a tensor-core tile need nothing
+    f32 = lib.dp_ghost_norms_ws_bytes(d, 2, 0, B, T)
+    widened = 2 * 3 * B * T * (768 + 50264) * 2
+    assert widened <= f32 <= widened + (1 << 20) and f32 % 256 == 0
+    tiny = (_LinearDesc * 1)()
+    tiny[0].A, tiny[0].G, tiny[0].d, tiny[0].p, tiny[0].lda, tiny[0].ldg, tiny[0].mode = 4096, 8192, 64, 64, 64, 64, 0
+    assert lib.dp_ghost_norms_ws_bytes(tiny, 1, 0, 4, 16) == 0
     # few output tiles -> K is split and partial planes are needed; many tiles -> only clip factors
     small = lib.dp_clip_accumulate_ws_bytes(1, B, T, 768, 768)
     big = lib.dp_clip_accumulate_ws_bytes(1, B, T, 768, 50257)
