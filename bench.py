@@ -591,6 +591,11 @@ def run_ours(args):
                 "peak_source": "%s %s bf16 peak: %s" % (peaks["source"], peak_kind, peak_why),
                 "frac_of_burst_peak": achieved_tf / peaks["bf16_tflops"],
                 "frac_of_sustained_peak": achieved_tf / peaks["bf16_tflops_sustained"],
+                # the burst peak scaled to the SM clock sampled during this timed region: what the
+                # same tensor cores deliver at the clock the power cap left them
+                "frac_of_burst_peak_at_sampled_clock": (
+                    achieved_tf / (peaks["bf16_tflops"] * clocks["sm_mhz"] / clocks["sm_max_mhz"])
+                    if clocks and clocks.get("sm_mhz") and clocks.get("sm_max_mhz") else None),
                 "launches_per_step": 1 if exchange is None else 4, "ms_per_launch_avg": gemm_ms_avg,
                 "timed_bracket": ("the grouped GEMM call" if exchange is None else
                                   "the whole clip phase (four GEMM launches, scatters, vectors): N > 1"),
@@ -766,17 +771,19 @@ def run_case(args):
 
     out = {"case": args.case, "reps": reps}
     c = args.case
-    if c in ("gemm", "gemm_unclipped", "gemm_noise"):
-        # one layer 768 -> 18944 at B=32, T=128: 74 x 3 output tiles of 256 x 256, three waves
-        B, T = 32, 128
-        L = [dp.Linear(rb(B, T, 768), rb(B, T, 148 * 128, std=1e-2))]
-        outs = [torch.empty(148 * 128, 768, device="cuda")]
+    if c in ("gemm", "gemm_unclipped", "gemm_noise", "gemm_head"):
+        # three full waves of 256 x 256 output tiles on 74 CTA pairs.  gemm*: a block-like layer
+        # 1536 -> 9472 at B=64, T=128 (clip factors applied inside the pipeline); gemm_head: a
+        # head-like layer 768 -> 18944 at B=32 (its narrow operand is scaled in a pass of its own)
+        B, T, d_, p_ = (32, 128, 768, 148 * 128) if c == "gemm_head" else (64, 128, 1536, 37 * 256)
+        L = [dp.Linear(rb(B, T, d_), rb(B, T, p_, std=1e-2))]
+        outs = [torch.empty(p_, d_, device="cuda")]
         sq = torch.full((B,), 1e-12 if c == "gemm_unclipped" else 4.0, device="cuda")
         if c == "gemm_noise":
             ms = timed(lambda: dp.dp_clip_accumulate_noise_grouped(L, B, T, sq, 1.0, outs, 0.8, 1.0, 0, [0], 0))
         else:
             ms = timed(lambda: dp.dp_clip_accumulate_grouped(L, B, T, sq, 1.0, outs))
-        out.update(ms=ms, TFLOPs=2 * B * T * 768 * 148 * 128 / ms / 1e9)
+        out.update(ms=ms, TFLOPs=2 * B * T * d_ * p_ / ms / 1e9)
     elif c == "direct":
         # DIRECT norm (gradient tiles in tensor memory, square-sum epilogue): 768 -> 3072, T = 256
         B, T = 64, 256

@@ -21,6 +21,7 @@ struct GtaLayer {
   int item_begin;
   int col_begin;          // square-sum mode: first partial-sum column of this layer
   float beta;
+  int prescaled;          // 1: the clip factors were applied to this layer's narrow operand beforehand
   float noise_amp;        // sigma*C of the fused noise, negative = none
   uint32_t tensor_id;     // noise stream id of this output tensor
 };
@@ -34,6 +35,8 @@ struct GtaNoise {
 };
 
 int gta_choose_nsplit(const dp_linear_desc* layers, int n_layers, int B, int T, int sms);
+// scratch of a grouped call behind the clip factors: K-split planes (if any) and the pre-scaled
+// copies of very narrow operands
 size_t gta_partial_bytes(const dp_linear_desc* layers, int n_layers, int B, int T, int sms);
 
 // One persistent launch over the output tiles of all layers (plus split-K reduces if needed).

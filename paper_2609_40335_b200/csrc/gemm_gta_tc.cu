@@ -295,15 +295,17 @@ gemm_gta_kernel(const __grid_constant__ GtaParams P) {
       bool ok = true;
       for (int item = first_item; item < P.total_items && ok; item += item_stride) {
         const Item it = decode_item<kSqsum>(P, item);
+        const bool scale_here = P.clip && !P.layer[it.layer].prescaled;
         // first K step of this item that belongs to this warp
         int ks = it.k0 + int((uint32_t(sw) + kScalerWarps - cnt % kScalerWarps) % kScalerWarps);
         uint32_t c = cnt + uint32_t(ks - it.k0);
-        // clip == NULL: the operand is already scaled (the split fp32 path)
-        float r_next = (P.clip && ks < it.k1) ? __ldg(P.clip + ks / P.tsteps) : 1.f;
+        // no scaling here when the operand arrives scaled: clip == NULL (the split fp32 path) or a
+        // layer whose narrow operand was multiplied by R_i in a pass of its own (see prescale)
+        float r_next = (scale_here && ks < it.k1) ? __ldg(P.clip + ks / P.tsteps) : 1.f;
         for (; ks < it.k1; ks += kScalerWarps, c += kScalerWarps) {
           const float r = r_next;
           // the factor of this warp's next K step is fetched before the waits, off the stage's path
-          if (P.clip && ks + kScalerWarps < it.k1) r_next = __ldg(P.clip + (ks + kScalerWarps) / P.tsteps);
+          if (scale_here && ks + kScalerWarps < it.k1) r_next = __ldg(P.clip + (ks + kScalerWarps) / P.tsteps);
           const uint32_t stage = c % kStages, fill = c / kStages, phase = fill & 1u;
           // A warp hops between stages, so it has not seen the previous fill of this one, and the
           // parity of `full` alone cannot tell "fill n landed" from "fill n-1 still in flight".
@@ -519,6 +521,40 @@ __global__ void splitk_reduce_kernel(const float* __restrict__ partial, int nspl
   }
 }
 
+// out[r, :] = bf16(R_{r / T} * src[r, :]) for the B*T token rows of a narrow operand
+__global__ void __launch_bounds__(256)
+prescale_rows_kernel(const __nv_bfloat16* __restrict__ src, long long lds, __nv_bfloat16* __restrict__ dst,
+                     int cp, long long rows, int T, int c, const float* __restrict__ clip) {
+  const int per_row = cp >> 3;                      // 16-byte chunks per output row
+  const long long total = rows * per_row;
+  const bool vec = ((reinterpret_cast<uintptr_t>(src) & 15) == 0) && ((lds & 7) == 0);
+  for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total;
+       e += (long long)gridDim.x * blockDim.x) {
+    const long long r = e / per_row;
+    const int c0 = int(e - r * per_row) << 3;
+    float v[8];
+    load8<__nv_bfloat16>(src + r * lds + c0, c - c0, vec, v);   // columns >= c read as zero
+    const float f = clip[r / T];
+    uint4 o;
+    __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) o2[k] = __floats2bfloat162_rn(v[2 * k] * f, v[2 * k + 1] * f);
+    *reinterpret_cast<uint4*>(dst + r * cp + c0) = o;
+  }
+}
+
+// A layer whose narrow operand is at most a twentieth of its input bytes (the LM head: d = 768
+// against p = 50257) gets that operand multiplied by R_i in a pass of its own -- a few
+// microseconds -- and then runs through the GEMM unscaled: the in-pipeline scaling costs
+// shared-memory bandwidth on EVERY K step of every tile of the wide operand, the copy does not.
+inline bool prescale_layer(const dp_linear_desc& L) {
+  return 20LL * std::min(L.d, L.p) <= (long long)L.d + L.p;
+}
+inline size_t prescale_bytes(const dp_linear_desc& L, int B, int T) {
+  const int cp = (std::min(L.d, L.p) + 7) / 8 * 8;
+  return align_up(size_t(B) * T * cp * 2, 256);
+}
+
 // The clipped sum always runs with kScale = true: on CTA pairs the scaler warps are also what
 // tells rank 0's MMA issuer that BOTH CTAs' halves of a stage have landed.  (kScale = false is
 // for the single-CTA DIRECT-norm kernel only; a pair kernel without the scalers' hand-off would
@@ -574,10 +610,11 @@ int gta_choose_nsplit(const dp_linear_desc* layers, int n_layers, int B, int T, 
 
 size_t gta_partial_bytes(const dp_linear_desc* layers, int n_layers, int B, int T, int sms) {
   const int ns = gta_choose_nsplit(layers, n_layers, B, T, sms);
-  if (ns <= 1) return 0;
   size_t n = 0;
-  for (int l = 0; l < n_layers; ++l)
-    n += align_up(size_t(ns) * size_t(layers[l].p) * size_t(layers[l].d) * sizeof(float), 256);
+  for (int l = 0; l < n_layers; ++l) {
+    if (ns > 1) n += align_up(size_t(ns) * size_t(layers[l].p) * size_t(layers[l].d) * sizeof(float), 256);
+    if (prescale_layer(layers[l])) n += prescale_bytes(layers[l], B, T);
+  }
   return n;
 }
 
@@ -594,18 +631,38 @@ dp_status launch_clip_accumulate_tc(const dp_linear_desc* layers, int n_layers, 
   const int kps = ceil_div(ksteps, nsplit);
   nsplit = ceil_div(ksteps, kps);                       // drop empty trailing splits
   char* pw = reinterpret_cast<char*>(partial_ws);
+  char* pre = pw;                                       // pre-scaled copies sit behind the K-split planes
+  if (pw && nsplit > 1)
+    for (int l = 0; l < n_layers; ++l)
+      pre += align_up(size_t(nsplit) * size_t(layers[l].p) * size_t(layers[l].d) * sizeof(float), 256);
   for (int g0 = 0; g0 < n_layers; g0 += kGtaMaxLayers) {
     const int g1 = std::min(n_layers, g0 + kGtaMaxLayers);
     GtaParams P;
     memset(&P, 0, sizeof(P));
     int items = 0;
     for (int g = g0; g < g1; ++g) {
-      const dp_linear_desc& D = layers[g];
+      dp_linear_desc D = layers[g];
+      GtaLayer& L = P.layer[g - g0];
+      L.prescaled = 0;
+      if (clip && pw && prescale_layer(D)) {
+        // R_i onto the narrow operand, into the workspace; the GEMM then reads the copy
+        const bool narrow_a = D.d <= D.p;
+        const int c = narrow_a ? D.d : D.p, cp = (c + 7) / 8 * 8;
+        __nv_bfloat16* copy = reinterpret_cast<__nv_bfloat16*>(pre);
+        pre += prescale_bytes(D, B, T);
+        const long long rows = (long long)B * T;
+        const int blocks = (int)std::min<long long>((rows * (cp >> 3) + 255) / 256, (long long)sms * 16);
+        prescale_rows_kernel<<<blocks, 256, 0, st>>>(
+            static_cast<const __nv_bfloat16*>(narrow_a ? D.A : D.G), narrow_a ? D.lda : D.ldg, copy, cp,
+            rows, T, c, clip);
+        DP_LAUNCH_OK();
+        if (narrow_a) { D.A = copy; D.lda = cp; } else { D.G = copy; D.ldg = cp; }
+        L.prescaled = 1;
+      }
       s = make_tmap_bf16_3d(&P.tmG[g - g0], D.G, D.ldg, D.p, T, B, 64, kBK);
       if (s != DP_OK) return s;
       s = make_tmap_bf16_3d(&P.tmA[g - g0], D.A, D.lda, D.d, T, B, 64, kBK);
       if (s != DP_OK) return s;
-      GtaLayer& L = P.layer[g - g0];
       L.out = outs[g]; L.ldo = ldos[g]; L.beta = beta;
       L.M = D.p; L.N = D.d;
       L.tiles_m = ceil_div(D.p, Geo<kUsePair>::kTileM); L.tiles_n = ceil_div(D.d, kBN);
