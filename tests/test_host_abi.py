@@ -75,8 +75,10 @@ def test_workspace_sizes_follow_the_plan(lib):
     tiny = (_LinearDesc * 1)()
     tiny[0].A, tiny[0].G, tiny[0].d, tiny[0].p, tiny[0].lda, tiny[0].ldg, tiny[0].mode = 4096, 8192, 64, 64, 64, 64, 0
     assert lib.dp_ghost_norms_ws_bytes(tiny, 1, 0, 4, 16) == 0
-    # few output tiles -> K is split and partial planes are needed; many tiles -> only clip factors
+    # few output tiles -> K is split and partial planes are needed; many tiles -> the clip factors
+    # and, for a layer as lopsided as the LM head, the pre-scaled bf16 copy of its narrow operand
     small = lib.dp_clip_accumulate_ws_bytes(1, B, T, 768, 768)
     big = lib.dp_clip_accumulate_ws_bytes(1, B, T, 768, 50257)
-    assert small > 768 * 768 * 4 and big == 256
+    mid = lib.dp_clip_accumulate_ws_bytes(1, 64, 256, 768, 3072)
+    assert small > 768 * 768 * 4 and big == 256 + B * T * 768 * 2 and mid == 256
     assert lib.dp_clip_accumulate_embed_ws_bytes(B, T, 768, 50257) >= (4 * 50257 + 50258 + B * T) * 4
