@@ -79,6 +79,6 @@ def test_workspace_sizes_follow_the_plan(lib):
     # and, for a layer as lopsided as the LM head, the pre-scaled bf16 copy of its narrow operand
     small = lib.dp_clip_accumulate_ws_bytes(1, B, T, 768, 768)
     big = lib.dp_clip_accumulate_ws_bytes(1, B, T, 768, 50257)
-    mid = lib.dp_clip_accumulate_ws_bytes(1, 64, 256, 768, 3072)
+    mid = lib.dp_clip_accumulate_ws_bytes(1, 64, 256, 3072, 4096)      # many tiles, balanced widths
     assert small > 768 * 768 * 4 and big == 256 + B * T * 768 * 2 and mid == 256
     assert lib.dp_clip_accumulate_embed_ws_bytes(B, T, 768, 50257) >= (4 * 50257 + 50258 + B * T) * 4
