@@ -310,9 +310,13 @@ def measure_cell(P, dp, name, B, T, d_model, n_blocks, tied, positions, sigma, p
     dev = torch.cuda.current_device()
     torch.cuda.synchronize()
     torch.cuda.empty_cache()
-    torch.cuda.reset_peak_memory_stats(dev)
     ds = P.synthesize_on_device(name, B, T, d_model, n_blocks, tied=tied, positions=positions,
                                 sigma=sigma, seed=seed)
+    # footprint of the step itself: resident inputs + outputs + workspaces (the staging buffers of
+    # the input synthesis are gone by now)
+    torch.cuda.synchronize()
+    torch.cuda.empty_cache()
+    torch.cuda.reset_peak_memory_stats(dev)
     counts = work_counts(shape_of(ds, name))
     sg = P.StepGraph(ds, seed=seed, first_step=0)
     for _ in range(warmup):
@@ -583,8 +587,10 @@ def run_ours(args):
     # dominant kernel: the tensor-core G^T A GEMM of the clipped sums, timed live (see above)
     achieved_tf = counts["acc_flops"] / (gemm_ms_avg * 1e-3) / 1e12
     roofline = {"kernel": "gemm_gta_kernel<scale, pair> (%s)" % (
-                    "dp_clip_accumulate_noise_grouped, Gaussian noise drawn in the epilogue" if fused
-                    else "dp_clip_accumulate_grouped"),
+                    "dp_clip_accumulate_noise_grouped, Gaussian noise drawn in the epilogue"
+                    if fused and not args.prefill else
+                    "dp_clip_accumulate_grouped, accumulating onto noise filled beside the norm phase"
+                    if fused else "dp_clip_accumulate_grouped"),
                 "bound": "tensor",
                 "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
                 "frac": achieved_tf / peak_tf,
