@@ -467,9 +467,9 @@ def run_ours(args):
     counts = work_counts(w)
     stream = torch.cuda.current_stream()
 
-    fused = (world == 1) and not args.unfused     # noise inside the clipped-sum kernels
+    fused = (world == 1) and not args.unfused and not args.bucketed     # noise inside the clipped-sum kernels
     exchange = None
-    if world > 1 and args.exchange == "reduce_scatter":
+    if (world > 1 or args.bucketed) and args.exchange == "reduce_scatter":
         # bucketed reduce-scatter on a communication stream; each rank noises the slices it owns
         step_box = [0]
         exchange = parallel.BucketedExchange(
@@ -874,6 +874,9 @@ def main():
                          "slice (default), or a blocking all-reduce per tensor followed by the noise pass")
     ap.add_argument("--gather", action="store_true",
                     help="N > 1, reduce_scatter: all-gather the noised slices back into the full tensors")
+    ap.add_argument("--bucketed", action="store_true",
+                    help="N = 1: run the multi-GPU step order (clipped sums bucket by bucket through the "
+                         "exchange object, noise on the communication stream) on one GPU")
     ap.add_argument("--eager", action="store_true",
                     help="issue the step call by call instead of replaying a captured CUDA graph")
     ap.add_argument("--workload", default="cfg3")
