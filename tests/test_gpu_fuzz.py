@@ -1,5 +1,6 @@
 """Seeded random-shape parity: the linear-layer norms and clipped sums (single and grouped calls),
-the embedding norm / sort / scatter and the tied cross term on shapes drawn at random -- ragged T,
+the embedding norm / sort / scatter, the tied cross term, the noise stream (stand-alone slices and
+fused into the clipped sums) and the bias / LayerNorm parameters on shapes drawn at random -- ragged T,
 d, p and V, padded leading dimensions (the padding holds NaN), every norm mode, both input types --
 each compared with the oracle.  The fixed cases of test_gpu_parity.py pin the shapes of the
 workloads; this file looks for the shape nobody thought of."""
@@ -8,6 +9,7 @@ import pytest
 import torch
 
 from oracle import dp_oracle as O
+from oracle import noise_oracle as NO
 from paper_2609_40335_b200 import binding as dp
 from paper_2609_40335_b200 import pipeline as P
 from paper_2609_40335_b200 import workloads as W
@@ -272,9 +274,122 @@ def grouped_case(rng, k):
             bad.append(f"sum err {d}x{p} {fe:.3e}")
     return desc, bad
 
+def noise_case(rng, k):
+    """stand-alone noise on a slice that starts anywhere on a counter boundary (the counter's high
+    word included), with random keys; a buffer that is not 16-byte aligned is refused"""
+    n = pick(rng, [1, 2, 3, 4, 5, 7, 8, 31, 100, 1023, 4096, 10007, 65537, 300001])
+    first = 4 * int(rng.integers(0, 1 << 20)) * pick(rng, [0, 1, 1, 4097])
+    seed = int(rng.integers(0, 1 << 63)) * 2 + int(rng.integers(2))
+    tid, step = int(rng.integers(0, 1 << 32)), int(rng.integers(0, 1 << 31))
+    sigma, C_, scale = float(rng.uniform(0.1, 2.0)), float(rng.uniform(0.1, 3.0)), pick(rng, [1.0, 0.5, 1.0 / 64])
+    off = pick(rng, [0, 0, 4, 1, 2, 3])
+    buf = torch.randn(n + 8, device=_dev())
+    part = buf[off:off + n]
+    base = part.clone()
+    desc = f"#{k} noise n{n} first{first} off{off} tid{tid} step{step}"
+    bad = []
+    if off % 4:
+        try:
+            dp.dp_add_noise_slice(part, first, sigma, C_, scale, seed, tid, step)
+            bad.append("misaligned buffer accepted")
+        except dp.DpGhostError as e:
+            if e.status != 3:
+                bad.append(f"misaligned buffer: status {e.status}")
+        if not torch.equal(part, base):
+            bad.append("refused call wrote")
+        return desc, bad
+    dp.dp_add_noise_slice(part, first, sigma, C_, scale, seed, tid, step)
+    torch.cuda.synchronize()
+    z = NO.standard_normals(n, seed, tid, step, start=first)
+    want = scale * (base.cpu().numpy().astype(np.float64) + sigma * C_ * z)
+    e = np.abs(part.cpu().numpy() - want).max()
+    if not e < 1e-6 * max(1.0, sigma * C_ * scale) + 2e-7 * np.abs(want).max():
+        bad.append(f"noise err {e:.3e}")
+    rest = torch.cat([buf[:off], buf[off + n:]])
+    if not torch.isfinite(rest).all():
+        bad.append("neighbours damaged")
+    return desc, bad
+
+
+def fused_noise_case(rng, k):
+    """grouped clipped sums with the noise drawn in the same call == plain sums + dp_add_noise"""
+    B = int(rng.integers(1, 5))
+    T = pick(rng, [16, 64, 100, 128, 200, 256])
+    n = int(rng.integers(1, 4))
+    lays, shapes = [], []
+    for _ in range(n):
+        d, p = rand_dim(rng), rand_dim(rng)
+        if int(rng.integers(4)) == 0:
+            p = pick(rng, [128 * 40, 128 * 100])             # enough tiles for the epilogue path
+        lda = W.round_up(d, 8) if d % 8 else None
+        ldg = W.round_up(p, 8) if p % 8 else None
+        A = W._normal((B, T, d), 1.0, "bf16", int(rng.integers(1 << 60)), ld=lda)
+        G = W._normal((B, T, p), 1e-2, "bf16", int(rng.integers(1 << 60)), ld=ldg)
+        lays.append(dp.Linear(P.to_device(A), P.to_device(G), d=d, p=p))
+        shapes.append((d, p))
+    desc = f"#{k} fused noise B{B} T{T} " + " ".join(f"{d}x{p}" for d, p in shapes)
+    bad = []
+    sq = torch.full((B,), float(rng.uniform(0.5, 8.0)), device=_dev())
+    tids = [int(rng.integers(0, 1000)) for _ in shapes]
+    seed, step = int(rng.integers(1 << 62)), int(rng.integers(1 << 20))
+    sigma, C_, scale = 0.8, float(rng.uniform(0.5, 2.0)), pick(rng, [1.0, 0.25])
+    fused = [torch.empty(p, d, device=_dev()) for d, p in shapes]
+    dp.dp_clip_accumulate_noise_grouped(lays, B, T, sq, C_, fused, sigma, scale, seed, tids, step)
+    plain = [torch.empty(p, d, device=_dev()) for d, p in shapes]
+    dp.dp_clip_accumulate_grouped(lays, B, T, sq, C_, plain)
+    sums = [t.clone() for t in plain]
+    torch.cuda.synchronize()
+    for f, s0, tid, (d, p) in zip(fused, sums, tids, shapes):
+        want = NO.add_noise(s0.cpu().numpy().astype(np.float64), sigma, C_, scale, seed, tid, step)
+        e = np.abs(f.cpu().numpy() - want).max()
+        if not e < 1e-6 * max(1.0, C_) + 1e-6 * np.abs(want).max():
+            bad.append(f"{d}x{p} err {e:.3e}")
+    return desc, bad
+
+
+def vector_case(rng, k):
+    dtype = pick(rng, ["bf16", "f32"])
+    B = int(rng.integers(1, 6))
+    T = pick(rng, [1, 16, 37, 100, 128, 300, 512])
+    n = int(rng.integers(1, 4))
+    prm, hosts = [], []
+    g_std = 1.0 if dtype == "f32" else 1e-2
+    for _ in range(n):
+        p = rand_dim(rng)
+        with_x = bool(rng.integers(2))
+        G = W._normal((B, T, p), g_std, dtype, int(rng.integers(1 << 60)))
+        X = W._normal((B, T, p), 1.0, dtype, int(rng.integers(1 << 60))) if with_x else None
+        prm.append(dp.Vector(P.to_device(G), P.to_device(X) if with_x else None, p=p))
+        hosts.append((G.widened(), X.widened() if with_x else None, p))
+    desc = f"#{k} vectors {dtype} B{B} T{T} " + " ".join(str(p) + ("x" if x is not None else "") for _, x, p in hosts)
+    bad = []
+    sq = torch.zeros(B, device=_dev())
+    dp.dp_vector_norms(prm, B, T, sq)
+    torch.cuda.synchronize()
+    want = sum(O.vector_sq_norms(g, x) for g, x, _ in hosts)
+    e = rel(sq.cpu().numpy(), want).max()
+    if not e < (1e-4 if dtype == "f32" else 2e-3):
+        bad.append(f"norm err {e:.3e}")
+    Cc = float(np.median(np.sqrt(want)))
+    sq_in = torch.from_numpy(want.astype(np.float32)).to(_dev())
+    _, R = O.clip_factors(sq_in.cpu().numpy().astype(np.float64), Cc)
+    beta = pick(rng, [0.0, 1.0])
+    outs0 = [torch.randn(p, device=_dev()) for _, _, p in hosts]
+    outs = [o.clone() for o in outs0]
+    dp.dp_clip_accumulate_vectors(prm, B, T, sq_in, Cc, outs, beta=beta)
+    torch.cuda.synchronize()
+    for (g, x, p), o, o0 in zip(hosts, outs, outs0):
+        w = O.clipped_sum_vector(g, x, R) + beta * o0.cpu().numpy().astype(np.float64)
+        fe = frob_rel(o.cpu().numpy(), w)
+        if not fe < 1e-5:
+            bad.append(f"sum err p{p} {fe:.3e}")
+    return desc, bad
+
 
 @pytest.mark.parametrize("case,n,seed", [(linear_case, 200, 101), (grouped_case, 80, 102),
-                                          (embed_case, 80, 103), (cross_case, 60, 104)])
+                                          (embed_case, 80, 103), (cross_case, 60, 104),
+                                          (noise_case, 150, 105), (fused_noise_case, 40, 106),
+                                          (vector_case, 80, 107)])
 def test_random_shapes_against_the_oracle(case, n, seed):
     rng = np.random.default_rng(seed)
     failures = []
