@@ -449,10 +449,24 @@ def run_ours(args):
         raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
+    reserve = args.reserve_sms
     if world > 1:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        # The collectives run beside persistent kernels that take every SM they are given (and all
+        # of its shared memory): cap the collectives' CTAs and leave them that many SMs.  With no
+        # free SM a collective waits for the end of the running launch and then delays part of the
+        # next one by a whole wave (measured on one GPU with a stand-in kernel: +36 % on the
+        # clipped-sum phase, against 3 % for 16 SMs set aside).
+        os.environ.setdefault("NCCL_MAX_CTAS", "16")
+        if reserve is None:
+            try:
+                reserve = max(0, int(os.environ["NCCL_MAX_CTAS"]))
+            except ValueError:
+                reserve = 16
         dist.init_process_group("nccl", device_id=dev)
     dp.load()
+    reserve = int(reserve or 0)
+    dp.dp_set_reserved_sms(reserve)
     peaks = measured_peaks()
 
     # every rank holds its own batch of the same shape (weak scaling over examples)
@@ -730,6 +744,7 @@ def run_ours(args):
                    "bias_and_layernorm_params": n_vec,
                    "accumulate": "fp32", "input_bytes_per_step": memory["input_bytes"],
                    "exchange": (args.exchange + (" + all_gather" if args.gather else "")) if world > 1 else None,
+                   "reserved_sms": reserve,
                    "l2": "inputs (%.2f GB per step) are larger than the 126 MB L2" % (memory["input_bytes"] / 1e9)},
         "phases_ms": {"norms": ms_norm, "clip_accumulate": ms_clip, "noise": ms_noise,
                       "norm_plus_clip": ms_norm + ms_clip,
@@ -874,6 +889,9 @@ def main():
                          "slice (default), or a blocking all-reduce per tensor followed by the noise pass")
     ap.add_argument("--gather", action="store_true",
                     help="N > 1, reduce_scatter: all-gather the noised slices back into the full tensors")
+    ap.add_argument("--reserve-sms", type=int, default=None,
+                    help="SMs left free of the library's persistent kernels (default: 0 at N = 1, "
+                         "NCCL_MAX_CTAS = 16 at N > 1, for the collectives)")
     ap.add_argument("--bucketed", action="store_true",
                     help="N = 1: run the multi-GPU step order (clipped sums bucket by bucket through the "
                          "exchange object, noise on the communication stream) on one GPU")

@@ -318,6 +318,14 @@ const char* dp_version(void);
 /* Number of CUDA kernels this library has enqueued since it was loaded (memsets and copies
  * are not counted).  Lets a caller report how many of its launches a timed region held. */
 int64_t dp_kernel_launches(void);
+/* Sets aside n SMs: every persistent kernel of the library (Gram, clipped-sum GEMM, cross term,
+ * bias / LayerNorm passes) then sizes its grid for the device's SM count less n, so that kernels
+ * of another stream -- the collectives of a data-parallel step, which cannot share an SM with
+ * CTAs that take all of its shared memory -- find free SMs while a long launch is running instead
+ * of waiting for its end.  Process-wide; applies to launches enqueued afterwards; the workspace
+ * sizes depend on it, so set it before asking for them.  0 (the default) uses every SM; values are
+ * clamped to [0, SMs - 2].  Returns the previous value.  Not part of the paper. */
+int32_t dp_set_reserved_sms(int32_t n);
 /* Test hook: when non-zero, linear-layer calls (DP_BF16 and DP_F32 alike) run the plain fp32-FMA
  * kernels instead of the tensor-core ones (used to cross-check the two on the device).  Returns
  * the previous value.  Off by default; not meant for production use. */

@@ -52,7 +52,7 @@ EXPORTS = ["dp_vector_norms", "dp_vector_norms_ws_bytes", "dp_clip_accumulate_ve
            "dp_last_cuda_error", "dp_version", "dp_kernel_launches", "dp_debug_force_fma",
            "dp_debug_noise_error_scan", "dp_debug_bounds_checked", "dp_debug_bounds_probe",
            "dp_debug_tensor_map_encodes", "dp_debug_set_wait_limit",
-           "dp_debug_ghost_single"]
+           "dp_debug_ghost_single", "dp_set_reserved_sms"]
 
 
 def lib_path() -> str:
@@ -134,6 +134,8 @@ def load():
     L.dp_debug_ghost_single.restype = i32
     L.dp_debug_force_fma.argtypes = [i32]
     L.dp_debug_force_fma.restype = i32
+    L.dp_set_reserved_sms.argtypes = [i32]
+    L.dp_set_reserved_sms.restype = i32
     for name in EXPORTS:
         fn = getattr(L, name)
         if fn.restype is C.c_int:          # ctypes default: the dp_status functions
@@ -525,6 +527,12 @@ def dp_sigma_for_epsilon(q: float, steps: int, target_epsilon: float, delta: flo
     _check(load().dp_sigma_for_epsilon(float(q), int(steps), float(target_epsilon), float(delta),
                                        float(tolerance), C.byref(sigma)), "dp_sigma_for_epsilon")
     return sigma.value
+
+
+def dp_set_reserved_sms(n: int) -> int:
+    """Leave n SMs free of the library's persistent kernels (for the collectives of another
+    stream); returns the previous setting."""
+    return int(load().dp_set_reserved_sms(int(n)))
 
 
 def dp_debug_ghost_single(on: bool) -> bool:

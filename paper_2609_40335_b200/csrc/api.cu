@@ -23,13 +23,14 @@ long long g_kernel_launches = 0;
 long long g_wait_limit = 1500000000LL;
 const uint32_t* g_step_dev = nullptr;
 int g_ghost_single = 0;
+int g_reserved_sms = 0;
 
 namespace {
 constexpr int kMaxDevices = 64;
 std::mutex g_device_mutex;
 }
 
-int sm_count() {
+static int device_sm_count() {
   static int n[kMaxDevices] = {};
   int dev = 0, v = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 148;
@@ -40,6 +41,13 @@ int sm_count() {
       return 148;          // B200; not cached so a later call can still query the device
   }
   return n[dev];
+}
+
+// SMs the persistent kernels size their grids for: all of the device's, less the ones the caller
+// set aside (dp_set_reserved_sms), kept even (CTA pairs) and never below two.
+int sm_count() {
+  const int n = device_sm_count() - g_reserved_sms;
+  return std::max(2, n & ~1);
 }
 
 bool first_use_on_this_device(const void* key) {
@@ -242,6 +250,11 @@ int32_t dp_last_cuda_error(void) { return g_last_cuda_error; }
 const char* dp_version(void) { return "dp_ghost 0.1.0 (sm_100a)"; }
 int64_t dp_kernel_launches(void) { return g_kernel_launches; }
 
+int32_t dp_set_reserved_sms(int32_t n) {
+  const int prev = g_reserved_sms;
+  g_reserved_sms = std::max(0, std::min(n, device_sm_count() - 2));
+  return prev;
+}
 int32_t dp_debug_ghost_single(int32_t on) {
   const int prev = g_ghost_single;
   g_ghost_single = on ? 1 : 0;

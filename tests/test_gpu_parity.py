@@ -905,6 +905,39 @@ def test_bucketed_clip_phase_equals_the_plain_phases(cfg):
         assert (lo, hi) == (0, a.outs[name].numel()) and mine.data_ptr() == b.outs[name].data_ptr()
 
 
+@pytest.mark.parametrize("reserve", [16, 1000])
+def test_reserved_sms_leave_the_results_unchanged(reserve):
+    """dp_set_reserved_sms: the persistent kernels run on fewer SMs (what a data-parallel step sets
+    so that its collectives find free SMs); every result still matches the oracle, with a second
+    kernel holding SMs on another stream while the step runs."""
+    prev = dp.dp_set_reserved_sms(reserve)
+    try:
+        assert prev == 0
+        w = W.named_workload("cfg3", B=3, T=256, n_blocks=2, V=3001)
+        ds = P.upload(w)
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            busy = torch.randn(4096, 4096, device=dev())
+            for _ in range(4):
+                busy = busy @ busy * 1e-2                   # keeps SMs busy beside the step
+        P.dp_step(ds, noise=False)
+        torch.cuda.synchronize()
+        check_status(ds.dev_status)
+        lin = [(l.A.widened(), l.G.widened()) for l in w.linears]
+        ref = O.dp_step(lin, w.ids, w.G_emb.widened(), w.V, w.C, lm=(w.lm.A.widened(), w.lm.G.widened()),
+                        tied=w.tied, positions=w.positions)
+        assert rel(ds.sq.cpu().numpy(), ref["sq"]).max() < TIGHT_BF16
+        for k, want in ref["sums"].items():
+            got = ds.outs[k].cpu().numpy()
+            if k == "wpe":
+                got = got[: w.T]
+            assert frob_rel(got, want) < TOL_SUM, k
+    finally:
+        back = dp.dp_set_reserved_sms(0)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    assert back == min(reserve, sms - 2)                    # clamped: at least one CTA pair stays
+
+
 # ------------------------------- full-size configurations in the launch configuration of the bench
 def _oracle_example(w, i):
     """The oracle's squared norm (and, tied, cross term) of example i over every layer of w."""
