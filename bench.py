@@ -871,6 +871,22 @@ def run_case(args):
             dp.dp_vector_norms(vec, B, T, sq)
             dp.dp_clip_accumulate_vectors(vec, B, T, sq, 1.0, outs)
         out.update(ms=timed(both))
+    elif c == "f32":
+        # fp32 inputs: the two-term bf16 split on the tensor cores against the plain fp32-FMA kernels
+        # (norm in both modes, clipped sum), 768 -> 3072 at B = 8, T = 128
+        B, T, d_, p_ = 8, 128, 768, 3072
+        A, G = torch.randn(B, T, d_, device="cuda"), torch.randn(B, T, p_, device="cuda") * 1e-2
+        sq = torch.zeros(B, device="cuda")
+        o = torch.empty(p_, d_, device="cuda")
+        clipsq = torch.full((B,), 4.0, device="cuda")
+        for name, on in (("tensor", False), ("fma", True)):
+            dp.dp_debug_force_fma(on)
+            for mode, key in ((dp.DP_NORM_GHOST, "ghost"), (dp.DP_NORM_DIRECT, "direct")):
+                L = [dp.Linear(A, G, mode=mode)]
+                out[f"{name}_{key}_norm_ms"] = timed(lambda: dp.dp_ghost_norms(L, B, T, sq))
+            out[f"{name}_clipped_sum_ms"] = timed(lambda: dp.dp_clip_accumulate(A, G, clipsq, 1.0, o))
+        dp.dp_debug_force_fma(False)
+        out["clipped_sum_TFLOPs_fp32_equivalent"] = 2 * B * T * d_ * p_ / out["tensor_clipped_sum_ms"] / 1e9
     else:
         raise SystemExit("unknown --case %r" % c)
     print(json.dumps(out), flush=True)
