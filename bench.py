@@ -627,12 +627,22 @@ def run_ours(args):
     ghost = ghost_norm_alone(dp, ds, peaks, peak_tf, counts)
     big = ds.outs["wte"]
     noise_n = big.numel()
-    noise_ms = time_graph(lambda: dp.dp_add_noise(big, ds.sigma, ds.C, 1.0, args.seed, 0, 0), reps=5)
+    noise_fn = lambda: dp.dp_add_noise(big, ds.sigma, ds.C, 1.0, args.seed, 0, 0)   # noqa: E731
+    noise_ms = time_graph(noise_fn, reps=5)
+    # the pass is bound by instruction issue, so it follows the SM clock: right after the timed
+    # steps the clock is what the power cap left of it; after a pause it is the idle boost clock
+    time.sleep(1.5)
+    noise_ms_rested = time_graph(noise_fn, reps=20)
     others = {
         "%s (dp_ghost_norms)" % ghost["kernel"]: ghost,
         "add_noise_kernel (dp_add_noise, %d elements)" % noise_n: {
-            "bound": "hbm", "ms": noise_ms, "achieved_GBs": 8 * noise_n / (noise_ms * 1e-3) / 1e9,
-            "peak_GBs": peaks["hbm_gbs"], "frac": 8 * noise_n / (noise_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+            "bound": "hbm", "note": "bound by instruction issue in practice (about 61 per element)",
+            "ms": noise_ms,
+            "achieved_GBs": 8 * noise_n / (noise_ms * 1e-3) / 1e9,
+            "peak_GBs": peaks["hbm_gbs"], "frac": 8 * noise_n / (noise_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+            "ms_after_1p5s_pause": noise_ms_rested,
+            "achieved_GBs_after_pause": 8 * noise_n / (noise_ms_rested * 1e-3) / 1e9,
+            "frac_after_pause": 8 * noise_n / (noise_ms_rested * 1e-3) / 1e9 / peaks["hbm_gbs"]},
     }
 
     # end to end through the public API with HOST buffers: every step copies the step's inputs
