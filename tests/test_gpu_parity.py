@@ -938,6 +938,26 @@ def test_reserved_sms_leave_the_results_unchanged(reserve):
     assert back == min(reserve, sms - 2)                    # clamped: at least one CTA pair stays
 
 
+@pytest.mark.parametrize("cfg", ["cfg3", "cfg4"])
+def test_repeated_steps_are_bitwise_identical(cfg):
+    """Race check: the same step (same seed and step word) issued 40 times gives the same bits in
+    every norm, clip factor and noised sum -- partial sums are combined in a fixed order everywhere,
+    so any difference would be an unordered access."""
+    w = W.named_workload(cfg, B=6, T=256 if cfg == "cfg3" else 128, n_blocks=2, V=5003)
+    ds = P.upload(w)
+    P.dp_step(ds, seed=5, step=7)
+    torch.cuda.synchronize()
+    ref = {k: v.clone() for k, v in ds.outs.items()}
+    ref_sq, ref_clip = ds.sq.clone(), ds.clip.clone()
+    for _ in range(40):
+        P.dp_step(ds, seed=5, step=7)
+    torch.cuda.synchronize()
+    check_status(ds.dev_status)
+    assert torch.equal(ds.sq, ref_sq) and torch.equal(ds.clip, ref_clip)
+    for k in ref:
+        assert torch.equal(ds.outs[k], ref[k]), k
+
+
 # ------------------------------- full-size configurations in the launch configuration of the bench
 def _oracle_example(w, i):
     """The oracle's squared norm (and, tied, cross term) of example i over every layer of w."""
